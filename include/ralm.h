@@ -1,0 +1,143 @@
+/* ralm.h -- C ABI of the exact dense retrieval library for sm_100a (NVIDIA B200).
+ *
+ * The library implements the retrieval calls of RaLMSpec's serving loop (Algorithm 1):
+ *
+ *   C.retrieve(q_1..q_s)      -> ralm_search        batched verification retrieval with an
+ *                                                   exact dense retriever (Algorithm 1,
+ *                                                   batched verification step; Section 3,
+ *                                                   "Batched verification")
+ *   Q.retrieve(q_i)           -> ralm_cache_search  speculative retrieval from a request's
+ *                                                   local cache, ranked with the retriever's
+ *                                                   own metric (Algorithm 1, speculative
+ *                                                   retrieval step; Section 3, "Speculative
+ *                                                   retrieval"; Fig. 3)
+ *   m = argmin_i d^_i != d_i  -> ralm_verify        first mis-speculated position
+ *                                                   (Algorithm 1, verification step; toy
+ *                                                   example of Section 3)
+ *
+ * Conventions
+ *   - Every call returns a ralm_status_t; nothing throws, aborts or prints.
+ *   - Argument errors are detected on the host before any launch.
+ *   - Calls taking a `stream` (a cudaStream_t passed as void*, NULL = default stream) only
+ *     enqueue work; outputs are valid once the stream has reached that point.
+ *   - All fp16 data is IEEE binary16 and must be finite.
+ *   - Ranking is a total order: inner product (score descending, id ascending); L2
+ *     (squared distance ascending, id ascending). L2 scores are SQUARED distances.
+ *   - When fewer than k rows qualify, trailing slots hold id -1 and score -inf (inner
+ *     product) or +inf (L2).
+ *   - Scores are accumulated in fp32.
+ *   - One index may be used from one stream at a time (its workspace is shared by calls).
+ *   - Device-side anomalies (an out-of-range cache id, a wait that ran out) set a sticky
+ *     status word that ralm_device_status reads.
+ */
+#ifndef RALM_H_
+#define RALM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ralm_index ralm_index_t; /* opaque */
+
+typedef enum { RALM_IP = 0, RALM_L2 = 1 } ralm_metric_t;
+
+typedef enum {
+    RALM_OK = 0,
+    RALM_ERR_INVALID_ARG = 1,
+    RALM_ERR_OOM = 2,
+    RALM_ERR_CUDA = 3,
+    RALM_ERR_TIMEOUT = 4,
+    RALM_ERR_UNSUPPORTED = 5,
+    RALM_ERR_BAD_CACHE_ID = 6
+} ralm_status_t;
+
+/* Limits checked by the host side. */
+#define RALM_MAX_K 1024       /* neighbours per query (the KNN-LM evaluation's largest k) */
+#define RALM_MAX_D 4096       /* vector dimension */
+#define RALM_MAX_QUERIES 4096 /* queries per ralm_search call */
+#define RALM_MAX_CACHE 4096   /* cache slots per request */
+#define RALM_MAX_CACHE_KEYS (1 << 20) /* R * q * (C rounded up to a power of two) per call */
+
+/* Create an index over a corpus that is already resident in device memory.
+ *   corpus  DEVICE pointer, fp16 [N][d] row-major, 16-byte aligned, d % 8 == 0,
+ *           8 <= d <= RALM_MAX_D, 0 <= N < 2^31. BORROWED: never copied; the caller keeps it
+ *           alive and unmodified until ralm_index_destroy. May be NULL only when N == 0.
+ *   metric  RALM_IP (QA dense retriever) or RALM_L2 (KNN-LM datastore).
+ *   max_s   largest number of queries a later ralm_search will pass (1..RALM_MAX_QUERIES).
+ *   max_k   largest k a later call will pass (1..RALM_MAX_K).
+ *   out     receives the handle (host memory owned by the library).
+ * Allocates the per-index device workspace (partial top-k lists, staging buffers, status
+ * word) on the current device. Synchronous.
+ * Errors: INVALID_ARG (null pointer, misaligned corpus, bad sizes), OOM, CUDA,
+ * UNSUPPORTED (device is not compute capability 10.x). */
+ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_metric_t metric,
+                                int32_t max_s, int32_t max_k, ralm_index_t **out);
+
+/* Free the workspace and the handle. The corpus is untouched. NULL is accepted. */
+ralm_status_t ralm_index_destroy(ralm_index_t *idx);
+
+/* C.retrieve(q_1..q_s): exact top-k of s queries over the whole corpus, one stream of the
+ * corpus from HBM per group of up to 8 queries.
+ *   queries DEVICE fp16 [s][d], 16-byte aligned.     0 <= s <= max_s
+ *   ids     DEVICE int64 [s][k]  (written)           1 <= k <= max_k
+ *   scores  DEVICE fp32  [s][k]  (written)
+ * Asynchronous on `stream`. s == 0 is a no-op. */
+ralm_status_t ralm_search(ralm_index_t *idx, const void *queries, int32_t s, int32_t k,
+                          int64_t *ids, float *scores, void *stream);
+
+/* Same as ralm_search with HOST buffers: copies the queries to the device, searches, copies
+ * ids and scores back, and returns after the results are in host memory (synchronises
+ * `stream`). Pinned host memory makes the copies asynchronous up to that point. */
+ralm_status_t ralm_search_host(ralm_index_t *idx, const void *queries_host, int32_t s,
+                               int32_t k, int64_t *ids_host, float *scores_host, void *stream);
+
+/* Q.retrieve for R requests at once: request r owns C cache slots holding corpus ids
+ * (-1 = empty slot; the cache is a set, a repeated id counts once) and q queries; each
+ * query is ranked against that request's cached rows only, with the index's metric and the
+ * same total order as ralm_search.
+ *   cache_ids DEVICE int64 [R][C]       queries DEVICE fp16 [R][q][d], 16-byte aligned
+ *   ids       DEVICE int64 [R][q][k]    scores  DEVICE fp32 [R][q][k]
+ *   1 <= C <= RALM_MAX_CACHE, 1 <= q, 1 <= k <= max_k,
+ *   R * q * pow2ceil(C) <= RALM_MAX_CACHE_KEYS. R == 0 is a no-op.
+ * An id outside [-1, N) is skipped and sets RALM_ERR_BAD_CACHE_ID in the status word.
+ * Asynchronous on `stream`. */
+ralm_status_t ralm_cache_search(ralm_index_t *idx, const int64_t *cache_ids, int32_t R,
+                                int32_t C, const void *queries, int32_t q, int32_t k,
+                                int64_t *ids, float *scores, void *stream);
+
+/* Verification: first_mismatch[r] = the smallest step i in [0, stride) at which any of the
+ * first cmp_k speculated ids differs from the retrieved ones, or `stride` if every step
+ * matches (0-based; Algorithm 1's "m <= s" becomes first_mismatch < stride).
+ *   speculated_ids DEVICE int64 [R][stride][cmp_k]
+ *   retrieved_ids  DEVICE int64 [R][stride][ld]   (ld = k of the search that produced them)
+ *   first_mismatch DEVICE int32 [R] (written)
+ *   `stride` is the speculation stride s of the paper, not a memory pitch.
+ *   1 <= cmp_k <= ld; cmp_k == 1 compares the top-ranked document only.
+ * Needs no index. Asynchronous on `stream`. R == 0 or stride == 0 are accepted. */
+ralm_status_t ralm_verify(const int64_t *speculated_ids, const int64_t *retrieved_ids, int32_t R,
+                          int32_t stride, int32_t ld, int32_t cmp_k, int32_t *first_mismatch,
+                          void *stream);
+
+/* Synchronise `stream`, read and clear the index's sticky device status word. Returns
+ * RALM_OK, RALM_ERR_TIMEOUT, RALM_ERR_BAD_CACHE_ID, or RALM_ERR_CUDA if the stream itself
+ * reports an error. */
+ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
+
+/* Pin the scan variant used by ralm_search on this index (benchmarking aid).
+ *   0 = automatic, 1 = FMA scan (fp32 FMAs, any metric), 2 = warp-MMA scan (inner product,
+ *   up to 8 queries per pass), 3 = tcgen05 scan (inner product, large batches).
+ * UNSUPPORTED if the variant cannot serve the index's metric or dimension. */
+ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant);
+
+/* Number of kernels the library launched on behalf of this index since creation. */
+int64_t ralm_index_launch_count(const ralm_index_t *idx);
+
+/* Static description of a status code. */
+const char *ralm_status_string(ralm_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RALM_H_ */

@@ -1,0 +1,178 @@
+"""ctypes marshalling for libralm.so; names follow include/ralm.h."""
+import ctypes
+import os
+
+import torch
+
+IP = 0
+L2 = 1
+
+STATUS_NAMES = {0: "RALM_OK", 1: "RALM_ERR_INVALID_ARG", 2: "RALM_ERR_OOM", 3: "RALM_ERR_CUDA",
+                4: "RALM_ERR_TIMEOUT", 5: "RALM_ERR_UNSUPPORTED", 6: "RALM_ERR_BAD_CACHE_ID"}
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_lib = None
+
+
+class RalmError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s" % (where, STATUS_NAMES.get(status, str(status))))
+
+
+def lib_path() -> str:
+    return os.path.join(_HERE, "libralm.so")
+
+
+def load_library() -> ctypes.CDLL:
+    """Load the compiled CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = lib_path()
+    if not os.path.exists(path):
+        raise RuntimeError("%s is missing: build it with `python -m paper_2401_14021_b200.build` "
+                           "(there is no CPU fallback)" % path)
+    lib = ctypes.CDLL(path)
+    i32, i64, p = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p
+    lib.ralm_index_create.restype = i32
+    lib.ralm_index_create.argtypes = [p, i64, i32, i32, i32, i32, ctypes.POINTER(p)]
+    lib.ralm_index_destroy.restype = i32
+    lib.ralm_index_destroy.argtypes = [p]
+    lib.ralm_search.restype = i32
+    lib.ralm_search.argtypes = [p, p, i32, i32, p, p, p]
+    lib.ralm_search_host.restype = i32
+    lib.ralm_search_host.argtypes = [p, p, i32, i32, p, p, p]
+    lib.ralm_cache_search.restype = i32
+    lib.ralm_cache_search.argtypes = [p, p, i32, i32, p, i32, i32, p, p, p]
+    lib.ralm_verify.restype = i32
+    lib.ralm_verify.argtypes = [p, p, i32, i32, i32, i32, p, p]
+    lib.ralm_device_status.restype = i32
+    lib.ralm_device_status.argtypes = [p, p]
+    lib.ralm_index_set_variant.restype = i32
+    lib.ralm_index_set_variant.argtypes = [p, i32]
+    lib.ralm_index_launch_count.restype = i64
+    lib.ralm_index_launch_count.argtypes = [p]
+    lib.ralm_status_string.restype = ctypes.c_char_p
+    lib.ralm_status_string.argtypes = [i32]
+    _lib = lib
+    return lib
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise RalmError(status, where)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError("%s must be a contiguous CUDA tensor of %s" % (name, dtype))
+    return t.data_ptr()
+
+
+class Index:
+    """ralm_index_create / ralm_index_destroy. Keeps a reference to the corpus tensor."""
+
+    def __init__(self, corpus: torch.Tensor, metric: int, max_s: int = 8, max_k: int = 32):
+        self._lib = load_library()
+        self._handle = ctypes.c_void_p()
+        if corpus.dim() != 2:
+            raise TypeError("corpus must be [N][d]")
+        ptr = _dev(corpus, torch.float16, "corpus") if corpus.numel() else 0
+        self.corpus = corpus
+        self.N, self.d = corpus.shape
+        self.metric = metric
+        self.max_s, self.max_k = max_s, max_k
+        with torch.cuda.device(corpus.device):
+            _check(self._lib.ralm_index_create(ptr, self.N, self.d, metric, max_s, max_k,
+                                               ctypes.byref(self._handle)), "ralm_index_create")
+
+    def close(self):
+        if self._handle:
+            self._lib.ralm_index_destroy(self._handle)
+            self._handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def handle(self):
+        return self._handle
+
+    def set_variant(self, variant: int):
+        _check(self._lib.ralm_index_set_variant(self._handle, variant), "ralm_index_set_variant")
+
+    def launch_count(self) -> int:
+        return self._lib.ralm_index_launch_count(self._handle)
+
+    def device_status(self, stream=None) -> int:
+        return self._lib.ralm_device_status(self._handle, _stream_ptr(stream))
+
+
+def search(index: Index, queries: torch.Tensor, k: int, ids: torch.Tensor = None,
+           scores: torch.Tensor = None, stream=None):
+    """ralm_search: queries fp16 [s][d] on the device -> (ids int64 [s][k], scores fp32 [s][k])."""
+    s = queries.shape[0]
+    if ids is None:
+        ids = torch.empty((s, k), dtype=torch.int64, device=queries.device)
+    if scores is None:
+        scores = torch.empty((s, k), dtype=torch.float32, device=queries.device)
+    qp = _dev(queries, torch.float16, "queries") if s else 0
+    _check(index._lib.ralm_search(index.handle, qp, s, k, _dev(ids, torch.int64, "ids") if s else 0,
+                                  _dev(scores, torch.float32, "scores") if s else 0,
+                                  _stream_ptr(stream)), "ralm_search")
+    return ids, scores
+
+
+def search_host(index: Index, queries: torch.Tensor, k: int, ids: torch.Tensor, scores: torch.Tensor,
+                stream=None):
+    """ralm_search_host: all three tensors live in (preferably pinned) host memory."""
+    s = queries.shape[0]
+    for t, dt in ((queries, torch.float16), (ids, torch.int64), (scores, torch.float32)):
+        if t.is_cuda or t.dtype != dt or not t.is_contiguous():
+            raise TypeError("host tensors must be contiguous CPU tensors of the right dtype")
+    _check(index._lib.ralm_search_host(index.handle, queries.data_ptr(), s, k, ids.data_ptr(),
+                                       scores.data_ptr(), _stream_ptr(stream)), "ralm_search_host")
+    return ids, scores
+
+
+def cache_search(index: Index, cache_ids: torch.Tensor, queries: torch.Tensor, k: int,
+                 ids: torch.Tensor = None, scores: torch.Tensor = None, stream=None):
+    """ralm_cache_search: cache_ids int64 [R][C], queries fp16 [R][q][d]."""
+    R, C = cache_ids.shape
+    q = queries.shape[1]
+    if ids is None:
+        ids = torch.empty((R, q, k), dtype=torch.int64, device=queries.device)
+    if scores is None:
+        scores = torch.empty((R, q, k), dtype=torch.float32, device=queries.device)
+    _check(index._lib.ralm_cache_search(index.handle, _dev(cache_ids, torch.int64, "cache_ids") if R else 0,
+                                        R, C, _dev(queries, torch.float16, "queries") if R else 0, q, k,
+                                        _dev(ids, torch.int64, "ids") if R else 0,
+                                        _dev(scores, torch.float32, "scores") if R else 0,
+                                        _stream_ptr(stream)), "ralm_cache_search")
+    return ids, scores
+
+
+def verify(speculated_ids: torch.Tensor, retrieved_ids: torch.Tensor, cmp_k: int = 1,
+           first_mismatch: torch.Tensor = None, stream=None):
+    """ralm_verify: speculated int64 [R][stride] (or [R][stride][cmp_k]); retrieved int64
+    [R][stride][ld] (or [R][stride], ld = 1) -> first_mismatch int32 [R]."""
+    load_library()
+    R, stride = speculated_ids.shape[0], speculated_ids.shape[1]
+    ld = retrieved_ids.shape[2] if retrieved_ids.dim() == 3 else 1
+    if first_mismatch is None:
+        first_mismatch = torch.empty((R,), dtype=torch.int32, device=speculated_ids.device)
+    sp = _dev(speculated_ids, torch.int64, "speculated_ids") if speculated_ids.numel() else 0
+    rp = _dev(retrieved_ids, torch.int64, "retrieved_ids") if retrieved_ids.numel() else 0
+    fp = _dev(first_mismatch, torch.int32, "first_mismatch") if R else 0
+    _check(_lib.ralm_verify(sp, rp, R, stride, ld, cmp_k, fp, _stream_ptr(stream)), "ralm_verify")
+    return first_mismatch

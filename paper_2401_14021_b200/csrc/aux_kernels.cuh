@@ -1,0 +1,214 @@
+// Small kernels beside the scan: cross-CTA merge of partial top-k lists, the per-request
+// speculation-cache lookup (score + rank) and the first-mismatch verification.
+#pragma once
+
+#include "common.cuh"
+
+namespace ralm {
+
+constexpr int kMergeThreads = 1024;
+constexpr int kMergeSortMax = 4096;  // keys sorted in one go when all lists fit
+
+__device__ __forceinline__ void write_result(uint64_t key, bool l2, int64_t *id_out,
+                                             float *score_out) {
+    if (key == 0ull) {
+        *id_out = -1;
+        *score_out = l2 ? INFINITY : -INFINITY;
+    } else {
+        *id_out = static_cast<int64_t>(key_row(key));
+        const float v = key_value(key);
+        *score_out = l2 ? (0.0f - v) : v;
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Merge: one CTA per query. `partial` holds B lists of k keys, each sorted descending and
+// padded with 0, laid out [B][s][k]. Writes ids [s][k] (int64) and scores [s][k] (fp32).
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kMergeThreads, 1)
+merge_kernel(const uint64_t *__restrict__ partial, int B, int s, int k, int l2,
+             int64_t *__restrict__ ids, float *__restrict__ scores) {
+    __shared__ uint64_t buf[kMergeSortMax];
+    const int q = blockIdx.x;
+    const int tid = threadIdx.x;
+    const long long total = static_cast<long long>(B) * k;
+    if (total <= kMergeSortMax) {
+        const int P = next_pow2(total > 1 ? static_cast<int>(total) : 2);
+        for (int i = tid; i < P; i += kMergeThreads) {
+            uint64_t key = 0;
+            if (i < total) {
+                const int b = i / k, j = i - b * k;
+                key = partial[(static_cast<size_t>(b) * s + q) * k + j];
+            }
+            buf[i] = key;
+        }
+        __syncthreads();
+        bitonic_sort_desc(buf, P, tid, kMergeThreads, -1);
+    } else {
+        // running best list merged with one sorted list at a time: the element-wise maximum
+        // of a descending list and a reversed descending list holds the best P keys of both
+        // and is bitonic
+        const int P = next_pow2(k);
+        for (int i = tid; i < P; i += kMergeThreads)
+            buf[i] = (i < k) ? partial[(static_cast<size_t>(q)) * k + i] : 0ull;
+        __syncthreads();
+        for (int b = 1; b < B; ++b) {
+            const uint64_t *list = partial + (static_cast<size_t>(b) * s + q) * k;
+            for (int i = tid; i < P; i += kMergeThreads) {
+                const int j = P - 1 - i;
+                const uint64_t other = (j < k) ? list[j] : 0ull;
+                const uint64_t mine = buf[i];
+                buf[i] = mine > other ? mine : other;
+            }
+            __syncthreads();
+            bitonic_merge_desc(buf, P, tid, kMergeThreads, -1);
+        }
+    }
+    for (int i = tid; i < k; i += kMergeThreads) {
+        const uint64_t key = (i < total) ? buf[i] : 0ull;
+        write_result(key, l2 != 0, ids + static_cast<size_t>(q) * k + i,
+                     scores + static_cast<size_t>(q) * k + i);
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Cache lookup, step 1: score. One warp per (request, cache slot); the warp scores its
+// cached corpus row against up to 8 of the request's queries at a time and stores one key
+// per query in keys[r][u][c] (Cp = C rounded up to a power of two; slots >= C hold 0).
+// grid = (ceil(Cp / slots_per_cta), R), block = 256.
+// ------------------------------------------------------------------------------------
+constexpr int kCacheThreads = 256;
+constexpr int kCacheSlotsPerCta = 32;
+
+__global__ void __launch_bounds__(kCacheThreads)
+cache_score_kernel(const __half *__restrict__ corpus, long long N, int d, int l2,
+                   const int64_t *__restrict__ cache_ids, int C, int Cp,
+                   const __half *__restrict__ queries, int q, uint64_t *__restrict__ keys,
+                   int *status) {
+    const int r = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pieces = d >> 3;
+    for (int c = blockIdx.x * kCacheSlotsPerCta + warp; c < (blockIdx.x + 1) * kCacheSlotsPerCta && c < Cp;
+         c += kCacheThreads / 32) {
+        long long id = -1;
+        if (c < C) id = cache_ids[static_cast<size_t>(r) * C + c];
+        const bool valid = id >= 0 && id < N;
+        if (c < C && !valid && id != -1 && lane == 0) atomicMax(status, kStatusBadCacheId);
+        const __half *row = corpus + (valid ? id : 0) * d;
+        for (int u0 = 0; u0 < q; u0 += 8) {
+            float acc[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+            if (valid) {
+                for (int pc = lane; pc < pieces; pc += 32) {
+                    const uint4 raw = *reinterpret_cast<const uint4 *>(row + pc * 8);
+                    const uint32_t xw[4] = {raw.x, raw.y, raw.z, raw.w};
+                    float2 x[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        x[e] = __half22float2(*reinterpret_cast<const __half2 *>(&xw[e]));
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (u0 + j < q) {
+                            const uint4 qr = *reinterpret_cast<const uint4 *>(
+                                queries + (static_cast<size_t>(r) * q + u0 + j) * d + pc * 8);
+                            const uint32_t qw[4] = {qr.x, qr.y, qr.z, qr.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float2 qv =
+                                    __half22float2(*reinterpret_cast<const __half2 *>(&qw[e]));
+                                if (l2) {
+                                    const float dx = x[e].x - qv.x, dy = x[e].y - qv.y;
+                                    acc[j] = fmaf(dx, dx, acc[j]);
+                                    acc[j] = fmaf(dy, dy, acc[j]);
+                                } else {
+                                    acc[j] = fmaf(x[e].x, qv.x, acc[j]);
+                                    acc[j] = fmaf(x[e].y, qv.y, acc[j]);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+            }
+            if (lane < 8 && u0 + lane < q) {
+                float v = 0.f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (j == lane) v = acc[j];
+                if (l2) v = 0.0f - v;
+                keys[(static_cast<size_t>(r) * q + u0 + lane) * Cp + c] =
+                    valid ? make_key(v, static_cast<uint32_t>(id)) : 0ull;
+            }
+        }
+    }
+}
+
+// Cache lookup, step 2: rank. One CTA per (request, query): sort the Cp keys, drop repeated
+// ids (equal keys are adjacent after the sort), write the best k.
+__global__ void __launch_bounds__(kMergeThreads, 1)
+cache_rank_kernel(const uint64_t *__restrict__ keys, int Cp, int k, int l2,
+                  int64_t *__restrict__ ids, float *__restrict__ scores) {
+    __shared__ uint64_t buf[kMergeSortMax];
+    __shared__ int warp_total[kMergeSortMax / 32];
+    const int tid = threadIdx.x;
+    const size_t ru = blockIdx.x;
+    const int P = Cp < 2 ? 2 : Cp;
+    for (int i = tid; i < P; i += kMergeThreads) buf[i] = (i < Cp) ? keys[ru * Cp + i] : 0ull;
+    __syncthreads();
+    bitonic_sort_desc(buf, P, tid, kMergeThreads, -1);
+    // keep[i]: a real key that differs from its predecessor
+    const int lane = tid & 31;
+    const int chunks = (P + 31) / 32;  // 32-element chunks, one per warp iteration
+    for (int ch = tid >> 5; ch < chunks; ch += kMergeThreads / 32) {
+        const int i = ch * 32 + lane;
+        const bool keep = i < P && buf[i] != 0ull && (i == 0 || buf[i] != buf[i - 1]);
+        const unsigned m = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) warp_total[ch] = __popc(m);
+    }
+    __syncthreads();
+    for (int i = tid; i < k; i += kMergeThreads) {
+        ids[ru * k + i] = -1;
+        scores[ru * k + i] = l2 ? INFINITY : -INFINITY;
+    }
+    __syncthreads();
+    for (int ch = tid >> 5; ch < chunks; ch += kMergeThreads / 32) {
+        const int i = ch * 32 + lane;
+        const bool keep = i < P && buf[i] != 0ull && (i == 0 || buf[i] != buf[i - 1]);
+        const unsigned m = __ballot_sync(0xffffffffu, keep);
+        int base = 0;
+        for (int c2 = 0; c2 < ch; ++c2) base += warp_total[c2];
+        const int rank = base + __popc(m & ((1u << lane) - 1u));
+        if (keep && rank < k) write_result(buf[i], l2 != 0, ids + ru * k + rank, scores + ru * k + rank);
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Verification: one warp per request; lanes take speculation steps 32 at a time.
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+verify_kernel(const int64_t *__restrict__ spec, const int64_t *__restrict__ retr, int R, int stride,
+              int ld, int cmp_k, int *__restrict__ first_mismatch) {
+    const int r = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (r >= R) return;
+    int m = stride;
+    for (int base = 0; base < stride && m == stride; base += 32) {
+        const int i = base + lane;
+        bool differ = false;
+        if (i < stride) {
+            const int64_t *a = spec + (static_cast<size_t>(r) * stride + i) * cmp_k;
+            const int64_t *b = retr + (static_cast<size_t>(r) * stride + i) * ld;
+            for (int c = 0; c < cmp_k; ++c) differ |= (a[c] != b[c]);
+        }
+        const unsigned mask = __ballot_sync(0xffffffffu, differ);
+        if (mask) m = base + __ffs(mask) - 1;
+    }
+    if (lane == 0) first_mismatch[r] = m;
+}
+
+}  // namespace ralm

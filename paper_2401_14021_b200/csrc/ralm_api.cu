@@ -1,0 +1,318 @@
+// Host side of the C ABI declared in include/ralm.h: argument checks, workspace, variant
+// dispatch and launches. All device work is in the kernels included below.
+#include "../../include/ralm.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <new>
+
+#include "aux_kernels.cuh"
+#include "scan.cuh"
+
+using namespace ralm;
+
+struct ralm_index {
+    const __half *corpus;
+    int64_t N;
+    int32_t d;
+    ralm_metric_t metric;
+    int32_t max_s, max_k;
+    int device;
+    int num_sms;
+    int smem_optin;
+    int variant;  // 0 auto, 1 FMA, 2 warp-MMA, 3 tcgen05
+    uint64_t *partial;   // [num_sms][max_s][max_k]
+    uint64_t *cache_keys;  // [RALM_MAX_CACHE_KEYS]
+    int *status;
+    // staging for the host-buffer entry point
+    __half *h_queries;
+    int64_t *h_ids;
+    float *h_scores;
+    int64_t launches;
+};
+
+namespace {
+
+struct ScanPlan {
+    int nstages, stage_bytes, cap, off_q, off_cand, off_stage, smem_bytes;
+};
+
+int align_up(int v, int a) { return (v + a - 1) / a * a; }
+
+// Shared-memory layout of one scan CTA. Returns false if not even one stage fits.
+bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl) {
+    pl->stage_bytes = align_up(kTileRows * idx->d * 2, 128);
+    pl->off_q = kScanHeaderBytes;
+    int off = pl->off_q + (mma ? align_up(kScanMaxQueries * idx->d * 2, 128) : 0);
+    pl->off_cand = off;
+    pl->cap = 0;
+    if (k > 1) {
+        pl->cap = std::max(512, 2 * next_pow2(k));
+        off += s_pass * pl->cap * 8;
+    }
+    pl->off_stage = align_up(off, 128);
+    const int room = idx->smem_optin - pl->off_stage;
+    if (room < pl->stage_bytes) return false;
+    pl->nstages = std::min(kMaxStages, room / pl->stage_bytes);
+    pl->smem_bytes = pl->off_stage + pl->nstages * pl->stage_bytes;
+    return true;
+}
+
+template <bool MMA, bool L2, int SQ, int DP, bool TOP1>
+cudaError_t launch_scan(const ScanParams &p, int grid, int smem, cudaStream_t st) {
+    auto kern = scan_kernel<MMA, L2, SQ, DP, TOP1>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, 32 * (p.nstages + 1), smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+template <bool L2, int SQ, bool TOP1>
+cudaError_t launch_fma_dp(const ScanParams &p, int grid, int smem, cudaStream_t st) {
+    if (p.d <= 256) return launch_scan<false, L2, SQ, 1, TOP1>(p, grid, smem, st);
+    if (p.d <= 768) return launch_scan<false, L2, SQ, 3, TOP1>(p, grid, smem, st);
+    return launch_scan<false, L2, SQ, 4, TOP1>(p, grid, smem, st);
+}
+
+template <bool L2>
+cudaError_t launch_fma(const ScanParams &p, int grid, int smem, cudaStream_t st) {
+    const bool top1 = p.k == 1;
+    if (p.s == 1)
+        return top1 ? launch_fma_dp<L2, 1, true>(p, grid, smem, st)
+                    : launch_fma_dp<L2, 1, false>(p, grid, smem, st);
+    return top1 ? launch_fma_dp<L2, 4, true>(p, grid, smem, st)
+                : launch_fma_dp<L2, 4, false>(p, grid, smem, st);
+}
+
+constexpr int kFmaMaxD = 1024;
+constexpr int kFmaQueriesPerPass = 4;
+
+// Which scan serves this index: 1 = FMA, 2 = warp-MMA.
+int resolve_variant(const ralm_index *idx) {
+    if (idx->variant == 1 || idx->variant == 2) return idx->variant;
+    return idx->metric == RALM_IP ? 2 : 1;
+}
+
+ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k, int64_t *ids,
+                            float *scores, cudaStream_t st) {
+    if (s == 0) return RALM_OK;
+    const int variant = resolve_variant(idx);
+    const bool mma = variant == 2;
+    if (!mma && idx->d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
+    const int per_pass = mma ? kScanMaxQueries : kFmaQueriesPerPass;
+    const long long ntiles = (idx->N + kTileRows - 1) / kTileRows;
+    const int grid = static_cast<int>(std::min<long long>(idx->num_sms, ntiles));
+    if (grid > 0) {
+        for (int q0 = 0; q0 < s; q0 += per_pass) {
+            const int sp = std::min(per_pass, s - q0);
+            ScanPlan pl;
+            if (!plan_scan(idx, mma, sp, k, &pl)) return RALM_ERR_UNSUPPORTED;
+            ScanParams p;
+            p.corpus = idx->corpus;
+            p.queries = queries + static_cast<size_t>(q0) * idx->d;
+            p.partial = idx->partial;
+            p.status = idx->status;
+            p.N = idx->N;
+            p.ntiles = ntiles;
+            p.d = idx->d;
+            p.s = sp;
+            p.s_total = s;
+            p.q_base = q0;
+            p.k = k;
+            p.cap = pl.cap;
+            p.nstages = pl.nstages;
+            p.stage_bytes = pl.stage_bytes;
+            p.off_q = pl.off_q;
+            p.off_cand = pl.off_cand;
+            p.off_stage = pl.off_stage;
+            cudaError_t e;
+            if (mma) {
+                e = (k == 1) ? launch_scan<true, false, 8, 1, true>(p, grid, pl.smem_bytes, st)
+                             : launch_scan<true, false, 8, 1, false>(p, grid, pl.smem_bytes, st);
+            } else if (idx->metric == RALM_L2) {
+                e = launch_fma<true>(p, grid, pl.smem_bytes, st);
+            } else {
+                e = launch_fma<false>(p, grid, pl.smem_bytes, st);
+            }
+            if (e != cudaSuccess) return RALM_ERR_CUDA;
+            idx->launches++;
+        }
+    }
+    merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, idx->metric == RALM_L2, ids,
+                                              scores);
+    if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
+    idx->launches++;
+    return RALM_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_metric_t metric,
+                                int32_t max_s, int32_t max_k, ralm_index_t **out) {
+    if (!out) return RALM_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (N < 0 || N >= (int64_t{1} << 31)) return RALM_ERR_INVALID_ARG;
+    if (!corpus && N > 0) return RALM_ERR_INVALID_ARG;
+    if (!aligned16(corpus)) return RALM_ERR_INVALID_ARG;
+    if (d < 8 || d > RALM_MAX_D || d % 8 != 0) return RALM_ERR_INVALID_ARG;
+    if (metric != RALM_IP && metric != RALM_L2) return RALM_ERR_INVALID_ARG;
+    if (max_s < 1 || max_s > RALM_MAX_QUERIES || max_k < 1 || max_k > RALM_MAX_K)
+        return RALM_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RALM_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return RALM_ERR_CUDA;
+    if (prop.major != 10) return RALM_ERR_UNSUPPORTED;
+    ralm_index *idx = new (std::nothrow) ralm_index();
+    if (!idx) return RALM_ERR_OOM;
+    idx->corpus = static_cast<const __half *>(corpus);
+    idx->N = N;
+    idx->d = d;
+    idx->metric = metric;
+    idx->max_s = max_s;
+    idx->max_k = max_k;
+    idx->device = dev;
+    idx->num_sms = prop.multiProcessorCount;
+    idx->smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
+    idx->variant = 0;
+    idx->launches = 0;
+    const size_t partial_bytes = sizeof(uint64_t) * idx->num_sms * max_s * static_cast<size_t>(max_k);
+    const size_t sk = static_cast<size_t>(max_s) * max_k;
+    bool ok = cudaMalloc(&idx->partial, partial_bytes) == cudaSuccess;
+    ok = ok && cudaMalloc(&idx->cache_keys, sizeof(uint64_t) * RALM_MAX_CACHE_KEYS) == cudaSuccess;
+    ok = ok && cudaMalloc(&idx->status, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&idx->h_queries, static_cast<size_t>(max_s) * d * 2) == cudaSuccess;
+    ok = ok && cudaMalloc(&idx->h_ids, sk * sizeof(int64_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&idx->h_scores, sk * sizeof(float)) == cudaSuccess;
+    if (!ok) {
+        const bool oom = cudaGetLastError() == cudaErrorMemoryAllocation;
+        ralm_index_destroy(idx);
+        return oom ? RALM_ERR_OOM : RALM_ERR_CUDA;
+    }
+    if (cudaMemset(idx->status, 0, sizeof(int)) != cudaSuccess) {
+        ralm_index_destroy(idx);
+        return RALM_ERR_CUDA;
+    }
+    *out = idx;
+    return RALM_OK;
+}
+
+ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
+    if (!idx) return RALM_OK;
+    cudaFree(idx->partial);
+    cudaFree(idx->cache_keys);
+    cudaFree(idx->status);
+    cudaFree(idx->h_queries);
+    cudaFree(idx->h_ids);
+    cudaFree(idx->h_scores);
+    delete idx;
+    return RALM_OK;
+}
+
+ralm_status_t ralm_search(ralm_index_t *idx, const void *queries, int32_t s, int32_t k,
+                          int64_t *ids, float *scores, void *stream) {
+    if (!idx || s < 0 || s > idx->max_s || k < 1 || k > idx->max_k) return RALM_ERR_INVALID_ARG;
+    if (s == 0) return RALM_OK;
+    if (!queries || !ids || !scores || !aligned16(queries)) return RALM_ERR_INVALID_ARG;
+    return search_device(idx, static_cast<const __half *>(queries), s, k, ids, scores,
+                         static_cast<cudaStream_t>(stream));
+}
+
+ralm_status_t ralm_search_host(ralm_index_t *idx, const void *queries_host, int32_t s, int32_t k,
+                               int64_t *ids_host, float *scores_host, void *stream) {
+    if (!idx || s < 0 || s > idx->max_s || k < 1 || k > idx->max_k) return RALM_ERR_INVALID_ARG;
+    if (s == 0) return RALM_OK;
+    if (!queries_host || !ids_host || !scores_host) return RALM_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t sk = static_cast<size_t>(s) * k;
+    if (cudaMemcpyAsync(idx->h_queries, queries_host, static_cast<size_t>(s) * idx->d * 2,
+                        cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return RALM_ERR_CUDA;
+    ralm_status_t rs = search_device(idx, idx->h_queries, s, k, idx->h_ids, idx->h_scores, st);
+    if (rs != RALM_OK) return rs;
+    if (cudaMemcpyAsync(ids_host, idx->h_ids, sk * sizeof(int64_t), cudaMemcpyDeviceToHost, st) !=
+            cudaSuccess ||
+        cudaMemcpyAsync(scores_host, idx->h_scores, sk * sizeof(float), cudaMemcpyDeviceToHost, st) !=
+            cudaSuccess)
+        return RALM_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
+}
+
+ralm_status_t ralm_cache_search(ralm_index_t *idx, const int64_t *cache_ids, int32_t R, int32_t C,
+                                const void *queries, int32_t q, int32_t k, int64_t *ids,
+                                float *scores, void *stream) {
+    if (!idx || R < 0 || C < 1 || C > RALM_MAX_CACHE || q < 1 || k < 1 || k > idx->max_k)
+        return RALM_ERR_INVALID_ARG;
+    if (R == 0) return RALM_OK;
+    if (!cache_ids || !queries || !ids || !scores || !aligned16(queries)) return RALM_ERR_INVALID_ARG;
+    const int Cp = next_pow2(C);
+    if (static_cast<long long>(R) * q * Cp > RALM_MAX_CACHE_KEYS) return RALM_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const dim3 grid((Cp + kCacheSlotsPerCta - 1) / kCacheSlotsPerCta, R);
+    cache_score_kernel<<<grid, kCacheThreads, 0, st>>>(idx->corpus, idx->N, idx->d,
+                                                       idx->metric == RALM_L2, cache_ids, C, Cp,
+                                                       static_cast<const __half *>(queries), q,
+                                                       idx->cache_keys, idx->status);
+    if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
+    cache_rank_kernel<<<R * q, kMergeThreads, 0, st>>>(idx->cache_keys, Cp, k, idx->metric == RALM_L2,
+                                                       ids, scores);
+    if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
+    idx->launches += 2;
+    return RALM_OK;
+}
+
+ralm_status_t ralm_verify(const int64_t *speculated_ids, const int64_t *retrieved_ids, int32_t R,
+                          int32_t stride, int32_t ld, int32_t cmp_k, int32_t *first_mismatch,
+                          void *stream) {
+    if (R < 0 || stride < 0 || cmp_k < 1 || ld < cmp_k) return RALM_ERR_INVALID_ARG;
+    if (R == 0) return RALM_OK;
+    if (!first_mismatch) return RALM_ERR_INVALID_ARG;
+    if (stride > 0 && (!speculated_ids || !retrieved_ids)) return RALM_ERR_INVALID_ARG;
+    verify_kernel<<<(R + 3) / 4, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        speculated_ids, retrieved_ids, R, stride, ld, cmp_k, first_mismatch);
+    return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
+}
+
+ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream) {
+    if (!idx) return RALM_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int word = 0;
+    if (cudaMemcpyAsync(&word, idx->status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemsetAsync(idx->status, 0, sizeof(int), st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return RALM_ERR_CUDA;
+    if (word == kStatusTimeout) return RALM_ERR_TIMEOUT;
+    if (word == kStatusBadCacheId) return RALM_ERR_BAD_CACHE_ID;
+    return word == 0 ? RALM_OK : RALM_ERR_CUDA;
+}
+
+ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant) {
+    if (!idx || variant < 0 || variant > 3) return RALM_ERR_INVALID_ARG;
+    if (variant == 1 && idx->d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
+    if (variant == 2 && idx->metric != RALM_IP) return RALM_ERR_UNSUPPORTED;
+    if (variant == 3) return RALM_ERR_UNSUPPORTED;
+    idx->variant = variant;
+    return RALM_OK;
+}
+
+int64_t ralm_index_launch_count(const ralm_index_t *idx) { return idx ? idx->launches : 0; }
+
+const char *ralm_status_string(ralm_status_t status) {
+    switch (status) {
+        case RALM_OK: return "ok";
+        case RALM_ERR_INVALID_ARG: return "invalid argument";
+        case RALM_ERR_OOM: return "out of device memory";
+        case RALM_ERR_CUDA: return "CUDA runtime error";
+        case RALM_ERR_TIMEOUT: return "a device-side wait ran out";
+        case RALM_ERR_UNSUPPORTED: return "unsupported device, shape or variant";
+        case RALM_ERR_BAD_CACHE_ID: return "a cache id was outside [-1, N)";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,418 @@
+// Corpus scan for small query batches (at most 8 queries per pass): scores every corpus
+// row against every query and keeps, per CTA and query, the best k rows.
+//
+// One persistent CTA per SM. Warp 0 is the producer: one thread streams 16-row tiles of
+// the row-major corpus (a tile is one contiguous block of memory) into a ring of shared
+// memory stages with 1-D bulk copies that complete on mbarriers. Every other warp owns one
+// stage: it waits for its tile, scores it, hands the stage back, and keeps candidates.
+//
+// Two ways of scoring a tile:
+//   FMA flavour: each lane holds its slice of every query in registers (fp32, packed
+//     pairs), converts its slice of a row and issues packed fp32 FMAs; per-lane partial
+//     sums are combined with a transposing shuffle reduction. Serves both metrics (L2 in
+//     the direct sum-of-squared-differences form, which has no cancellation).
+//   warp-MMA flavour (inner product): m16n8k16 tensor-core tiles with the 16 corpus rows as
+//     M and the (up to) 8 queries as N, fp32 accumulators. The k index is permuted so that
+//     each lane reads 16 contiguous bytes per row and chunks are rotated by row group to
+//     keep shared-memory reads conflict-free without padding.
+//
+// Selection: k == 1 keeps a running best key per thread. k > 1 uses a per-query threshold
+// (the current k-th best of this CTA) and a shared-memory candidate buffer; consumer warps
+// advance in lock-step rounds so that the buffer can be compacted (sorted, truncated to k,
+// threshold raised) before it could overflow.
+#pragma once
+
+#include "common.cuh"
+
+namespace ralm {
+
+constexpr int kTileRows = 16;
+constexpr int kMaxStages = 7;
+constexpr int kScanMaxQueries = 8;
+constexpr int kScanThreads = 32 * (kMaxStages + 1);
+
+struct ScanParams {
+    const __half *corpus;
+    const __half *queries;  // [s][d] of this pass
+    uint64_t *partial;      // [gridDim.x][s_total][k] sorted keys, 0 = empty
+    int *status;
+    long long N;
+    long long ntiles;
+    int d;
+    int s;        // queries in this pass (<= 8)
+    int s_total;  // queries of the whole call (layout of `partial`)
+    int q_base;   // index of this pass's first query in the call
+    int k;
+    int cap;      // candidate buffer capacity per query (power of two); unused when k == 1
+    int nstages;  // ring depth = number of consumer warps
+    int stage_bytes;
+    int off_q;  // shared-memory offsets (bytes)
+    int off_cand;
+    int off_stage;
+};
+
+struct ScanHeader {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    unsigned long long best[kScanMaxQueries];
+    float thr[kScanMaxQueries];
+    int cnt[kScanMaxQueries];
+    int abort;
+};
+constexpr int kScanHeaderBytes = 512;
+static_assert(sizeof(ScanHeader) <= kScanHeaderBytes, "header too large");
+
+// Sort query q's candidates, keep the best k, raise the threshold. Called by all consumer
+// threads (group of `nthr`, ranks `tid`, named barrier 1).
+__device__ inline void compact_query(ScanHeader *hdr, uint64_t *cand, int cap, int q, int k,
+                                     int tid, int nthr) {
+    uint64_t *a = cand + static_cast<size_t>(q) * cap;
+    const int n = hdr->cnt[q];
+    const int P = next_pow2(n > 1 ? n : 2);
+    for (int i = n + tid; i < P; i += nthr) a[i] = 0;
+    named_barrier(1, nthr);
+    bitonic_sort_desc(a, P, tid, nthr, 1);
+    if (tid == 0) {
+        hdr->cnt[q] = n < k ? n : k;
+        hdr->thr[q] = (n >= k) ? key_value(a[k - 1]) : -INFINITY;
+    }
+    named_barrier(1, nthr);
+}
+
+// FMA flavour: transposing shuffle reduction. On entry every lane holds V partial sums
+// (V = 16); on exit a[0] of lanes 2v and 2v+1 is the full sum of value index v.
+template <int V>
+__device__ __forceinline__ void transpose_reduce(float (&a)[V], int lane) {
+    int off = 16;
+#pragma unroll
+    for (int n = V; n > 1; n >>= 1) {
+        const bool upper = (lane & off) != 0;
+#pragma unroll
+        for (int i = 0; i < n / 2; ++i) {
+            const float keep = upper ? a[i + n / 2] : a[i];
+            const float send = upper ? a[i] : a[i + n / 2];
+            a[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+        off >>= 1;
+    }
+#pragma unroll
+    for (int o = 16 / V; o > 0; o >>= 1) a[0] += __shfl_xor_sync(0xffffffffu, a[0], o);
+}
+
+__device__ __forceinline__ void mma_m16n8k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                             uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+        "{%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(addr));
+    return v;
+}
+
+__device__ __forceinline__ float2 h2_to_f2(uint32_t h2) {
+    return __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+}
+
+__device__ __forceinline__ void push_candidate(ScanHeader *hdr, uint64_t *cand, int cap, int q,
+                                               uint64_t key) {
+    const int slot = atomicAdd(&hdr->cnt[q], 1);
+    cand[static_cast<size_t>(q) * cap + slot] = key;
+}
+
+// ------------------------------------------------------------------------------------
+// The kernel. MMA: warp-MMA flavour (inner product only) or FMA flavour.
+// L2: metric of the FMA flavour. SQ: queries held per lane (1, 2 or 4; FMA flavour).
+// DP: 16-byte pieces of a row per lane (d <= 256 * DP; FMA flavour). TOP1: k == 1.
+// ------------------------------------------------------------------------------------
+template <bool MMA, bool L2, int SQ, int DP, bool TOP1>
+__global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    ScanHeader *hdr = reinterpret_cast<ScanHeader *>(smem);
+    uint64_t *cand = reinterpret_cast<uint64_t *>(smem + p.off_cand);
+    const int W = p.nstages;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int d = p.d;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < W; ++i) {
+            mbar_init(smem_u32(&hdr->full[i]), 1);
+            mbar_init(smem_u32(&hdr->empty[i]), 1);
+        }
+        mbar_fence_init();
+        hdr->abort = 0;
+    }
+    if (threadIdx.x < kScanMaxQueries) {
+        hdr->thr[threadIdx.x] = -INFINITY;
+        hdr->cnt[threadIdx.x] = 0;
+        hdr->best[threadIdx.x] = 0ull;
+    }
+    if (MMA) {
+        // queries as fp16 [8][d] in shared memory, rows >= s zeroed
+        uint4 *qs = reinterpret_cast<uint4 *>(smem + p.off_q);
+        const uint4 *qg = reinterpret_cast<const uint4 *>(p.queries);
+        const int per_row = d / 8;
+        for (int i = threadIdx.x; i < kScanMaxQueries * per_row; i += blockDim.x) {
+            const int row = i / per_row;
+            qs[i] = (row < p.s) ? qg[i] : make_uint4(0, 0, 0, 0);
+        }
+    }
+    __syncthreads();
+
+    const long long my_tiles =
+        (p.ntiles > blockIdx.x) ? (p.ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    volatile int *abort_flag = &hdr->abort;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- producer
+        if (lane == 0) {
+            long long issued = 0;
+            bool ok = true;
+            for (long long it = 0; it < my_tiles; ++it) {
+                const int st = static_cast<int>(it % W);
+                const long long use = it / W;
+                if (use > 0) {
+                    ok = mbar_wait_bounded(smem_u32(&hdr->empty[st]), (use - 1) & 1);
+                    if (!ok) break;
+                }
+                if (*abort_flag) break;
+                const long long tile = blockIdx.x + it * static_cast<long long>(gridDim.x);
+                const long long row0 = tile * kTileRows;
+                const long long rows = (p.N - row0 < kTileRows) ? (p.N - row0) : kTileRows;
+                const uint32_t bytes = static_cast<uint32_t>(rows * d * 2);
+                const uint32_t bar = smem_u32(&hdr->full[st]);
+                mbar_arrive_expect_tx(bar, bytes);
+                bulk_load(smem_u32(smem + p.off_stage + static_cast<size_t>(st) * p.stage_bytes),
+                          p.corpus + row0 * d, bytes, bar);
+                issued = it + 1;
+            }
+            if (!ok) {
+                atomicMax(p.status, kStatusTimeout);
+                *abort_flag = 1;
+            }
+            if (*abort_flag) {
+                // winding down early: let every copy already issued land before exit
+                for (long long it = (issued > W ? issued - W : 0); it < issued; ++it)
+                    mbar_wait_bounded(smem_u32(&hdr->full[it % W]), (it / W) & 1);
+            }
+        }
+    } else if (warp - 1 < W) {
+        // ---------------------------------------------------------------- consumers
+        const int w = warp - 1;
+        const int ctid = threadIdx.x - 32;
+        const int cthreads = W * 32;
+        const uint32_t stage_addr =
+            smem_u32(smem + p.off_stage + static_cast<size_t>(w) * p.stage_bytes);
+        const long long rounds = (my_tiles + W - 1) / W;
+        const int g = lane >> 2, t = lane & 3;
+
+        uint64_t best0 = 0, best1 = 0;
+        // FMA flavour: this lane's slice of every query as fp32 pairs (negated for L2 so
+        // that the difference is one packed add)
+        constexpr int DPR = MMA ? 1 : DP;
+        constexpr int SQR = MMA ? 1 : SQ;
+        float2 qreg[SQR][DPR][4];
+        if (!MMA) {
+#pragma unroll
+            for (int j = 0; j < SQR; ++j)
+#pragma unroll
+                for (int i = 0; i < DPR; ++i) {
+                    const int piece = lane + 32 * i;
+                    uint4 raw = make_uint4(0, 0, 0, 0);
+                    if (j < p.s && piece * 8 < d)
+                        raw = *reinterpret_cast<const uint4 *>(p.queries +
+                                                               static_cast<size_t>(j) * d + piece * 8);
+                    const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        float2 v = h2_to_f2(words[e]);
+                        if (L2) {
+                            v.x = -v.x;
+                            v.y = -v.y;
+                        }
+                        qreg[j][i][e] = v;
+                    }
+                }
+        }
+
+        for (long long j = 0; j < rounds; ++j) {
+            const long long it = j * W + w;
+            if (it < my_tiles && !*abort_flag) {
+                if (!mbar_wait_bounded(smem_u32(&hdr->full[w]), j & 1)) {
+                    if (lane == 0) {
+                        atomicMax(p.status, kStatusTimeout);
+                        *abort_flag = 1;
+                    }
+                } else {
+                    const long long tile = blockIdx.x + it * static_cast<long long>(gridDim.x);
+                    const long long row0 = tile * kTileRows;
+                    if (MMA) {
+                        // ---- 16 rows x 8 queries on tensor cores
+                        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                        const int nchunks = (d + 31) >> 5;
+                        const uint32_t q_addr = smem_u32(smem + p.off_q) + g * d * 2;
+                        const uint32_t a_lo_addr = stage_addr + g * d * 2;
+                        const uint32_t a_hi_addr = stage_addr + (g + 8) * d * 2;
+                        int cc = g % nchunks;
+#pragma unroll 4
+                        for (int c = 0; c < nchunks; ++c) {
+                            const int off = cc * 32 + t * 8;  // halves
+                            uint4 b = make_uint4(0, 0, 0, 0), lo = b, hi = b;
+                            if (off < d) {  // ragged last chunk: absent pieces stay zero
+                                b = lds128(q_addr + off * 2);
+                                lo = lds128(a_lo_addr + off * 2);
+                                hi = lds128(a_hi_addr + off * 2);
+                            }
+                            mma_m16n8k16(acc, lo.x, hi.x, lo.y, hi.y, b.x, b.y);
+                            mma_m16n8k16(acc, lo.z, hi.z, lo.w, hi.w, b.z, b.w);
+                            cc = (cc + 1 == nchunks) ? 0 : cc + 1;
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[w]));
+                        // acc[0]: (row g, query 2t)     acc[1]: (row g, query 2t+1)
+                        // acc[2]: (row g+8, query 2t)   acc[3]: (row g+8, query 2t+1)
+                        const long long r_lo = row0 + g, r_hi = row0 + g + 8;
+                        const int q0 = 2 * t, q1 = 2 * t + 1;
+                        if (TOP1) {
+                            if (r_lo < p.N) {
+                                const uint64_t k0 = make_key(acc[0], static_cast<uint32_t>(r_lo));
+                                const uint64_t k1 = make_key(acc[1], static_cast<uint32_t>(r_lo));
+                                best0 = k0 > best0 ? k0 : best0;
+                                best1 = k1 > best1 ? k1 : best1;
+                            }
+                            if (r_hi < p.N) {
+                                const uint64_t k0 = make_key(acc[2], static_cast<uint32_t>(r_hi));
+                                const uint64_t k1 = make_key(acc[3], static_cast<uint32_t>(r_hi));
+                                best0 = k0 > best0 ? k0 : best0;
+                                best1 = k1 > best1 ? k1 : best1;
+                            }
+                        } else {
+                            const float th0 = hdr->thr[q0], th1 = hdr->thr[q1];
+                            if (r_lo < p.N) {
+                                if (q0 < p.s && acc[0] >= th0)
+                                    push_candidate(hdr, cand, p.cap, q0,
+                                                   make_key(acc[0], static_cast<uint32_t>(r_lo)));
+                                if (q1 < p.s && acc[1] >= th1)
+                                    push_candidate(hdr, cand, p.cap, q1,
+                                                   make_key(acc[1], static_cast<uint32_t>(r_lo)));
+                            }
+                            if (r_hi < p.N) {
+                                if (q0 < p.s && acc[2] >= th0)
+                                    push_candidate(hdr, cand, p.cap, q0,
+                                                   make_key(acc[2], static_cast<uint32_t>(r_hi)));
+                                if (q1 < p.s && acc[3] >= th1)
+                                    push_candidate(hdr, cand, p.cap, q1,
+                                                   make_key(acc[3], static_cast<uint32_t>(r_hi)));
+                            }
+                        }
+                    } else {
+                        // ---- FMA flavour: RG rows at a time, RG * SQ = 16 partial sums
+                        constexpr int RG = 16 / SQR;
+                        constexpr int V = 16;
+#pragma unroll 1
+                        for (int rg = 0; rg < kTileRows; rg += RG) {
+                            float2 acc2[RG][SQR];
+#pragma unroll
+                            for (int r = 0; r < RG; ++r)
+#pragma unroll
+                                for (int jq = 0; jq < SQR; ++jq) acc2[r][jq] = make_float2(0.f, 0.f);
+#pragma unroll
+                            for (int i = 0; i < DPR; ++i) {
+                                const int piece = lane + 32 * i;
+                                if (piece * 8 < d) {
+#pragma unroll
+                                    for (int r = 0; r < RG; ++r) {
+                                        const uint4 raw =
+                                            lds128(stage_addr + ((rg + r) * d + piece * 8) * 2);
+                                        const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                                        for (int e = 0; e < 4; ++e) {
+                                            const float2 x = h2_to_f2(words[e]);
+#pragma unroll
+                                            for (int jq = 0; jq < SQR; ++jq) {
+                                                if (L2) {
+                                                    const float2 df = __fadd2_rn(x, qreg[jq][i][e]);
+                                                    acc2[r][jq] = __ffma2_rn(df, df, acc2[r][jq]);
+                                                } else {
+                                                    acc2[r][jq] =
+                                                        __ffma2_rn(x, qreg[jq][i][e], acc2[r][jq]);
+                                                }
+                                            }
+                                        }
+                                    }
+                                }
+                            }
+                            float a[V];
+#pragma unroll
+                            for (int r = 0; r < RG; ++r)
+#pragma unroll
+                                for (int jq = 0; jq < SQR; ++jq)
+                                    a[r * SQR + jq] = acc2[r][jq].x + acc2[r][jq].y;
+                            transpose_reduce<V>(a, lane);
+                            if (rg + RG >= kTileRows) {
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[w]));
+                            }
+                            // lanes 2v and 2v+1 hold value v = r * SQ + jq
+                            const int v = lane >> 1;
+                            const int r = v / SQR, jq = v % SQR;
+                            const long long row = row0 + rg + r;
+                            const float val = L2 ? (0.0f - a[0]) : a[0];
+                            if ((lane & 1) == 0 && row < p.N && jq < p.s) {
+                                if (TOP1) {
+                                    const uint64_t key = make_key(val, static_cast<uint32_t>(row));
+                                    best0 = key > best0 ? key : best0;
+                                } else if (val >= hdr->thr[jq]) {
+                                    push_candidate(hdr, cand, p.cap, jq,
+                                                   make_key(val, static_cast<uint32_t>(row)));
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            if (!TOP1) {
+                // lock-step round: nobody pushes between this barrier and the decision
+                named_barrier(1, cthreads);
+                for (int q = 0; q < p.s; ++q) {
+                    if (hdr->cnt[q] > p.cap - W * kTileRows)
+                        compact_query(hdr, cand, p.cap, q, p.k, ctid, cthreads);
+                }
+            }
+        }
+
+        // ------------------------------------------------------------ CTA result
+        if (TOP1) {
+            if (MMA) {
+                if (best0) atomicMax(&hdr->best[2 * t], static_cast<unsigned long long>(best0));
+                if (best1) atomicMax(&hdr->best[2 * t + 1], static_cast<unsigned long long>(best1));
+            } else {
+                const int jq = (lane >> 1) % SQR;
+                if (best0) atomicMax(&hdr->best[jq], static_cast<unsigned long long>(best0));
+            }
+            named_barrier(1, cthreads);
+            if (ctid < p.s)
+                p.partial[static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + ctid] =
+                    hdr->best[ctid];
+        } else {
+            named_barrier(1, cthreads);
+            for (int q = 0; q < p.s; ++q) {
+                compact_query(hdr, cand, p.cap, q, p.k, ctid, cthreads);
+                const int n = hdr->cnt[q];
+                uint64_t *dst =
+                    p.partial + (static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
+                for (int i = ctid; i < p.k; i += cthreads)
+                    dst[i] = (i < n) ? cand[static_cast<size_t>(q) * p.cap + i] : 0ull;
+            }
+        }
+    }
+}
+
+}  // namespace ralm
