@@ -44,7 +44,7 @@ int align_up(int v, int a) { return (v + a - 1) / a * a; }
 bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl) {
     pl->stage_bytes = align_up(kTileRows * idx->d * 2, 128);
     pl->off_q = kScanHeaderBytes;
-    int off = pl->off_q + (mma ? align_up(kScanMaxQueries * idx->d * 2, 128) : 0);
+    int off = pl->off_q + (mma ? align_up(kScanMaxQueries * (idx->d * 2 + kQueryPadBytes), 128) : 0);
     pl->off_cand = off;
     pl->cap = 0;
     if (k > 1) {

@@ -12,9 +12,8 @@
 //     sums are combined with a transposing shuffle reduction. Serves both metrics (L2 in
 //     the direct sum-of-squared-differences form, which has no cancellation).
 //   warp-MMA flavour (inner product): m16n8k16 tensor-core tiles with the 16 corpus rows as
-//     M and the (up to) 8 queries as N, fp32 accumulators. The k index is permuted so that
-//     each lane reads 16 contiguous bytes per row and chunks are rotated by row group to
-//     keep shared-memory reads conflict-free without padding.
+//     M and the (up to) 8 queries as N, fp32 accumulators. The k index is permuted (the
+//     same way for rows and queries) so that each lane reads 16 contiguous bytes per row.
 //
 // Selection: k == 1 keeps a running best key per thread. k > 1 uses a per-query threshold
 // (the current k-th best of this CTA) and a shared-memory candidate buffer; consumer warps
@@ -30,6 +29,7 @@ constexpr int kTileRows = 16;
 constexpr int kMaxStages = 7;
 constexpr int kScanMaxQueries = 8;
 constexpr int kScanThreads = 32 * (kMaxStages + 1);
+constexpr int kQueryPadBytes = 64;
 
 struct ScanParams {
     const __half *corpus;
@@ -155,13 +155,14 @@ __global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams 
         hdr->best[threadIdx.x] = 0ull;
     }
     if (MMA) {
-        // queries as fp16 [8][d] in shared memory, rows >= s zeroed
-        uint4 *qs = reinterpret_cast<uint4 *>(smem + p.off_q);
+        // queries as fp16 [8][d] in shared memory, rows >= s zeroed; rows are padded by
+        // kQueryPadBytes so that the eight query rows do not all start on the same bank
         const uint4 *qg = reinterpret_cast<const uint4 *>(p.queries);
         const int per_row = d / 8;
         for (int i = threadIdx.x; i < kScanMaxQueries * per_row; i += blockDim.x) {
-            const int row = i / per_row;
-            qs[i] = (row < p.s) ? qg[i] : make_uint4(0, 0, 0, 0);
+            const int row = i / per_row, col = i - row * per_row;
+            *reinterpret_cast<uint4 *>(smem + p.off_q + row * (d * 2 + kQueryPadBytes) + col * 16) =
+                (row < p.s) ? qg[i] : make_uint4(0, 0, 0, 0);
         }
     }
     __syncthreads();
@@ -257,13 +258,14 @@ __global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams 
                         // ---- 16 rows x 8 queries on tensor cores
                         float acc[4] = {0.f, 0.f, 0.f, 0.f};
                         const int nchunks = (d + 31) >> 5;
-                        const uint32_t q_addr = smem_u32(smem + p.off_q) + g * d * 2;
+                        const uint32_t q_addr = smem_u32(smem + p.off_q) + g * (d * 2 + kQueryPadBytes);
                         const uint32_t a_lo_addr = stage_addr + g * d * 2;
                         const uint32_t a_hi_addr = stage_addr + (g + 8) * d * 2;
-                        int cc = g % nchunks;
 #pragma unroll 4
                         for (int c = 0; c < nchunks; ++c) {
-                            const int off = cc * 32 + t * 8;  // halves
+                            // logical k (2t, 2t+1, 2t+8, 2t+9 of two MMAs) <- physical halves
+                            // off..off+7, the same permutation for every row and query
+                            const int off = c * 32 + t * 8;
                             uint4 b = make_uint4(0, 0, 0, 0), lo = b, hi = b;
                             if (off < d) {  // ragged last chunk: absent pieces stay zero
                                 b = lds128(q_addr + off * 2);
@@ -272,7 +274,6 @@ __global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams 
                             }
                             mma_m16n8k16(acc, lo.x, hi.x, lo.y, hi.y, b.x, b.y);
                             mma_m16n8k16(acc, lo.z, hi.z, lo.w, hi.w, b.z, b.w);
-                            cc = (cc + 1 == nchunks) ? 0 : cc + 1;
                         }
                         __syncwarp();
                         if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[w]));

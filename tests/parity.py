@@ -1,0 +1,65 @@
+"""Acceptance rule shared by the GPU parity tests.
+
+For rank p of a query (oracle = fp64 CPU reference on the same fp16 bytes):
+  strict-OK  gpu_id[p] == oracle_id[p]
+  band-OK    gpu_id[p] is a valid row, appears once in the GPU list, and its ORACLE score
+             is within 2e-3 relative of the oracle's score at rank p (the two rows sit in
+             one near-tie band)
+  FAIL       anything else
+Scores: |gpu_score - oracle_score(gpu_id)| <= 2e-3 * |oracle_score| + 1e-5 * scale, where
+`scale` bounds |q||x| (only matters for inner products near zero).
+"""
+import numpy as np
+
+import oracle
+
+REL = 2e-3
+
+
+def check_lists(gpu_ids, gpu_scores, ora_ids, ora_scores, score_of, metric, scale=1.0, n_valid=None):
+    """One query. score_of(id) -> oracle fp64 score of that row for this query.
+    Returns (strict, band); raises AssertionError on FAIL."""
+    k = len(ora_ids)
+    strict = band = 0
+    seen = set()
+    for p in range(k):
+        gid, oid = int(gpu_ids[p]), int(ora_ids[p])
+        if oid < 0:
+            assert gid == -1, "rank %d: expected padding, got id %d" % (p, gid)
+            assert np.isinf(gpu_scores[p]) and (gpu_scores[p] < 0) == (metric == oracle.IP)
+            strict += 1
+            continue
+        assert gid >= 0 and (n_valid is None or gid < n_valid), "rank %d: invalid id %d" % (p, gid)
+        assert gid not in seen, "rank %d: id %d repeated" % (p, gid)
+        seen.add(gid)
+        s_true = ora_scores[p] if gid == oid else score_of(gid)
+        if gid == oid:
+            strict += 1
+        else:
+            assert abs(s_true - ora_scores[p]) < REL * abs(ora_scores[p]) + 1e-30, \
+                "rank %d: id %d (score %r) is outside the near-tie band of oracle id %d (score %r)" % (
+                    p, gid, s_true, oid, ora_scores[p])
+            band += 1
+        assert abs(float(gpu_scores[p]) - s_true) <= REL * abs(s_true) + 1e-5 * scale, \
+            "rank %d: score %r vs oracle %r" % (p, float(gpu_scores[p]), s_true)
+    return strict, band
+
+
+def check_search(gpu_ids, gpu_scores, corpus_np, queries_np, metric, k, exact=False):
+    """Whole-batch comparison against oracle.search. Returns (strict, band) totals."""
+    ora_ids, ora_scores = oracle.search(corpus_np, queries_np, metric, k)
+    gi, gs = gpu_ids.cpu().numpy(), gpu_scores.cpu().numpy()
+    if exact:
+        assert np.array_equal(gi, ora_ids)
+        assert np.array_equal(gs.astype(np.float64), ora_scores)
+        return gi.size, 0
+    strict = band = 0
+    norms = np.linalg.norm(corpus_np.astype(np.float64), axis=1).max() if corpus_np.shape[0] else 1.0
+    for i in range(queries_np.shape[0]):
+        scale = norms * np.linalg.norm(queries_np[i].astype(np.float64))
+        a, b = check_lists(gi[i], gs[i], ora_ids[i], ora_scores[i],
+                           lambda j, i=i: oracle.pair_score(corpus_np[j], queries_np[i], metric),
+                           metric, scale=scale, n_valid=corpus_np.shape[0])
+        strict += a
+        band += b
+    return strict, band

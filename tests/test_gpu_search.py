@@ -1,0 +1,213 @@
+"""GPU parity: ralm_search against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+from parity import check_search
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _ralm():
+    import paper_2401_14021_b200 as ralm
+    return ralm
+
+
+def _run(corpus, queries, metric, k, variant=0):
+    ralm = _ralm()
+    idx = ralm.Index(corpus, metric, max_s=max(1, queries.shape[0]), max_k=k)
+    if variant:
+        idx.set_variant(variant)
+    ids, scores = ralm.search(idx, queries, k)
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    idx.close()
+    return ids, scores
+
+
+VARIANTS = {oracle.IP: (2, 1), oracle.L2: (1,)}
+
+
+# ------------------------------------------------------------------ exact integer cases
+@pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
+@pytest.mark.parametrize("N,d,s,k", [(1, 8, 1, 1), (15, 8, 3, 4), (16, 16, 8, 1), (17, 64, 5, 20),
+                                     (33, 40, 2, 40), (1000, 72, 8, 7), (5000, 768, 4, 5),
+                                     (3001, 1024, 4, 1024), (257, 264, 9, 3), (64, 8, 17, 64)])
+def test_integer_inputs_are_bit_exact(metric, N, d, s, k):
+    """Small-integer rows: every score is an integer that fp32 holds exactly, and ties abound,
+    so ids (tie-break included) and scores must equal the oracle's bit for bit."""
+    x = workloads.integer_valued((N, d), seed=100 + N, lo=-3, hi=3, device=DEV)
+    q = workloads.integer_valued((s, d), seed=200 + N, lo=-3, hi=3, device=DEV)
+    for variant in VARIANTS[metric]:
+        ids, scores = _run(x, q, metric, k, variant)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), metric, k, exact=True)
+
+
+# ------------------------------------------------------------------ shape sweep, real values
+@pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
+@pytest.mark.parametrize("N", [1, 31, 32, 33, 1000, 100_003])
+@pytest.mark.parametrize("d,s,k", [(8, 1, 1), (64, 3, 5), (768, 8, 20), (1024, 4, 1), (1024, 4, 200)])
+def test_shape_sweep(metric, N, d, s, k):
+    x, _ = workloads.mixture_corpus(N, d, 16, seed=300 + d, device=DEV, normalise=(metric == oracle.IP),
+                                    lognormal_sigma=0.0 if metric == oracle.IP else 0.3)
+    q, _ = workloads.noisy_copy_queries(x, s, seed=301 + d) if N >= s else \
+        (workloads.unit_gaussian_corpus(s, d, seed=5, device=DEV), None)
+    for variant in VARIANTS[metric]:
+        ids, scores = _run(x, q, metric, k, variant)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), metric, k)
+
+
+def test_empty_corpus_and_empty_batch():
+    ralm = _ralm()
+    x = torch.empty((0, 64), dtype=torch.float16, device=DEV)
+    q = workloads.unit_gaussian_corpus(2, 64, seed=1, device=DEV)
+    ids, scores = _run(x, q, oracle.IP, 3)
+    assert (ids == -1).all() and torch.isinf(scores).all() and (scores < 0).all()
+    ids, scores = _run(x, q, oracle.L2, 3)
+    assert (ids == -1).all() and torch.isinf(scores).all() and (scores > 0).all()
+    x = workloads.unit_gaussian_corpus(10, 64, seed=2, device=DEV)
+    idx = ralm.Index(x, oracle.IP, 4, 4)
+    ids, _ = ralm.search(idx, q[:0], 2)
+    assert ids.shape == (0, 2)
+
+
+# ------------------------------------------------------------------ properties
+@pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
+def test_planted_duplicates_rank_first(metric):
+    x, _ = workloads.mixture_corpus(50_000, 768, 64, seed=41, device=DEV, normalise=(metric == oracle.IP),
+                                    lognormal_sigma=0.0 if metric == oracle.IP else 0.3)
+    rows = torch.tensor([0, 15, 16, 4999, 25_000, 49_999], device=DEV)
+    x[40_000] = x[15]                      # exact duplicate: lower id must come first
+    ids, scores = _run(x, x[rows].contiguous(), metric, 2)
+    assert ids[:, 0].tolist() == rows.tolist()
+    assert ids[1].tolist() == [15, 40_000] and scores[1, 0] == scores[1, 1]
+    if metric == oracle.L2:
+        assert (scores[:, 0] == 0).all()
+
+
+@pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
+def test_batched_equals_sequential_and_is_deterministic(metric):
+    ralm = _ralm()
+    x, _ = workloads.mixture_corpus(200_000, 768, 128, seed=43, device=DEV)
+    q, _ = workloads.noisy_copy_queries(x, 8, seed=44)
+    idx = ralm.Index(x, metric, 8, 20)
+    ids, scores = ralm.search(idx, q, 20)
+    ids2, scores2 = ralm.search(idx, q, 20)
+    assert torch.equal(ids, ids2) and torch.equal(scores, scores2)
+    for i in range(8):
+        one_ids, one_scores = ralm.search(idx, q[i:i + 1].contiguous(), 20)
+        assert torch.equal(one_ids[0], ids[i])
+        torch.testing.assert_close(one_scores[0], scores[i], rtol=1e-5, atol=1e-6)
+    assert idx.device_status() == 0
+
+
+def test_adversarial_row_order_sorted_by_score():
+    """Rows sorted so that scores increase along the corpus: every row beats the threshold."""
+    N, d = 40_000, 64
+    x = torch.zeros((N, d), dtype=torch.float16, device=DEV)
+    x[:, 0] = (torch.arange(N, device=DEV) // 32).to(torch.float16)   # runs of 32 equal scores
+    q = torch.zeros((2, d), dtype=torch.float16, device=DEV)
+    q[0, 0] = 1.0
+    q[1, 0] = -1.0
+    for variant in (2, 1):
+        ids, scores = _run(x, q, oracle.IP, 100, variant)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 100, exact=True)
+    ids, scores = _run(x, q[:1].contiguous(), oracle.L2, 1024)
+    check_search(ids, scores, x.cpu().numpy(), q[:1].cpu().numpy(), oracle.L2, 1024, exact=True)
+
+
+def test_clustered_row_order():
+    x, _ = workloads.mixture_corpus(100_000, 128, 32, seed=47, device=DEV, clustered_order=True)
+    q, _ = workloads.noisy_copy_queries(x, 4, seed=48)
+    ids, scores = _run(x, q, oracle.IP, 50)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 50)
+
+
+def test_fp16_extremes_subnormals_and_signed_zero():
+    N, d = 4096, 64
+    g = torch.Generator(device="cpu").manual_seed(7)
+    bits = torch.randint(0, 1 << 16, (N, d), generator=g, dtype=torch.int32)
+    bits = torch.where((bits & 0x7C00) == 0x7C00, bits & 0x83FF, bits)      # no inf / NaN
+    x = bits.to(torch.int16).view(torch.float16)
+    x = x.float().clamp(-60, 60).to(torch.float16)
+    # rows 0..63: only subnormals and signed zeros
+    x[:64] = (bits[:64] & 0x83FF).to(torch.int16).view(torch.float16)
+    x = x.to(DEV)
+    q = x[[3, 100, 2000, 4000]].contiguous()
+    for metric in (oracle.IP, oracle.L2):
+        ids, scores = _run(x, q, metric, 10)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), metric, 10)
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    ralm = _ralm()
+    x, _ = workloads.mixture_corpus(50_000, 768, 64, seed=51, device=DEV)
+    q, _ = workloads.noisy_copy_queries(x, 8, seed=52)
+    idx = ralm.Index(x, oracle.IP, 8, 20)
+    ids, scores = ralm.search(idx, q, 20)
+    qh = q.cpu().pin_memory()
+    ih = torch.empty((8, 20), dtype=torch.int64).pin_memory()
+    sh = torch.empty((8, 20), dtype=torch.float32).pin_memory()
+    ralm.search_host(idx, qh, 20, ih, sh)
+    assert torch.equal(ih, ids.cpu()) and torch.equal(sh, scores.cpu())
+
+
+def test_argument_errors():
+    ralm = _ralm()
+    x = workloads.unit_gaussian_corpus(100, 64, seed=3, device=DEV)
+    q = workloads.unit_gaussian_corpus(4, 64, seed=4, device=DEV)
+    idx = ralm.Index(x, oracle.IP, 2, 5)
+    with pytest.raises(ralm.RalmError):
+        ralm.search(idx, q, 5)            # s > max_s
+    with pytest.raises(ralm.RalmError):
+        ralm.search(idx, q[:2].contiguous(), 6)   # k > max_k
+    with pytest.raises(ralm.RalmError):
+        idx.set_variant(7)
+    l2 = ralm.Index(x, oracle.L2, 2, 5)
+    with pytest.raises(ralm.RalmError):
+        l2.set_variant(2)                 # warp-MMA scan cannot serve L2
+
+
+# ------------------------------------------------------------------ the configs
+def test_config_c1():
+    c = workloads.CONFIGS["C1"]
+    x = workloads.unit_gaussian_corpus(c.N, c.d, workloads.seed_for(1), device=DEV)
+    q, src = workloads.noisy_copy_queries(x, 4, workloads.seed_for(1, "queries"))
+    for k in c.k_values:
+        for variant in (2, 1):
+            ids, scores = _run(x, q, oracle.IP, k, variant)
+            strict, band = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k)
+            assert ids[:, 0].tolist() == src.tolist()
+
+
+@pytest.mark.parametrize("s", [1, 2, 4, 8])
+def test_config_c2(s, c2_corpus):
+    x, xn = c2_corpus
+    q, src = workloads.noisy_copy_queries(x, s, workloads.seed_for(2, "queries"))
+    for k in (1, 20):
+        ids, scores = _run(x, q, oracle.IP, k)
+        strict, band = check_search(ids, scores, xn, q.cpu().numpy(), oracle.IP, k)
+        assert ids[:, 0].tolist() == src.tolist()
+        print("C2 s=%d k=%d strict=%d band=%d" % (s, k, strict, band))
+
+
+@pytest.fixture(scope="module")
+def c2_corpus():
+    c = workloads.CONFIGS["C2"]
+    x, _ = workloads.mixture_corpus(c.N, c.d, c.n_centres, workloads.seed_for(2), device=DEV)
+    return x, x.cpu().numpy()
+
+
+def test_knn_lm_shape_l2_k1024():
+    """The KNN-LM datastore shape at 1/50 scale: d = 1024, unnormalised keys, L2, k = 1024."""
+    x, _ = workloads.mixture_corpus(1_000_000, 1024, 4096, workloads.seed_for(4), device=DEV,
+                                    normalise=False, lognormal_sigma=0.3)
+    q, src = workloads.noisy_copy_queries(x, 4, workloads.seed_for(4, "queries"))
+    ids, scores = _run(x, q, oracle.L2, 1024)
+    strict, band = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, 1024)
+    assert ids[:, 0].tolist() == src.tolist()
+    print("C4/50 strict=%d band=%d" % (strict, band))
