@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the exact-retrieval verification step on synthetic corpora.
+
+One step = one verification step of the serving loop, all kernels on one stream:
+  ralm_cache_search  speculation: R concurrent requests x q queries over their local caches
+  ralm_search        verification retrieval: s queries against the whole N x d corpus
+  ralm_verify        first mis-speculated position of the verified request
+Throughput is verified queries per second = s * steps / time. Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+                  [--workload C1|C2|C3|C4] [--s S] [--k K] [--variant V] [--rows N]
+
+With --gpus N > 1 (launched under torch.distributed.run) every rank runs an independent
+replica on its own GPU (the path does not shard); the value is the sum over replicas and the
+time is the maximum over ranks. --impl reference times the fp64 CPU oracle on a bounded
+sample of the same workload.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "verified queries/s at 21Mx768 fp16 top-1, s=8; % of HBM roofline"
+UNIT = "queries/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return json.load(fh), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3", choices=["C1", "C2", "C3", "C4"])
+    ap.add_argument("--s", type=int, default=None)
+    ap.add_argument("--k", type=int, default=None)
+    ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--rows", type=int, default=None, help="override the corpus size (profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def build_inputs(cfg, s, device, rows=None):
+    """Corpus, verification queries, speculation caches and cache queries of one replica."""
+    N = rows or cfg.N
+    seed = workloads.seed_for(cfg.index)
+    if cfg.corpus == "unit_gaussian":
+        corpus, assign = workloads.unit_gaussian_corpus(N, cfg.d, seed, device=device), None
+    else:
+        corpus, assign = workloads.mixture_corpus(N, cfg.d, cfg.n_centres, seed, device=device,
+                                                  sigma_within=cfg.sigma_within,
+                                                  normalise=cfg.normalise,
+                                                  lognormal_sigma=cfg.lognormal_sigma)
+    R = max(cfg.requests, 1)
+    stride = cfg.stride or s
+    C = cfg.cache_entries or 64
+    # request 0 is the one being verified; its first s queries form the verification batch
+    nq = max(R * stride, s)
+    queries, src = workloads.noisy_copy_queries(corpus, nq, workloads.seed_for(cfg.index, "queries"))
+    cache_q = queries[:R * stride].reshape(R, stride, cfg.d).contiguous()
+    cache = workloads.speculation_cache_ids(assign, N, src[:R * stride].reshape(R, stride), C,
+                                            workloads.seed_for(cfg.index, "caches"),
+                                            n_centres=max(cfg.n_centres, 1))
+    return corpus, queries[:s].contiguous(), src[:s], cache, cache_q
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.proc = None
+        self.path = None
+        try:
+            uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100", "-f", self.path], stdout=subprocess.DEVNULL, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons, smax, power = [], set(), None, []
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    smax = float(f[1])
+                    power.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                      "sw_power_cap"), f[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        finally:
+            try:
+                os.unlink(self.path)
+            except OSError:
+                pass
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=smax, reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(power) if power else None)
+        return out
+
+
+def cpu_baseline(corpus, queries, metric_id, k, N_full, s, budget_s=15.0):
+    """The oracle, as it stands, on a bounded sample: the first rows of the same corpus."""
+    import oracle
+    probe = min(corpus.shape[0], 20_000)
+    xq = queries.cpu().numpy()
+    xs = corpus[:probe].cpu().numpy()
+    t0 = time.perf_counter()
+    _, _, cores = oracle.search(xs, xq, metric_id, k, return_threads=True)
+    tp = time.perf_counter() - t0
+    rows = int(min(corpus.shape[0], max(probe, probe * budget_s / max(tp, 1e-6)), 2_000_000))
+    xs = corpus[:rows].cpu().numpy()
+    t0 = time.perf_counter()
+    _, _, cores = oracle.search(xs, xq, metric_id, k, return_threads=True)
+    t = time.perf_counter() - t0
+    value = s / (t * N_full / rows)
+    return {"value": value, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": "first %d of %d rows, all %d queries, k=%d, %.1f s; scaled linearly in N"
+                      % (rows, N_full, s, k, t)}
+
+
+def run_reference(args, cfg, s, k, metric_id):
+    """The CPU oracle as the reference arm: every step scores a bounded row sample."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    rows = min(cfg.N, args.rows or 60_000)
+    seed = workloads.seed_for(cfg.index)
+    if cfg.corpus == "unit_gaussian":
+        corpus = workloads.unit_gaussian_corpus(rows, cfg.d, seed)
+    else:
+        corpus, _ = workloads.mixture_corpus(rows, cfg.d, cfg.n_centres, seed, normalise=cfg.normalise,
+                                             lognormal_sigma=cfg.lognormal_sigma)
+    q, _ = workloads.noisy_copy_queries(corpus, s, workloads.seed_for(cfg.index, "queries"))
+    xn, qn = corpus.numpy(), q.numpy()
+    steps, warmup = min(args.steps, 8), min(args.warmup, 1)
+    cores = 1
+    for _ in range(warmup):
+        oracle.search(xn, qn, metric_id, k)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        ids, _, cores = oracle.search(xn, qn, metric_id, k, return_threads=True)
+        oracle.verify(ids[None, :, :1].reshape(1, s), ids[None, :, :])
+    t = (time.perf_counter() - t0) / steps
+    value = s / (t * cfg.N / rows)
+    sample = "%d of %d rows per step, %d queries, k=%d; scaled linearly in N" % (rows, cfg.N, s, k)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warmup, "ms_per_step": t * 1e3 * cfg.N / rows,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": "%s %dx%d %s s=%d k=%d" % (cfg.name, cfg.N, cfg.d, cfg.metric, s, k)},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    args = parse_args()
+    cfg = workloads.CONFIGS[args.workload]
+    s = args.s or (8 if args.workload == "C3" else cfg.s_values[-1])
+    k = args.k or cfg.k_values[0]
+    metric_id = 0 if cfg.metric == "ip" else 1
+    if args.impl == "reference":
+        run_reference(args, cfg, s, k, metric_id)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    import paper_2401_14021_b200 as ralm
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    corpus, queries, src, cache, cache_q = build_inputs(cfg, s, device, args.rows)
+    N, d = corpus.shape
+    R, stride = cache_q.shape[0], cache_q.shape[1]
+    idx = ralm.Index(corpus, metric_id, max_s=max(s, 1), max_k=max(k, 1))
+    if args.variant:
+        idx.set_variant(args.variant)
+    stream = torch.cuda.current_stream()
+
+    ids = torch.empty((s, k), dtype=torch.int64, device=device)
+    scores = torch.empty((s, k), dtype=torch.float32, device=device)
+    spec_ids = torch.empty((R, stride, 1), dtype=torch.int64, device=device)
+    spec_scores = torch.empty((R, stride, 1), dtype=torch.float32, device=device)
+    first_mismatch = torch.empty((1,), dtype=torch.int32, device=device)
+    vstride = min(stride, s)
+
+    def step():
+        ralm.cache_search(idx, cache, cache_q, 1, spec_ids, spec_scores, stream)
+        ralm.search(idx, queries, k, ids, scores, stream)
+        ralm.verify(spec_ids[0:1, :vstride, 0], ids[:vstride].unsqueeze(0), 1, first_mismatch, stream)
+
+    # ---- device-resident timing
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    idx.read_timing()
+    idx.set_timing(True)
+    launches0 = idx.launch_count()
+    sampler = ClockSampler(local_rank)
+    time.sleep(0.25)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    total_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    scan_ms, scan_launches = idx.read_timing()
+    idx.set_timing(False)
+    gpu_launches = idx.launch_count() - launches0 + args.steps   # + one verify launch per step
+    assert idx.device_status() == 0, "device status word set during the timed region"
+    assert ids[:, 0].tolist() == src.tolist(), "rank-0 ids are not the planted sources"
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region
+    h_q = queries.cpu().pin_memory()
+    h_cache = cache.cpu().pin_memory()
+    h_cache_q = cache_q.cpu().pin_memory()
+    h_ids = torch.empty((s, k), dtype=torch.int64).pin_memory()
+    h_scores = torch.empty((s, k), dtype=torch.float32).pin_memory()
+    h_spec = torch.empty((R, stride, 1), dtype=torch.int64).pin_memory()
+    h_fm = torch.empty((1,), dtype=torch.int32).pin_memory()
+    d_cache, d_cache_q = torch.empty_like(cache), torch.empty_like(cache_q)
+    retr1 = torch.empty((1, vstride, 1), dtype=torch.int64, device=device)
+    h2d = h_q.numel() * 2 + h_cache.numel() * 8 + h_cache_q.numel() * 2 + h_ids[:vstride, :1].numel() * 8
+    d2h = h_ids.numel() * 8 + h_scores.numel() * 4 + h_spec.numel() * 8 + 4
+
+    def step_e2e():
+        d_cache.copy_(h_cache, non_blocking=True)
+        d_cache_q.copy_(h_cache_q, non_blocking=True)
+        ralm.cache_search(idx, d_cache, d_cache_q, 1, spec_ids, spec_scores, stream)
+        ralm.search_host(idx, h_q, k, h_ids, h_scores, stream)          # H2D, scan, D2H, sync
+        retr1.copy_(h_ids[:vstride, :1].unsqueeze(0), non_blocking=True)
+        ralm.verify(spec_ids[0:1, :vstride, 0], retr1, 1, first_mismatch, stream)
+        h_spec.copy_(spec_ids, non_blocking=True)
+        h_fm.copy_(first_mismatch, non_blocking=True)
+        stream.synchronize()
+
+    for _ in range(3):
+        step_e2e()
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step_e2e()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+
+    # ---- aggregate over ranks: time = max, work = sum
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = t.tolist()
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        value = world * s * args.steps / (total_ms * 1e-3)
+        e2e_value = world * s * args.steps / (e2e_ms * 1e-3)
+        corpus_bytes = N * d * 2
+        passes = scan_launches / max(args.steps, 1)
+        scan_avg_ms = scan_ms / max(scan_launches, 1)
+        achieved = corpus_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f16 inputs, f32 accumulate", "data": "synthetic",
+            "config": {"workload": "%s %dx%d %s s=%d k=%d; cache lookup R=%d C=%d q=%d; verify stride %d"
+                                   % (cfg.name, N, d, cfg.metric, s, k, R, cache.shape[1], stride, vstride),
+                       "variant": args.variant, "replicas": world,
+                       "l2": "inputs larger than L2 (%.1f GB corpus streamed every step)"
+                             % (corpus_bytes / 1e9) if corpus_bytes > 2.5e8 else
+                             "corpus near L2 size: L2-warm figure, not an HBM number"},
+            "scan_gbs": achieved, "scan_ms": scan_avg_ms, "scan_passes_per_step": passes,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"] if achieved else None,
+                         "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / 8000.0 if achieved else None,
+                         "kernel": "scan_kernel", "bytes_per_launch": corpus_bytes,
+                         "traffic": TRAFFIC_BYTES.get((cfg.name, N, s, k))},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
+            "gpu_launches": int(gpu_launches),
+            "clocks": clocks,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            out["cpu_baseline"] = cpu_baseline(corpus, queries, metric_id, k, N, s)
+        elif world > 1:
+            out["cpu_baseline"] = None
+        print(json.dumps(out))
+    idx.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per scan launch from the committed ncu capture
+# (profiles/), keyed by (workload, rows, s, k); absent = not captured for that shape.
+TRAFFIC_BYTES = {}
+
+if __name__ == "__main__":
+    main()

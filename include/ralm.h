@@ -134,6 +134,14 @@ ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant);
 /* Number of kernels the library launched on behalf of this index since creation. */
 int64_t ralm_index_launch_count(const ralm_index_t *idx);
 
+/* Time every scan-kernel launch of this index with a pair of CUDA events recorded on the
+ * caller's stream directly around the launch (measurement aid; off by default). */
+ralm_status_t ralm_index_set_timing(ralm_index_t *idx, int32_t enabled);
+
+/* Wait for the scan launches timed since the last read, return the sum of their durations in
+ * milliseconds and how many there were, and forget them. HOST pointers. */
+ralm_status_t ralm_index_read_timing(ralm_index_t *idx, double *total_ms, int64_t *launches);
+
 /* Static description of a status code. */
 const char *ralm_status_string(ralm_status_t status);
 

@@ -53,6 +53,10 @@ def load_library() -> ctypes.CDLL:
     lib.ralm_index_set_variant.argtypes = [p, i32]
     lib.ralm_index_launch_count.restype = i64
     lib.ralm_index_launch_count.argtypes = [p]
+    lib.ralm_index_set_timing.restype = i32
+    lib.ralm_index_set_timing.argtypes = [p, i32]
+    lib.ralm_index_read_timing.restype = i32
+    lib.ralm_index_read_timing.argtypes = [p, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
     lib.ralm_status_string.restype = ctypes.c_char_p
     lib.ralm_status_string.argtypes = [i32]
     _lib = lib
@@ -113,6 +117,16 @@ class Index:
 
     def launch_count(self) -> int:
         return self._lib.ralm_index_launch_count(self._handle)
+
+    def set_timing(self, enabled: bool):
+        _check(self._lib.ralm_index_set_timing(self._handle, int(enabled)), "ralm_index_set_timing")
+
+    def read_timing(self):
+        """(sum of scan-kernel durations in ms, number of launches) since the last read."""
+        ms, n = ctypes.c_double(), ctypes.c_int64()
+        _check(self._lib.ralm_index_read_timing(self._handle, ctypes.byref(ms), ctypes.byref(n)),
+               "ralm_index_read_timing")
+        return ms.value, n.value
 
     def device_status(self, stream=None) -> int:
         return self._lib.ralm_device_status(self._handle, _stream_ptr(stream))

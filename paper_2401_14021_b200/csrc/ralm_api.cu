@@ -6,6 +6,8 @@
 
 #include <algorithm>
 #include <new>
+#include <utility>
+#include <vector>
 
 #include "aux_kernels.cuh"
 #include "scan.cuh"
@@ -30,6 +32,10 @@ struct ralm_index {
     int64_t *h_ids;
     float *h_scores;
     int64_t launches;
+    // optional per-launch timing of the scan kernel (events on the caller's stream)
+    bool timing;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timed;   // recorded, not yet read
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> spare;   // reusable
 };
 
 namespace {
@@ -127,6 +133,17 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             p.off_cand = pl.off_cand;
             p.off_stage = pl.off_stage;
             cudaError_t e;
+            std::pair<cudaEvent_t, cudaEvent_t> ev{nullptr, nullptr};
+            if (idx->timing) {
+                if (!idx->spare.empty()) {
+                    ev = idx->spare.back();
+                    idx->spare.pop_back();
+                } else if (cudaEventCreate(&ev.first) != cudaSuccess ||
+                           cudaEventCreate(&ev.second) != cudaSuccess) {
+                    return RALM_ERR_CUDA;
+                }
+                cudaEventRecord(ev.first, st);
+            }
             if (mma) {
                 e = (k == 1) ? launch_scan<true, false, 8, 1, true>(p, grid, pl.smem_bytes, st)
                              : launch_scan<true, false, 8, 1, false>(p, grid, pl.smem_bytes, st);
@@ -134,6 +151,10 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
                 e = launch_fma<true>(p, grid, pl.smem_bytes, st);
             } else {
                 e = launch_fma<false>(p, grid, pl.smem_bytes, st);
+            }
+            if (idx->timing) {
+                cudaEventRecord(ev.second, st);
+                idx->timed.push_back(ev);
             }
             if (e != cudaSuccess) return RALM_ERR_CUDA;
             idx->launches++;
@@ -181,6 +202,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
     idx->variant = 0;
     idx->launches = 0;
+    idx->timing = false;
     const size_t partial_bytes = sizeof(uint64_t) * idx->num_sms * max_s * static_cast<size_t>(max_k);
     const size_t sk = static_cast<size_t>(max_s) * max_k;
     bool ok = cudaMalloc(&idx->partial, partial_bytes) == cudaSuccess;
@@ -210,6 +232,11 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
     cudaFree(idx->h_queries);
     cudaFree(idx->h_ids);
     cudaFree(idx->h_scores);
+    for (auto *list : {&idx->timed, &idx->spare})
+        for (auto &ev : *list) {
+            cudaEventDestroy(ev.first);
+            cudaEventDestroy(ev.second);
+        }
     delete idx;
     return RALM_OK;
 }
@@ -301,6 +328,34 @@ ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant) {
 }
 
 int64_t ralm_index_launch_count(const ralm_index_t *idx) { return idx ? idx->launches : 0; }
+
+ralm_status_t ralm_index_set_timing(ralm_index_t *idx, int32_t enabled) {
+    if (!idx) return RALM_ERR_INVALID_ARG;
+    idx->timing = enabled != 0;
+    return RALM_OK;
+}
+
+ralm_status_t ralm_index_read_timing(ralm_index_t *idx, double *total_ms, int64_t *launches) {
+    if (!idx || !total_ms || !launches) return RALM_ERR_INVALID_ARG;
+    double sum = 0.0;
+    int64_t n = 0;
+    ralm_status_t rs = RALM_OK;
+    for (auto &ev : idx->timed) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(ev.second) != cudaSuccess ||
+            cudaEventElapsedTime(&ms, ev.first, ev.second) != cudaSuccess) {
+            rs = RALM_ERR_CUDA;
+        } else {
+            sum += ms;
+            ++n;
+        }
+        idx->spare.push_back(ev);
+    }
+    idx->timed.clear();
+    *total_ms = sum;
+    *launches = n;
+    return rs;
+}
 
 const char *ralm_status_string(ralm_status_t status) {
     switch (status) {
