@@ -50,7 +50,8 @@ typedef enum {
     RALM_ERR_CUDA = 3,
     RALM_ERR_TIMEOUT = 4,
     RALM_ERR_UNSUPPORTED = 5,
-    RALM_ERR_BAD_CACHE_ID = 6
+    RALM_ERR_BAD_CACHE_ID = 6,
+    RALM_ERR_STATIC_LIMIT = 7
 } ralm_status_t;
 
 /* Limits checked by the host side. */
@@ -92,6 +93,44 @@ ralm_status_t ralm_search(ralm_index_t *idx, const void *queries, int32_t s, int
  * `stream`). Pinned host memory makes the copies asynchronous up to that point. */
 ralm_status_t ralm_search_host(ralm_index_t *idx, const void *queries_host, int32_t s,
                                int32_t k, int64_t *ids_host, float *scores_host, void *stream);
+
+/* Limits of ralm_search_static (below). */
+#define RALM_STATIC_MAX_S 8        /* queries per call */
+#define RALM_STATIC_MAX_K 32       /* neighbours per query */
+#define RALM_STATIC_MAX_BLOCKS 160 /* scan CTAs whose partial lists the scratch can hold */
+
+/* ralm_search for callers that must not allocate. (The paper has no counterpart: this entry
+ * point exists for the way the library gets embedded, not for the method.)
+ *
+ * Who needs it: code that runs where device allocation is off the table -- a serving process
+ * whose memory pool has already claimed the whole GPU and hands out no more, a real-time or
+ * safety-certified host loop that forbids allocator calls after start-up, or a plug-in that
+ * is handed buffers by its host application and has no right to create its own.
+ * ralm_index_create calls cudaMalloc for its workspace, so those callers cannot use it.
+ *
+ * This call needs no index and calls no cudaMalloc, cudaFree or any other allocating routine.
+ * The scan's scratch (per-CTA partial top-k lists) is a fixed array inside the library image:
+ * RALM_STATIC_MAX_BLOCKS * RALM_STATIC_MAX_S * RALM_STATIC_MAX_K * 8 bytes = 320 KiB (plus a
+ * 256-byte status block), held by every GPU that loads the library until the process exits.
+ *
+ *   corpus, N, d, metric   as for ralm_index_create (DEVICE fp16 [N][d], borrowed for the call)
+ *   queries                DEVICE fp16 [s][d], 16-byte aligned, 0 <= s <= RALM_STATIC_MAX_S
+ *   ids, scores            DEVICE int64 [s][k] / fp32 [s][k] (written), 1 <= k <= RALM_STATIC_MAX_K
+ *   device_status          DEVICE int32, may be NULL: zeroed by the call, then set to a
+ *                          ralm_status_t value if a device-side wait ran out
+ * Results are identical to ralm_search's. L2 needs d <= 1024 (as ralm_search does).
+ * Errors: RALM_ERR_STATIC_LIMIT when s or k exceeds the limits above (nothing is launched);
+ * INVALID_ARG, UNSUPPORTED, CUDA as elsewhere.
+ *
+ * The first call on each device looks up the scratch's device address and the device's
+ * properties (with that device current); make that first call before any stream capture.
+ * Every call on a device shares the one scratch array, which keeps the previous call's
+ * contents: the call clears what must start at zero itself, but two calls whose GPU work
+ * overlaps (different streams, different threads) race on it -- serialise them.
+ * Asynchronous on `stream`. */
+ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_metric_t metric,
+                                 const void *queries, int32_t s, int32_t k, int64_t *ids,
+                                 float *scores, int32_t *device_status, void *stream);
 
 /* Q.retrieve for R requests at once: request r owns C cache slots holding corpus ids
  * (-1 = empty slot; the cache is a set, a repeated id counts once) and q queries; each

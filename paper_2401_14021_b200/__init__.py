@@ -5,7 +5,7 @@ library; torch is used for device memory and streams only. There is no CPU fallb
 the compiled library is missing or no CUDA device is present, calls raise.
 """
 from .binding import (IP, L2, Index, RalmError, cache_search, lib_path, load_library, search,
-                      search_host, verify, STATUS_NAMES)
+                      search_host, search_static, verify, STATUS_NAMES)
 
 __all__ = ["IP", "L2", "Index", "RalmError", "cache_search", "lib_path", "load_library", "search",
-           "search_host", "verify", "STATUS_NAMES"]
+           "search_host", "search_static", "verify", "STATUS_NAMES"]

@@ -8,7 +8,8 @@ IP = 0
 L2 = 1
 
 STATUS_NAMES = {0: "RALM_OK", 1: "RALM_ERR_INVALID_ARG", 2: "RALM_ERR_OOM", 3: "RALM_ERR_CUDA",
-                4: "RALM_ERR_TIMEOUT", 5: "RALM_ERR_UNSUPPORTED", 6: "RALM_ERR_BAD_CACHE_ID"}
+                4: "RALM_ERR_TIMEOUT", 5: "RALM_ERR_UNSUPPORTED", 6: "RALM_ERR_BAD_CACHE_ID",
+                7: "RALM_ERR_STATIC_LIMIT"}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _lib = None
@@ -43,6 +44,8 @@ def load_library() -> ctypes.CDLL:
     lib.ralm_search.argtypes = [p, p, i32, i32, p, p, p]
     lib.ralm_search_host.restype = i32
     lib.ralm_search_host.argtypes = [p, p, i32, i32, p, p, p]
+    lib.ralm_search_static.restype = i32
+    lib.ralm_search_static.argtypes = [p, i64, i32, i32, p, i32, i32, p, p, p, p]
     lib.ralm_cache_search.restype = i32
     lib.ralm_cache_search.argtypes = [p, p, i32, i32, p, i32, i32, p, p, p]
     lib.ralm_verify.restype = i32
@@ -156,6 +159,26 @@ def search_host(index: Index, queries: torch.Tensor, k: int, ids: torch.Tensor, 
             raise TypeError("host tensors must be contiguous CPU tensors of the right dtype")
     _check(index._lib.ralm_search_host(index.handle, queries.data_ptr(), s, k, ids.data_ptr(),
                                        scores.data_ptr(), _stream_ptr(stream)), "ralm_search_host")
+    return ids, scores
+
+
+def search_static(corpus: torch.Tensor, metric: int, queries: torch.Tensor, k: int,
+                  ids: torch.Tensor, scores: torch.Tensor, device_status: torch.Tensor = None,
+                  stream=None):
+    """ralm_search_static: the search for callers that cannot allocate device memory. No
+    index; the caller brings every buffer (ids int64 [s][k], scores fp32 [s][k], optionally a
+    one-element int32 status tensor) and the library uses its built-in scratch. This wrapper
+    allocates nothing either."""
+    lib = load_library()
+    s = queries.shape[0]
+    N, d = corpus.shape
+    _check(lib.ralm_search_static(_dev(corpus, torch.float16, "corpus") if N else 0, N, d, metric,
+                                  _dev(queries, torch.float16, "queries") if s else 0, s, k,
+                                  _dev(ids, torch.int64, "ids") if s else 0,
+                                  _dev(scores, torch.float32, "scores") if s else 0,
+                                  _dev(device_status, torch.int32, "device_status")
+                                  if device_status is not None else 0,
+                                  _stream_ptr(stream)), "ralm_search_static")
     return ids, scores
 
 

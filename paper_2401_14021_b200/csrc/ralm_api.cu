@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <utility>
 #include <vector>
@@ -171,6 +172,60 @@ bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 }  // namespace
 
+// ---------------------------------------------------------------------------------------
+// Scratch for ralm_search_static. It lives in the library image itself: every GPU that loads
+// the library holds these bytes until the process exits, whether or not the call is used.
+// Layout: [blocks][s][k] sorted partial top-k keys, exactly what the scan hands to the merge.
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned long long
+    g_static_partial[RALM_STATIC_MAX_BLOCKS * RALM_STATIC_MAX_S * RALM_STATIC_MAX_K];
+static __device__ __align__(256) int g_static_status[64];
+
+namespace {
+
+constexpr int kStaticMaxDevices = 64;
+
+struct StaticDeviceState {
+    bool ready = false;
+    uint64_t *partial = nullptr;  // device address of g_static_partial on this device
+    int *status = nullptr;        // device address of g_static_status on this device
+    int num_sms = 0;
+    int smem_optin = 0;
+    int cc_major = 0;
+};
+StaticDeviceState g_static_state[kStaticMaxDevices];
+std::mutex g_static_mutex;
+
+// One-time set-up per device, with that device current. In host code the array names above
+// are only handles; the addresses a kernel can use come from cudaGetSymbolAddress.
+ralm_status_t static_state_for_current_device(StaticDeviceState **out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return RALM_ERR_CUDA;
+    if (dev < 0 || dev >= kStaticMaxDevices) return RALM_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDeviceState &st = g_static_state[dev];
+    if (!st.ready) {
+        void *partial = nullptr, *status = nullptr;
+        if (cudaGetSymbolAddress(&partial, g_static_partial) != cudaSuccess) return RALM_ERR_CUDA;
+        if (cudaGetSymbolAddress(&status, g_static_status) != cudaSuccess) return RALM_ERR_CUDA;
+        int sms = 0, smem = 0, major = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+            return RALM_ERR_CUDA;
+        st.partial = static_cast<uint64_t *>(partial);
+        st.status = static_cast<int *>(status);
+        st.num_sms = sms;
+        st.smem_optin = smem;
+        st.cc_major = major;
+        st.ready = true;
+    }
+    *out = &st;
+    return RALM_OK;
+}
+
+}  // namespace
+
 extern "C" {
 
 ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_metric_t metric,
@@ -327,6 +382,50 @@ ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant) {
     return RALM_OK;
 }
 
+ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_metric_t metric,
+                                 const void *queries, int32_t s, int32_t k, int64_t *ids,
+                                 float *scores, int32_t *device_status, void *stream) {
+    if (N < 0 || N >= (int64_t{1} << 31) || (!corpus && N > 0) || !aligned16(corpus))
+        return RALM_ERR_INVALID_ARG;
+    if (d < 8 || d > RALM_MAX_D || d % 8 != 0) return RALM_ERR_INVALID_ARG;
+    if (metric != RALM_IP && metric != RALM_L2) return RALM_ERR_INVALID_ARG;
+    if (s < 0 || k < 1) return RALM_ERR_INVALID_ARG;
+    if (s > RALM_STATIC_MAX_S || k > RALM_STATIC_MAX_K) return RALM_ERR_STATIC_LIMIT;
+    if (s == 0) return RALM_OK;
+    if (!queries || !ids || !scores || !aligned16(queries)) return RALM_ERR_INVALID_ARG;
+    StaticDeviceState *dev = nullptr;
+    ralm_status_t rs = static_state_for_current_device(&dev);
+    if (rs != RALM_OK) return rs;
+    if (dev->cc_major != 10) return RALM_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int *status = device_status ? device_status : dev->status;
+    // the scratch keeps whatever the previous call left; the partial lists are fully
+    // rewritten by the scan, the status word is the one thing that must start at zero
+    if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return RALM_ERR_CUDA;
+    // a handle on the stack that points the ordinary search path at the static scratch
+    ralm_index view;
+    view.corpus = static_cast<const __half *>(corpus);
+    view.N = N;
+    view.d = d;
+    view.metric = metric;
+    view.max_s = RALM_STATIC_MAX_S;
+    view.max_k = RALM_STATIC_MAX_K;
+    view.device = 0;
+    view.num_sms = std::min(dev->num_sms, RALM_STATIC_MAX_BLOCKS);
+    view.smem_optin = dev->smem_optin;
+    view.variant = 0;
+    view.partial = dev->partial;
+    view.cache_keys = nullptr;
+    view.status = status;
+    view.h_queries = nullptr;
+    view.h_ids = nullptr;
+    view.h_scores = nullptr;
+    view.launches = 0;
+    view.timing = false;
+    if (view.metric == RALM_L2 && d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
+    return search_device(&view, static_cast<const __half *>(queries), s, k, ids, scores, st);
+}
+
 int64_t ralm_index_launch_count(const ralm_index_t *idx) { return idx ? idx->launches : 0; }
 
 ralm_status_t ralm_index_set_timing(ralm_index_t *idx, int32_t enabled) {
@@ -366,6 +465,8 @@ const char *ralm_status_string(ralm_status_t status) {
         case RALM_ERR_TIMEOUT: return "a device-side wait ran out";
         case RALM_ERR_UNSUPPORTED: return "unsupported device, shape or variant";
         case RALM_ERR_BAD_CACHE_ID: return "a cache id was outside [-1, N)";
+        case RALM_ERR_STATIC_LIMIT:
+            return "s or k exceeds what the built-in scratch of ralm_search_static can hold";
     }
     return "unknown status";
 }
