@@ -94,12 +94,14 @@ __device__ __forceinline__ void named_barrier(int id, int nthreads) {
 
 // ---------------------------------------------------------------------------------
 // Bitonic sort (descending) of P = 2^n keys in shared memory by a group of `nthr`
-// threads with ranks `tid`, synchronised through named barrier `bar_id` (or
-// __syncthreads when bar_id < 0). All threads of the group must call it.
+// threads with ranks `tid`, synchronised through group_sync(bar_id). All threads of the
+// group must call it.
 // ---------------------------------------------------------------------------------
+// bar_id >= 0: named barrier over nthr threads; -1: the whole CTA; -2: one warp.
 __device__ __forceinline__ void group_sync(int bar_id, int nthr) {
-    if (bar_id < 0) __syncthreads();
-    else named_barrier(bar_id, nthr);
+    if (bar_id >= 0) named_barrier(bar_id, nthr);
+    else if (bar_id == -1) __syncthreads();
+    else __syncwarp();
 }
 __device__ inline void bitonic_sort_desc(uint64_t *a, int P, int tid, int nthr, int bar_id) {
     for (int size = 2; size <= P; size <<= 1) {

@@ -42,27 +42,37 @@ struct ralm_index {
 namespace {
 
 struct ScanPlan {
-    int nstages, stage_bytes, cap, off_q, off_cand, off_stage, smem_bytes;
+    int nwarps, depth, tile_rows, stage_bytes, cap, soft_limit, off_q, off_cand, off_stage, smem_bytes;
 };
 
 int align_up(int v, int a) { return (v + a - 1) / a * a; }
 
-// Shared-memory layout of one scan CTA. Returns false if not even one stage fits.
+// Shared-memory layout of one scan CTA. Returns false if not even two stages fit.
 bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl) {
-    pl->stage_bytes = align_up(kTileRows * idx->d * 2, 128);
+    // warp-MMA tiles are 16 rows (the M of m16n8k16). The FMA flavour is bound by its
+    // arithmetic, so it wants many small tiles: several being scored while more are in flight.
+    pl->nwarps = mma ? kMaxConsumerWarps : kMaxConsumerWarps - 1;
+    pl->tile_rows = mma ? 16 : (s_pass == 1 ? 16 : 4);
+    pl->stage_bytes = align_up(pl->tile_rows * idx->d * 2, 128);
     pl->off_q = kScanHeaderBytes;
     int off = pl->off_q + (mma ? align_up(kScanMaxQueries * (idx->d * 2 + kQueryPadBytes), 128) : 0);
     pl->off_cand = off;
     pl->cap = 0;
+    pl->soft_limit = 0;
     if (k > 1) {
+        // after the flag is raised every warp may still finish the tile it is on
         pl->cap = std::max(512, 2 * next_pow2(k));
+        pl->soft_limit = pl->cap - (kMaxConsumerWarps + 1) * pl->tile_rows;
         off += s_pass * pl->cap * 8;
     }
     pl->off_stage = align_up(off, 128);
     const int room = idx->smem_optin - pl->off_stage;
-    if (room < pl->stage_bytes) return false;
-    pl->nstages = std::min(kMaxStages, room / pl->stage_bytes);
-    pl->smem_bytes = pl->off_stage + pl->nstages * pl->stage_bytes;
+    const int fit = std::min(kMaxStages, room / pl->stage_bytes);
+    if (fit < 2) return false;
+    // every consumer warp owns `depth` stages; fewer warps when the stages are large
+    pl->nwarps = std::min(pl->nwarps, fit);
+    pl->depth = std::min(fit / pl->nwarps, 3);
+    pl->smem_bytes = pl->off_stage + pl->nwarps * pl->depth * pl->stage_bytes;
     return true;
 }
 
@@ -71,7 +81,7 @@ cudaError_t launch_scan(const ScanParams &p, int grid, int smem, cudaStream_t st
     auto kern = scan_kernel<MMA, L2, SQ, DP, TOP1>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, 32 * (p.nstages + 1), smem, st>>>(p);
+    kern<<<grid, 32 * (p.nwarps + 1), smem, st>>>(p);
     return cudaGetLastError();
 }
 
@@ -108,8 +118,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     const bool mma = variant == 2;
     if (!mma && idx->d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
     const int per_pass = mma ? kScanMaxQueries : kFmaQueriesPerPass;
-    const long long ntiles = (idx->N + kTileRows - 1) / kTileRows;
-    const int grid = static_cast<int>(std::min<long long>(idx->num_sms, ntiles));
+    const int grid = static_cast<int>(std::min<long long>(idx->num_sms, (idx->N + 15) / 16));
     if (grid > 0) {
         for (int q0 = 0; q0 < s; q0 += per_pass) {
             const int sp = std::min(per_pass, s - q0);
@@ -121,14 +130,17 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             p.partial = idx->partial;
             p.status = idx->status;
             p.N = idx->N;
-            p.ntiles = ntiles;
+            p.ntiles = (idx->N + pl.tile_rows - 1) / pl.tile_rows;
             p.d = idx->d;
             p.s = sp;
             p.s_total = s;
             p.q_base = q0;
             p.k = k;
             p.cap = pl.cap;
-            p.nstages = pl.nstages;
+            p.soft_limit = pl.soft_limit;
+            p.tile_rows = pl.tile_rows;
+            p.nwarps = pl.nwarps;
+            p.depth = pl.depth;
             p.stage_bytes = pl.stage_bytes;
             p.off_q = pl.off_q;
             p.off_cand = pl.off_cand;

@@ -1,10 +1,11 @@
 // Corpus scan for small query batches (at most 8 queries per pass): scores every corpus
 // row against every query and keeps, per CTA and query, the best k rows.
 //
-// One persistent CTA per SM. Warp 0 is the producer: one thread streams 16-row tiles of
-// the row-major corpus (a tile is one contiguous block of memory) into a ring of shared
-// memory stages with 1-D bulk copies that complete on mbarriers. Every other warp owns one
-// stage: it waits for its tile, scores it, hands the stage back, and keeps candidates.
+// One persistent CTA per SM. Warp 0 is the producer: one thread streams tiles of whole rows
+// of the row-major corpus (a tile is one contiguous block of memory) into shared-memory
+// stages with 1-D bulk copies that complete on mbarriers. The consumer warps take the tiles
+// round-robin, each through a private ring of stages: wait for the tile, score it, hand the
+// stage back, keep candidates.
 //
 // Two ways of scoring a tile:
 //   FMA flavour: each lane holds its slice of every query in registers (fp32, packed
@@ -16,19 +17,21 @@
 //     same way for rows and queries) so that each lane reads 16 contiguous bytes per row.
 //
 // Selection: k == 1 keeps a running best key per thread. k > 1 uses a per-query threshold
-// (the current k-th best of this CTA) and a shared-memory candidate buffer; consumer warps
-// advance in lock-step rounds so that the buffer can be compacted (sorted, truncated to k,
-// threshold raised) before it could overflow.
+// (the current k-th best of this CTA) and a shared-memory candidate buffer. A push that lands
+// near the end of a buffer raises a flag; every consumer warp polls the flag while it waits
+// for a tile and all of them meet to compact (sort, keep k, raise the threshold) the buffers,
+// spread over the warps, before any buffer can overflow: after the flag is up each warp
+// pushes at most the rest of the tile it is on.
 #pragma once
 
 #include "common.cuh"
 
 namespace ralm {
 
-constexpr int kTileRows = 16;
-constexpr int kMaxStages = 7;
+constexpr int kMaxStages = 24;
+constexpr int kMaxConsumerWarps = 8;
 constexpr int kScanMaxQueries = 8;
-constexpr int kScanThreads = 32 * (kMaxStages + 1);
+constexpr int kScanThreads = 32 * (kMaxConsumerWarps + 1);
 constexpr int kQueryPadBytes = 64;
 
 struct ScanParams {
@@ -43,8 +46,11 @@ struct ScanParams {
     int s_total;  // queries of the whole call (layout of `partial`)
     int q_base;   // index of this pass's first query in the call
     int k;
-    int cap;      // candidate buffer capacity per query (power of two); unused when k == 1
-    int nstages;  // ring depth = number of consumer warps
+    int cap;         // candidate buffer capacity per query (power of two); unused when k == 1
+    int soft_limit;  // a push into a slot >= soft_limit asks for a compaction
+    int tile_rows;   // rows per tile (16 for the warp-MMA flavour)
+    int nwarps;      // consumer warps; warp w owns stages w, w + nwarps, ... (a private ring)
+    int depth;       // stages per consumer warp
     int stage_bytes;
     int off_q;  // shared-memory offsets (bytes)
     int off_cand;
@@ -58,25 +64,65 @@ struct ScanHeader {
     float thr[kScanMaxQueries];
     int cnt[kScanMaxQueries];
     int abort;
+    int flag;  // some query's candidate buffer is nearly full: everyone meet and compact
+    int done;  // consumer warps that have finished their tiles
 };
-constexpr int kScanHeaderBytes = 512;
+constexpr int kScanHeaderBytes = 1024;
 static_assert(sizeof(ScanHeader) <= kScanHeaderBytes, "header too large");
 
-// Sort query q's candidates, keep the best k, raise the threshold. Called by all consumer
-// threads (group of `nthr`, ranks `tid`, named barrier 1).
+// Sort query q's candidates, keep the best k, raise the threshold. Called by a group of
+// `nthr` threads with ranks `tid`, synchronised through group_sync(bar_id).
 __device__ inline void compact_query(ScanHeader *hdr, uint64_t *cand, int cap, int q, int k,
-                                     int tid, int nthr) {
+                                     int tid, int nthr, int bar_id) {
     uint64_t *a = cand + static_cast<size_t>(q) * cap;
     const int n = hdr->cnt[q];
     const int P = next_pow2(n > 1 ? n : 2);
     for (int i = n + tid; i < P; i += nthr) a[i] = 0;
-    named_barrier(1, nthr);
-    bitonic_sort_desc(a, P, tid, nthr, 1);
+    group_sync(bar_id, nthr);
+    bitonic_sort_desc(a, P, tid, nthr, bar_id);
     if (tid == 0) {
         hdr->cnt[q] = n < k ? n : k;
         hdr->thr[q] = (n >= k) ? key_value(a[k - 1]) : -INFINITY;
     }
-    named_barrier(1, nthr);
+    group_sync(bar_id, nthr);
+}
+
+// All W consumer warps (this one is w) compact every query that holds more than `min_count`
+// candidates; the queries are spread over groups of warps that sort in parallel. Must be
+// called by all W * 32 consumer threads, with no push in flight.
+__device__ inline void compact_all(ScanHeader *hdr, uint64_t *cand, int cap, int s, int k,
+                                   int min_count, int w, int lane, int W) {
+    int list[kScanMaxQueries];
+    int nq = 0;
+#pragma unroll
+    for (int q = 0; q < kScanMaxQueries; ++q)
+        if (q < s && hdr->cnt[q] > min_count) list[nq++] = q;
+    // nobody may start rewriting cnt[] before everybody has taken the same snapshot of it
+    named_barrier(1, W * 32);
+    if (nq == 0) return;
+    const int ngroups = nq < W ? nq : W;
+    const int G = W / ngroups;  // warps per group
+    const int group = w / G;
+    if (group >= ngroups) return;
+    const int tid = (w - group * G) * 32 + lane;
+    const int bar_id = (G == 1) ? -2 : 2 + group;
+    for (int i = group; i < nq; i += ngroups) {
+        int q = 0;
+#pragma unroll
+        for (int j = 0; j < kScanMaxQueries; ++j)
+            if (j == i) q = list[j];
+        compact_query(hdr, cand, cap, q, k, tid, G * 32, bar_id);
+    }
+}
+
+// The meeting itself: barrier, compact, lower the flag, barrier.
+__device__ __forceinline__ void compaction_meeting(ScanHeader *hdr, uint64_t *cand,
+                                                   const int cap, const int s, const int k, int w,
+                                                   int lane, int W) {
+    named_barrier(1, W * 32);
+    compact_all(hdr, cand, cap, s, k, k, w, lane, W);
+    if (w == 0 && lane == 0) *reinterpret_cast<volatile int *>(&hdr->flag) = 0;
+    named_barrier(1, W * 32);
 }
 
 // FMA flavour: transposing shuffle reduction. On entry every lane holds V partial sums
@@ -120,34 +166,40 @@ __device__ __forceinline__ float2 h2_to_f2(uint32_t h2) {
     return __half22float2(*reinterpret_cast<const __half2 *>(&h2));
 }
 
-__device__ __forceinline__ void push_candidate(ScanHeader *hdr, uint64_t *cand, int cap, int q,
-                                               uint64_t key) {
+__device__ __forceinline__ void push_candidate(ScanHeader *hdr, uint64_t *cand, int cap, int soft,
+                                               int q, uint64_t key) {
     const int slot = atomicAdd(&hdr->cnt[q], 1);
     cand[static_cast<size_t>(q) * cap + slot] = key;
+    if (slot >= soft) *reinterpret_cast<volatile int *>(&hdr->flag) = 1;
 }
 
 // ------------------------------------------------------------------------------------
 // The kernel. MMA: warp-MMA flavour (inner product only) or FMA flavour.
-// L2: metric of the FMA flavour. SQ: queries held per lane (1, 2 or 4; FMA flavour).
+// L2: metric of the FMA flavour. SQ: queries held per lane (1 or 4; FMA flavour).
 // DP: 16-byte pieces of a row per lane (d <= 256 * DP; FMA flavour). TOP1: k == 1.
 // ------------------------------------------------------------------------------------
 template <bool MMA, bool L2, int SQ, int DP, bool TOP1>
-__global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams p) {
+__global__ void __launch_bounds__(MMA ? kScanThreads : kScanThreads - 32, 1)
+scan_kernel(const ScanParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     ScanHeader *hdr = reinterpret_cast<ScanHeader *>(smem);
     uint64_t *cand = reinterpret_cast<uint64_t *>(smem + p.off_cand);
-    const int W = p.nstages;
+    const int W = p.nwarps;
+    const int S = W * p.depth;
+    const int T = p.tile_rows;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int d = p.d;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < W; ++i) {
+        for (int i = 0; i < S; ++i) {
             mbar_init(smem_u32(&hdr->full[i]), 1);
             mbar_init(smem_u32(&hdr->empty[i]), 1);
         }
         mbar_fence_init();
         hdr->abort = 0;
+        hdr->flag = 0;
+        hdr->done = 0;
     }
     if (threadIdx.x < kScanMaxQueries) {
         hdr->thr[threadIdx.x] = -INFINITY;
@@ -170,6 +222,8 @@ __global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams 
     const long long my_tiles =
         (p.ntiles > blockIdx.x) ? (p.ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
     volatile int *abort_flag = &hdr->abort;
+    volatile int *compact_flag = &hdr->flag;
+    volatile int *done_count = &hdr->done;
 
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
@@ -177,16 +231,19 @@ __global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams 
             long long issued = 0;
             bool ok = true;
             for (long long it = 0; it < my_tiles; ++it) {
-                const int st = static_cast<int>(it % W);
-                const long long use = it / W;
+                // tile `it` belongs to consumer warp it % W; it is that warp's (it / W)-th
+                // tile and goes to the warp's private ring of `depth` stages
+                const long long local = it / W;
+                const int st = static_cast<int>(it % W) + static_cast<int>(local % p.depth) * W;
+                const long long use = local / p.depth;
                 if (use > 0) {
                     ok = mbar_wait_bounded(smem_u32(&hdr->empty[st]), (use - 1) & 1);
                     if (!ok) break;
                 }
                 if (*abort_flag) break;
                 const long long tile = blockIdx.x + it * static_cast<long long>(gridDim.x);
-                const long long row0 = tile * kTileRows;
-                const long long rows = (p.N - row0 < kTileRows) ? (p.N - row0) : kTileRows;
+                const long long row0 = tile * T;
+                const long long rows = (p.N - row0 < T) ? (p.N - row0) : T;
                 const uint32_t bytes = static_cast<uint32_t>(rows * d * 2);
                 const uint32_t bar = smem_u32(&hdr->full[st]);
                 mbar_arrive_expect_tx(bar, bytes);
@@ -200,8 +257,11 @@ __global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams 
             }
             if (*abort_flag) {
                 // winding down early: let every copy already issued land before exit
-                for (long long it = (issued > W ? issued - W : 0); it < issued; ++it)
-                    mbar_wait_bounded(smem_u32(&hdr->full[it % W]), (it / W) & 1);
+                for (long long it = (issued > S ? issued - S : 0); it < issued; ++it) {
+                    const long long local = it / W;
+                    mbar_wait_bounded(smem_u32(&hdr->full[(it % W) + (local % p.depth) * W]),
+                                      (local / p.depth) & 1);
+                }
             }
         }
     } else if (warp - 1 < W) {
@@ -209,9 +269,6 @@ __global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams 
         const int w = warp - 1;
         const int ctid = threadIdx.x - 32;
         const int cthreads = W * 32;
-        const uint32_t stage_addr =
-            smem_u32(smem + p.off_stage + static_cast<size_t>(w) * p.stage_bytes);
-        const long long rounds = (my_tiles + W - 1) / W;
         const int g = lane >> 2, t = lane & 3;
 
         uint64_t best0 = 0, best1 = 0;
@@ -243,148 +300,171 @@ __global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams 
                 }
         }
 
-        for (long long j = 0; j < rounds; ++j) {
-            const long long it = j * W + w;
-            if (it < my_tiles && !*abort_flag) {
-                if (!mbar_wait_bounded(smem_u32(&hdr->full[w]), j & 1)) {
+        for (long long it = w; it < my_tiles; it += W) {
+            if (*abort_flag) continue;
+            // this warp's private ring: only this warp ever waits on these stages, in order,
+            // so a parity wait can never be satisfied by an older phase
+            const long long local = it / W;
+            const int st = w + static_cast<int>(local % p.depth) * W;
+            const uint32_t full_bar = smem_u32(&hdr->full[st]);
+            const uint32_t parity = (local / p.depth) & 1;
+            // Wait for the tile. Lane 0 polls; a raised compaction flag takes priority over a
+            // ready tile (after the flag is up a warp finishes at most the tile it is on), and
+            // a warp still waiting for its tile joins the meeting instead of blocking it.
+            bool have_tile = false;
+            {
+                const long long t0 = clock64();
+                int spins = 0;
+                while (!have_tile) {
+                    int state = 0;  // 1 tile ready, 2 compaction requested, 3 gave up
                     if (lane == 0) {
-                        atomicMax(p.status, kStatusTimeout);
-                        *abort_flag = 1;
+                        if (!TOP1 && *compact_flag) state = 2;
+                        else if (mbar_try_wait(full_bar, parity)) state = 1;
+                        else if ((++spins & 1023) == 0 && clock64() - t0 > kWaitCycleLimit) state = 3;
+                    }
+                    state = __shfl_sync(0xffffffffu, state, 0);
+                    if (state == 1) {
+                        while (!mbar_try_wait(full_bar, parity)) {}  // completed: returns at once
+                        have_tile = true;
+                    } else if (state == 2) {
+                        compaction_meeting(hdr, cand, p.cap, p.s, p.k, w, lane, W);
+                    } else if (state == 3) {
+                        if (lane == 0) {
+                            atomicMax(p.status, kStatusTimeout);
+                            *abort_flag = 1;
+                        }
+                        break;
+                    }
+                }
+            }
+            if (!have_tile) continue;
+            const uint32_t stage_addr =
+                smem_u32(smem + p.off_stage + static_cast<size_t>(st) * p.stage_bytes);
+            const uint32_t empty_bar = smem_u32(&hdr->empty[st]);
+            const long long tile = blockIdx.x + it * static_cast<long long>(gridDim.x);
+            const long long row0 = tile * T;
+            if (MMA) {
+                // ---- 16 rows x 8 queries on tensor cores; two accumulator sets halve the
+                // dependent chain
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                float acc_b[4] = {0.f, 0.f, 0.f, 0.f};
+                const int nchunks = (d + 31) >> 5;
+                const uint32_t q_addr = smem_u32(smem + p.off_q) + g * (d * 2 + kQueryPadBytes);
+                const uint32_t a_lo_addr = stage_addr + g * d * 2;
+                const uint32_t a_hi_addr = stage_addr + (g + 8) * d * 2;
+#pragma unroll 4
+                for (int c = 0; c < nchunks; ++c) {
+                    // logical k (2t, 2t+1, 2t+8, 2t+9 of two MMAs) <- physical halves
+                    // off..off+7, the same permutation for every row and query
+                    const int off = c * 32 + t * 8;
+                    uint4 b = make_uint4(0, 0, 0, 0), lo = b, hi = b;
+                    if (off < d) {  // ragged last chunk: absent pieces stay zero
+                        b = lds128(q_addr + off * 2);
+                        lo = lds128(a_lo_addr + off * 2);
+                        hi = lds128(a_hi_addr + off * 2);
+                    }
+                    mma_m16n8k16(acc, lo.x, hi.x, lo.y, hi.y, b.x, b.y);
+                    mma_m16n8k16(acc_b, lo.z, hi.z, lo.w, hi.w, b.z, b.w);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[i] += acc_b[i];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_bar);
+                // acc[0]: (row g, query 2t)     acc[1]: (row g, query 2t+1)
+                // acc[2]: (row g+8, query 2t)   acc[3]: (row g+8, query 2t+1)
+                const long long r_lo = row0 + g, r_hi = row0 + g + 8;
+                const int q0 = 2 * t, q1 = 2 * t + 1;
+                if (TOP1) {
+                    if (r_lo < p.N) {
+                        const uint64_t k0 = make_key(acc[0], static_cast<uint32_t>(r_lo));
+                        const uint64_t k1 = make_key(acc[1], static_cast<uint32_t>(r_lo));
+                        best0 = k0 > best0 ? k0 : best0;
+                        best1 = k1 > best1 ? k1 : best1;
+                    }
+                    if (r_hi < p.N) {
+                        const uint64_t k0 = make_key(acc[2], static_cast<uint32_t>(r_hi));
+                        const uint64_t k1 = make_key(acc[3], static_cast<uint32_t>(r_hi));
+                        best0 = k0 > best0 ? k0 : best0;
+                        best1 = k1 > best1 ? k1 : best1;
                     }
                 } else {
-                    const long long tile = blockIdx.x + it * static_cast<long long>(gridDim.x);
-                    const long long row0 = tile * kTileRows;
-                    if (MMA) {
-                        // ---- 16 rows x 8 queries on tensor cores
-                        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                        const int nchunks = (d + 31) >> 5;
-                        const uint32_t q_addr = smem_u32(smem + p.off_q) + g * (d * 2 + kQueryPadBytes);
-                        const uint32_t a_lo_addr = stage_addr + g * d * 2;
-                        const uint32_t a_hi_addr = stage_addr + (g + 8) * d * 2;
-#pragma unroll 4
-                        for (int c = 0; c < nchunks; ++c) {
-                            // logical k (2t, 2t+1, 2t+8, 2t+9 of two MMAs) <- physical halves
-                            // off..off+7, the same permutation for every row and query
-                            const int off = c * 32 + t * 8;
-                            uint4 b = make_uint4(0, 0, 0, 0), lo = b, hi = b;
-                            if (off < d) {  // ragged last chunk: absent pieces stay zero
-                                b = lds128(q_addr + off * 2);
-                                lo = lds128(a_lo_addr + off * 2);
-                                hi = lds128(a_hi_addr + off * 2);
-                            }
-                            mma_m16n8k16(acc, lo.x, hi.x, lo.y, hi.y, b.x, b.y);
-                            mma_m16n8k16(acc, lo.z, hi.z, lo.w, hi.w, b.z, b.w);
-                        }
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[w]));
-                        // acc[0]: (row g, query 2t)     acc[1]: (row g, query 2t+1)
-                        // acc[2]: (row g+8, query 2t)   acc[3]: (row g+8, query 2t+1)
-                        const long long r_lo = row0 + g, r_hi = row0 + g + 8;
-                        const int q0 = 2 * t, q1 = 2 * t + 1;
-                        if (TOP1) {
-                            if (r_lo < p.N) {
-                                const uint64_t k0 = make_key(acc[0], static_cast<uint32_t>(r_lo));
-                                const uint64_t k1 = make_key(acc[1], static_cast<uint32_t>(r_lo));
-                                best0 = k0 > best0 ? k0 : best0;
-                                best1 = k1 > best1 ? k1 : best1;
-                            }
-                            if (r_hi < p.N) {
-                                const uint64_t k0 = make_key(acc[2], static_cast<uint32_t>(r_hi));
-                                const uint64_t k1 = make_key(acc[3], static_cast<uint32_t>(r_hi));
-                                best0 = k0 > best0 ? k0 : best0;
-                                best1 = k1 > best1 ? k1 : best1;
-                            }
-                        } else {
-                            const float th0 = hdr->thr[q0], th1 = hdr->thr[q1];
-                            if (r_lo < p.N) {
-                                if (q0 < p.s && acc[0] >= th0)
-                                    push_candidate(hdr, cand, p.cap, q0,
-                                                   make_key(acc[0], static_cast<uint32_t>(r_lo)));
-                                if (q1 < p.s && acc[1] >= th1)
-                                    push_candidate(hdr, cand, p.cap, q1,
-                                                   make_key(acc[1], static_cast<uint32_t>(r_lo)));
-                            }
-                            if (r_hi < p.N) {
-                                if (q0 < p.s && acc[2] >= th0)
-                                    push_candidate(hdr, cand, p.cap, q0,
-                                                   make_key(acc[2], static_cast<uint32_t>(r_hi)));
-                                if (q1 < p.s && acc[3] >= th1)
-                                    push_candidate(hdr, cand, p.cap, q1,
-                                                   make_key(acc[3], static_cast<uint32_t>(r_hi)));
-                            }
-                        }
-                    } else {
-                        // ---- FMA flavour: RG rows at a time, RG * SQ = 16 partial sums
-                        constexpr int RG = 16 / SQR;
-                        constexpr int V = 16;
+                    const float th0 = hdr->thr[q0], th1 = hdr->thr[q1];
+                    if (r_lo < p.N) {
+                        if (q0 < p.s && acc[0] >= th0)
+                            push_candidate(hdr, cand, p.cap, p.soft_limit, q0,
+                                           make_key(acc[0], static_cast<uint32_t>(r_lo)));
+                        if (q1 < p.s && acc[1] >= th1)
+                            push_candidate(hdr, cand, p.cap, p.soft_limit, q1,
+                                           make_key(acc[1], static_cast<uint32_t>(r_lo)));
+                    }
+                    if (r_hi < p.N) {
+                        if (q0 < p.s && acc[2] >= th0)
+                            push_candidate(hdr, cand, p.cap, p.soft_limit, q0,
+                                           make_key(acc[2], static_cast<uint32_t>(r_hi)));
+                        if (q1 < p.s && acc[3] >= th1)
+                            push_candidate(hdr, cand, p.cap, p.soft_limit, q1,
+                                           make_key(acc[3], static_cast<uint32_t>(r_hi)));
+                    }
+                }
+            } else {
+                // ---- FMA flavour: RG rows at a time, RG * SQ = 16 partial sums
+                constexpr int RG = 16 / SQR;
+                constexpr int V = 16;
 #pragma unroll 1
-                        for (int rg = 0; rg < kTileRows; rg += RG) {
-                            float2 acc2[RG][SQR];
+                for (int rg = 0; rg < T; rg += RG) {
+                    float2 acc2[RG][SQR];
 #pragma unroll
-                            for (int r = 0; r < RG; ++r)
+                    for (int r = 0; r < RG; ++r)
 #pragma unroll
-                                for (int jq = 0; jq < SQR; ++jq) acc2[r][jq] = make_float2(0.f, 0.f);
+                        for (int jq = 0; jq < SQR; ++jq) acc2[r][jq] = make_float2(0.f, 0.f);
 #pragma unroll
-                            for (int i = 0; i < DPR; ++i) {
-                                const int piece = lane + 32 * i;
-                                if (piece * 8 < d) {
+                    for (int i = 0; i < DPR; ++i) {
+                        const int piece = lane + 32 * i;
+                        if (piece * 8 < d) {
 #pragma unroll
-                                    for (int r = 0; r < RG; ++r) {
-                                        const uint4 raw =
-                                            lds128(stage_addr + ((rg + r) * d + piece * 8) * 2);
-                                        const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
+                            for (int r = 0; r < RG; ++r) {
+                                const uint4 raw = lds128(stage_addr + ((rg + r) * d + piece * 8) * 2);
+                                const uint32_t words[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-                                        for (int e = 0; e < 4; ++e) {
-                                            const float2 x = h2_to_f2(words[e]);
+                                for (int e = 0; e < 4; ++e) {
+                                    const float2 x = h2_to_f2(words[e]);
 #pragma unroll
-                                            for (int jq = 0; jq < SQR; ++jq) {
-                                                if (L2) {
-                                                    const float2 df = __fadd2_rn(x, qreg[jq][i][e]);
-                                                    acc2[r][jq] = __ffma2_rn(df, df, acc2[r][jq]);
-                                                } else {
-                                                    acc2[r][jq] =
-                                                        __ffma2_rn(x, qreg[jq][i][e], acc2[r][jq]);
-                                                }
-                                            }
+                                    for (int jq = 0; jq < SQR; ++jq) {
+                                        if (L2) {
+                                            const float2 df = __fadd2_rn(x, qreg[jq][i][e]);
+                                            acc2[r][jq] = __ffma2_rn(df, df, acc2[r][jq]);
+                                        } else {
+                                            acc2[r][jq] = __ffma2_rn(x, qreg[jq][i][e], acc2[r][jq]);
                                         }
                                     }
                                 }
                             }
-                            float a[V];
-#pragma unroll
-                            for (int r = 0; r < RG; ++r)
-#pragma unroll
-                                for (int jq = 0; jq < SQR; ++jq)
-                                    a[r * SQR + jq] = acc2[r][jq].x + acc2[r][jq].y;
-                            transpose_reduce<V>(a, lane);
-                            if (rg + RG >= kTileRows) {
-                                __syncwarp();
-                                if (lane == 0) mbar_arrive(smem_u32(&hdr->empty[w]));
-                            }
-                            // lanes 2v and 2v+1 hold value v = r * SQ + jq
-                            const int v = lane >> 1;
-                            const int r = v / SQR, jq = v % SQR;
-                            const long long row = row0 + rg + r;
-                            const float val = L2 ? (0.0f - a[0]) : a[0];
-                            if ((lane & 1) == 0 && row < p.N && jq < p.s) {
-                                if (TOP1) {
-                                    const uint64_t key = make_key(val, static_cast<uint32_t>(row));
-                                    best0 = key > best0 ? key : best0;
-                                } else if (val >= hdr->thr[jq]) {
-                                    push_candidate(hdr, cand, p.cap, jq,
-                                                   make_key(val, static_cast<uint32_t>(row)));
-                                }
-                            }
                         }
                     }
-                }
-            }
-            if (!TOP1) {
-                // lock-step round: nobody pushes between this barrier and the decision
-                named_barrier(1, cthreads);
-                for (int q = 0; q < p.s; ++q) {
-                    if (hdr->cnt[q] > p.cap - W * kTileRows)
-                        compact_query(hdr, cand, p.cap, q, p.k, ctid, cthreads);
+                    if (rg + RG >= T) {
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(empty_bar);
+                    }
+                    float a[V];
+#pragma unroll
+                    for (int r = 0; r < RG; ++r)
+#pragma unroll
+                        for (int jq = 0; jq < SQR; ++jq) a[r * SQR + jq] = acc2[r][jq].x + acc2[r][jq].y;
+                    transpose_reduce<V>(a, lane);
+                    // lanes 2v and 2v+1 hold value v = r * SQ + jq
+                    const int v = lane >> 1;
+                    const int r = v / SQR, jq = v % SQR;
+                    const long long row = row0 + rg + r;
+                    const float val = L2 ? (0.0f - a[0]) : a[0];
+                    if ((lane & 1) == 0 && row < p.N && jq < p.s) {
+                        if (TOP1) {
+                            const uint64_t key = make_key(val, static_cast<uint32_t>(row));
+                            best0 = key > best0 ? key : best0;
+                        } else if (val >= hdr->thr[jq]) {
+                            push_candidate(hdr, cand, p.cap, p.soft_limit, jq,
+                                           make_key(val, static_cast<uint32_t>(row)));
+                        }
+                    }
                 }
             }
         }
@@ -403,9 +483,31 @@ __global__ void __launch_bounds__(kScanThreads, 1) scan_kernel(const ScanParams 
                 p.partial[static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + ctid] =
                     hdr->best[ctid];
         } else {
+            // this warp is out of tiles; keep answering compaction calls until every warp is
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence_block();
+                atomicAdd(&hdr->done, 1);
+            }
+            for (;;) {
+                int state = 0;  // 1: compaction requested, 2: everybody finished
+                if (lane == 0) {
+                    if (*compact_flag) {
+                        state = 1;
+                    } else if (*done_count >= W) {
+                        // the flag is raised before `done` is incremented: look again
+                        __threadfence_block();
+                        state = *compact_flag ? 1 : 2;
+                    }
+                }
+                state = __shfl_sync(0xffffffffu, state, 0);
+                if (state == 1) compaction_meeting(hdr, cand, p.cap, p.s, p.k, w, lane, W);
+                else if (state == 2) break;
+            }
+            named_barrier(1, cthreads);
+            compact_all(hdr, cand, p.cap, p.s, p.k, 0, w, lane, W);
             named_barrier(1, cthreads);
             for (int q = 0; q < p.s; ++q) {
-                compact_query(hdr, cand, p.cap, q, p.k, ctid, cthreads);
                 const int n = hdr->cnt[q];
                 uint64_t *dst =
                     p.partial + (static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
