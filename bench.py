@@ -53,6 +53,7 @@ def parse_args():
     ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--variant", type=int, default=0)
     ap.add_argument("--rows", type=int, default=None, help="override the corpus size (profiling)")
+    ap.add_argument("--tune", default=None, help="consumer_warps,ring_depth,tile_rows (0 = default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -230,6 +231,8 @@ def main():
     idx = ralm.Index(corpus, metric_id, max_s=max(s, 1), max_k=max(k, 1))
     if args.variant:
         idx.set_variant(args.variant)
+    if args.tune:
+        idx.set_tuning(*[int(v) for v in args.tune.split(",")])
     stream = torch.cuda.current_stream()
 
     ids = torch.empty((s, k), dtype=torch.int64, device=device)
@@ -323,7 +326,7 @@ def main():
             "dtype": "f16 inputs, f32 accumulate", "data": "synthetic",
             "config": {"workload": "%s %dx%d %s s=%d k=%d; cache lookup R=%d C=%d q=%d; verify stride %d"
                                    % (cfg.name, N, d, cfg.metric, s, k, R, cache.shape[1], stride, vstride),
-                       "variant": args.variant, "replicas": world,
+                       "variant": args.variant, "tune": args.tune, "replicas": world,
                        "l2": "inputs larger than L2 (%.1f GB corpus streamed every step)"
                              % (corpus_bytes / 1e9) if corpus_bytes > 2.5e8 else
                              "corpus near L2 size: L2-warm figure, not an HBM number"},

@@ -170,6 +170,13 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
  * UNSUPPORTED if the variant cannot serve the index's metric or dimension. */
 ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant);
 
+/* Override the scan kernel's launch shape on this index (benchmarking aid; 0 keeps the
+ * library's choice): consumer warps per CTA (1..8), shared-memory stages per consumer warp,
+ * rows per tile of the FMA scan (rounded down to its group size; the warp-MMA scan always
+ * uses 16). Values that do not fit in shared memory are reduced. Results do not depend on it. */
+ralm_status_t ralm_index_set_tuning(ralm_index_t *idx, int32_t consumer_warps, int32_t ring_depth,
+                                    int32_t tile_rows);
+
 /* Number of kernels the library launched on behalf of this index since creation. */
 int64_t ralm_index_launch_count(const ralm_index_t *idx);
 

@@ -54,6 +54,8 @@ def load_library() -> ctypes.CDLL:
     lib.ralm_device_status.argtypes = [p, p]
     lib.ralm_index_set_variant.restype = i32
     lib.ralm_index_set_variant.argtypes = [p, i32]
+    lib.ralm_index_set_tuning.restype = i32
+    lib.ralm_index_set_tuning.argtypes = [p, i32, i32, i32]
     lib.ralm_index_launch_count.restype = i64
     lib.ralm_index_launch_count.argtypes = [p]
     lib.ralm_index_set_timing.restype = i32
@@ -117,6 +119,10 @@ class Index:
 
     def set_variant(self, variant: int):
         _check(self._lib.ralm_index_set_variant(self._handle, variant), "ralm_index_set_variant")
+
+    def set_tuning(self, consumer_warps: int = 0, ring_depth: int = 0, tile_rows: int = 0):
+        _check(self._lib.ralm_index_set_tuning(self._handle, consumer_warps, ring_depth, tile_rows),
+               "ralm_index_set_tuning")
 
     def launch_count(self) -> int:
         return self._lib.ralm_index_launch_count(self._handle)

@@ -25,6 +25,7 @@ struct ralm_index {
     int num_sms;
     int smem_optin;
     int variant;  // 0 auto, 1 FMA, 2 warp-MMA, 3 tcgen05
+    int tune_warps, tune_depth, tune_rows;  // 0 = library default
     uint64_t *partial;   // [num_sms][max_s][max_k]
     uint64_t *cache_keys;  // [RALM_MAX_CACHE_KEYS]
     int *status;
@@ -53,6 +54,11 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
     // arithmetic, so it wants many small tiles: several being scored while more are in flight.
     pl->nwarps = mma ? kMaxConsumerWarps : kMaxConsumerWarps - 1;
     pl->tile_rows = mma ? 16 : (s_pass == 1 ? 16 : 4);
+    if (idx->tune_warps > 0) pl->nwarps = std::min(idx->tune_warps, pl->nwarps);
+    if (idx->tune_rows > 0 && !mma) {
+        const int unit = s_pass == 1 ? 16 : 4;  // rows per reduction group of the FMA flavour
+        pl->tile_rows = std::max(unit, idx->tune_rows / unit * unit);
+    }
     pl->stage_bytes = align_up(pl->tile_rows * idx->d * 2, 128);
     pl->off_q = kScanHeaderBytes;
     int off = pl->off_q + (mma ? align_up(kScanMaxQueries * (idx->d * 2 + kQueryPadBytes), 128) : 0);
@@ -71,7 +77,7 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
     if (fit < 2) return false;
     // every consumer warp owns `depth` stages; fewer warps when the stages are large
     pl->nwarps = std::min(pl->nwarps, fit);
-    pl->depth = std::min(fit / pl->nwarps, 3);
+    pl->depth = std::min(fit / pl->nwarps, idx->tune_depth > 0 ? idx->tune_depth : 3);
     pl->smem_bytes = pl->off_stage + pl->nwarps * pl->depth * pl->stage_bytes;
     return true;
 }
@@ -268,6 +274,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->num_sms = prop.multiProcessorCount;
     idx->smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
     idx->variant = 0;
+    idx->tune_warps = idx->tune_depth = idx->tune_rows = 0;
     idx->launches = 0;
     idx->timing = false;
     const size_t partial_bytes = sizeof(uint64_t) * idx->num_sms * max_s * static_cast<size_t>(max_k);
@@ -426,6 +433,7 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.num_sms = std::min(dev->num_sms, RALM_STATIC_MAX_BLOCKS);
     view.smem_optin = dev->smem_optin;
     view.variant = 0;
+    view.tune_warps = view.tune_depth = view.tune_rows = 0;
     view.partial = dev->partial;
     view.cache_keys = nullptr;
     view.status = status;
@@ -436,6 +444,17 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.timing = false;
     if (view.metric == RALM_L2 && d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
     return search_device(&view, static_cast<const __half *>(queries), s, k, ids, scores, st);
+}
+
+ralm_status_t ralm_index_set_tuning(ralm_index_t *idx, int32_t consumer_warps, int32_t ring_depth,
+                                    int32_t tile_rows) {
+    if (!idx || consumer_warps < 0 || consumer_warps > kMaxConsumerWarps || ring_depth < 0 ||
+        ring_depth > kMaxStages || tile_rows < 0 || tile_rows > 64)
+        return RALM_ERR_INVALID_ARG;
+    idx->tune_warps = consumer_warps;
+    idx->tune_depth = ring_depth;
+    idx->tune_rows = tile_rows;
+    return RALM_OK;
 }
 
 int64_t ralm_index_launch_count(const ralm_index_t *idx) { return idx ? idx->launches : 0; }

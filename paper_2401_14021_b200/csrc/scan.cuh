@@ -230,26 +230,36 @@ scan_kernel(const ScanParams p) {
         if (lane == 0) {
             long long issued = 0;
             bool ok = true;
+            // tile `it` belongs to consumer warp cw = it % W; it is that warp's (it / W)-th
+            // tile and goes to slot (it / W) % depth of the warp's private ring, for the
+            // use-th time. The counters advance incrementally: no division on this path.
+            int cw = 0, slot = 0;
+            uint32_t use = 0;
+            long long row0 = static_cast<long long>(blockIdx.x) * T;
+            const long long row_step = static_cast<long long>(gridDim.x) * T;
+            const uint32_t stage_base = smem_u32(smem + p.off_stage);
             for (long long it = 0; it < my_tiles; ++it) {
-                // tile `it` belongs to consumer warp it % W; it is that warp's (it / W)-th
-                // tile and goes to the warp's private ring of `depth` stages
-                const long long local = it / W;
-                const int st = static_cast<int>(it % W) + static_cast<int>(local % p.depth) * W;
-                const long long use = local / p.depth;
+                const int st = cw + slot * W;
                 if (use > 0) {
                     ok = mbar_wait_bounded(smem_u32(&hdr->empty[st]), (use - 1) & 1);
                     if (!ok) break;
                 }
                 if (*abort_flag) break;
-                const long long tile = blockIdx.x + it * static_cast<long long>(gridDim.x);
-                const long long row0 = tile * T;
                 const long long rows = (p.N - row0 < T) ? (p.N - row0) : T;
-                const uint32_t bytes = static_cast<uint32_t>(rows * d * 2);
+                const uint32_t bytes = static_cast<uint32_t>(rows) * static_cast<uint32_t>(d * 2);
                 const uint32_t bar = smem_u32(&hdr->full[st]);
                 mbar_arrive_expect_tx(bar, bytes);
-                bulk_load(smem_u32(smem + p.off_stage + static_cast<size_t>(st) * p.stage_bytes),
-                          p.corpus + row0 * d, bytes, bar);
+                bulk_load(stage_base + static_cast<uint32_t>(st) * p.stage_bytes, p.corpus + row0 * d,
+                          bytes, bar);
                 issued = it + 1;
+                row0 += row_step;
+                if (++cw == W) {
+                    cw = 0;
+                    if (++slot == p.depth) {
+                        slot = 0;
+                        ++use;
+                    }
+                }
             }
             if (!ok) {
                 atomicMax(p.status, kStatusTimeout);
@@ -300,14 +310,21 @@ scan_kernel(const ScanParams p) {
                 }
         }
 
-        for (long long it = w; it < my_tiles; it += W) {
+        int slot = 0;         // position in this warp's private ring
+        uint32_t parity = 0;  // phase parity of the ring's current lap
+        long long row0 = (static_cast<long long>(blockIdx.x) + static_cast<long long>(w) * gridDim.x) * T;
+        const long long row_step = static_cast<long long>(gridDim.x) * W * T;
+        for (long long it = w; it < my_tiles; it += W, row0 += row_step) {
             if (*abort_flag) continue;
             // this warp's private ring: only this warp ever waits on these stages, in order,
             // so a parity wait can never be satisfied by an older phase
-            const long long local = it / W;
-            const int st = w + static_cast<int>(local % p.depth) * W;
+            const int st = w + slot * W;
             const uint32_t full_bar = smem_u32(&hdr->full[st]);
-            const uint32_t parity = (local / p.depth) & 1;
+            const uint32_t my_parity = parity;
+            if (++slot == p.depth) {
+                slot = 0;
+                parity ^= 1;
+            }
             // Wait for the tile. Lane 0 polls; a raised compaction flag takes priority over a
             // ready tile (after the flag is up a warp finishes at most the tile it is on), and
             // a warp still waiting for its tile joins the meeting instead of blocking it.
@@ -319,12 +336,12 @@ scan_kernel(const ScanParams p) {
                     int state = 0;  // 1 tile ready, 2 compaction requested, 3 gave up
                     if (lane == 0) {
                         if (!TOP1 && *compact_flag) state = 2;
-                        else if (mbar_try_wait(full_bar, parity)) state = 1;
+                        else if (mbar_try_wait(full_bar, my_parity)) state = 1;
                         else if ((++spins & 1023) == 0 && clock64() - t0 > kWaitCycleLimit) state = 3;
                     }
                     state = __shfl_sync(0xffffffffu, state, 0);
                     if (state == 1) {
-                        while (!mbar_try_wait(full_bar, parity)) {}  // completed: returns at once
+                        while (!mbar_try_wait(full_bar, my_parity)) {}  // completed: returns at once
                         have_tile = true;
                     } else if (state == 2) {
                         compaction_meeting(hdr, cand, p.cap, p.s, p.k, w, lane, W);
@@ -341,8 +358,6 @@ scan_kernel(const ScanParams p) {
             const uint32_t stage_addr =
                 smem_u32(smem + p.off_stage + static_cast<size_t>(st) * p.stage_bytes);
             const uint32_t empty_bar = smem_u32(&hdr->empty[st]);
-            const long long tile = blockIdx.x + it * static_cast<long long>(gridDim.x);
-            const long long row0 = tile * T;
             if (MMA) {
                 // ---- 16 rows x 8 queries on tensor cores; two accumulator sets halve the
                 // dependent chain
