@@ -8,7 +8,7 @@ One step = one verification step of the serving loop, all kernels on one stream:
 Throughput is verified queries per second = s * steps / time. Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-                  [--workload C1|C2|C3|C4] [--s S] [--k K] [--variant V] [--rows N]
+                  [--workload C1|C2|C3|C4|C5] [--s S] [--k K] [--variant V] [--rows N]
 
 With --gpus N > 1 (launched under torch.distributed.run) every rank runs an independent
 replica on its own GPU (the path does not shard); the value is the sum over replicas and the
@@ -48,7 +48,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="C3", choices=["C1", "C2", "C3", "C4"])
+    ap.add_argument("--workload", default="C3", choices=["C1", "C2", "C3", "C4", "C5"])
     ap.add_argument("--s", type=int, default=None)
     ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--variant", type=int, default=0)
@@ -239,13 +239,17 @@ def main():
     scores = torch.empty((s, k), dtype=torch.float32, device=device)
     spec_ids = torch.empty((R, stride, 1), dtype=torch.int64, device=device)
     spec_scores = torch.empty((R, stride, 1), dtype=torch.float32, device=device)
-    first_mismatch = torch.empty((1,), dtype=torch.int32, device=device)
+    # the batch holds the strides of the first `nv` requests (one request at s <= stride)
     vstride = min(stride, s)
+    nv = max(1, min(R, s // stride))
+    first_mismatch = torch.empty((nv,), dtype=torch.int32, device=device)
+    spec_view = spec_ids[:nv, :vstride, 0] if vstride < stride else spec_ids[:nv].reshape(nv, stride)
+    retr_view = ids[:nv * vstride].reshape(nv, vstride, k)
 
     def step():
         ralm.cache_search(idx, cache, cache_q, 1, spec_ids, spec_scores, stream)
         ralm.search(idx, queries, k, ids, scores, stream)
-        ralm.verify(spec_ids[0:1, :vstride, 0], ids[:vstride].unsqueeze(0), 1, first_mismatch, stream)
+        ralm.verify(spec_view, retr_view, 1, first_mismatch, stream)
 
     # ---- device-resident timing
     for _ in range(max(args.warmup, 3)):
@@ -278,19 +282,20 @@ def main():
     h_ids = torch.empty((s, k), dtype=torch.int64).pin_memory()
     h_scores = torch.empty((s, k), dtype=torch.float32).pin_memory()
     h_spec = torch.empty((R, stride, 1), dtype=torch.int64).pin_memory()
-    h_fm = torch.empty((1,), dtype=torch.int32).pin_memory()
+    h_fm = torch.empty((nv,), dtype=torch.int32).pin_memory()
     d_cache, d_cache_q = torch.empty_like(cache), torch.empty_like(cache_q)
-    retr1 = torch.empty((1, vstride, 1), dtype=torch.int64, device=device)
-    h2d = h_q.numel() * 2 + h_cache.numel() * 8 + h_cache_q.numel() * 2 + h_ids[:vstride, :1].numel() * 8
-    d2h = h_ids.numel() * 8 + h_scores.numel() * 4 + h_spec.numel() * 8 + 4
+    retr1 = torch.empty((nv, vstride, 1), dtype=torch.int64, device=device)
+    h_top1 = h_ids[:nv * vstride, :1].reshape(nv, vstride, 1)
+    h2d = h_q.numel() * 2 + h_cache.numel() * 8 + h_cache_q.numel() * 2 + h_top1.numel() * 8
+    d2h = h_ids.numel() * 8 + h_scores.numel() * 4 + h_spec.numel() * 8 + 4 * nv
 
     def step_e2e():
         d_cache.copy_(h_cache, non_blocking=True)
         d_cache_q.copy_(h_cache_q, non_blocking=True)
         ralm.cache_search(idx, d_cache, d_cache_q, 1, spec_ids, spec_scores, stream)
         ralm.search_host(idx, h_q, k, h_ids, h_scores, stream)          # H2D, scan, D2H, sync
-        retr1.copy_(h_ids[:vstride, :1].unsqueeze(0), non_blocking=True)
-        ralm.verify(spec_ids[0:1, :vstride, 0], retr1, 1, first_mismatch, stream)
+        retr1.copy_(h_top1, non_blocking=True)
+        ralm.verify(spec_view, retr1, 1, first_mismatch, stream)
         h_spec.copy_(spec_ids, non_blocking=True)
         h_fm.copy_(first_mismatch, non_blocking=True)
         stream.synchronize()
@@ -306,19 +311,39 @@ def main():
     e2e_ms = e0.elapsed_time(e1)
 
     # ---- aggregate over ranks: time = max, work = sum
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = t.tolist()
+    from paper_2401_14021_b200 import replicas
+    (total_ms, e2e_ms), job_queries = replicas.aggregate([total_ms, e2e_ms], s * args.steps, device)
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        value = world * s * args.steps / (total_ms * 1e-3)
-        e2e_value = world * s * args.steps / (e2e_ms * 1e-3)
+        value = job_queries / (total_ms * 1e-3)
+        e2e_value = job_queries / (e2e_ms * 1e-3)
         corpus_bytes = N * d * 2
         passes = scan_launches / max(args.steps, 1)
         scan_avg_ms = scan_ms / max(scan_launches, 1)
         achieved = corpus_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"] if achieved else None,
+                    "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / 8000.0 if achieved else None,
+                    "kernel": "scan_kernel", "bytes_per_launch": corpus_bytes,
+                    "traffic": (corpus_bytes * TRAFFIC_RATIO["scan_kernel<mma,ip>"]
+                                if cfg.metric == "ip" and args.variant in (0, 2) and not args.tune
+                                and s <= 8 else None),
+                    "traffic_note": "2M-row ncu capture scaled by rows; null if the kernel changed since"}
+        uses_tc = cfg.metric == "ip" and k <= 64 and d >= 64 and (args.variant == 3 or (args.variant == 0 and s >= 9))
+        if uses_tc:
+            roofline["kernel"] = "scan_tc_kernel"
+        if uses_tc and s > 255:
+            # large batch: s flop per corpus byte is beyond the ridge, the tensor pipe bounds it.
+            # fp16 runs at the bf16 rate; the kernel is timed inside a long step: sustained peak
+            flops = 2.0 * s * N * d / passes if passes else 0.0
+            tf = flops / (scan_avg_ms * 1e-3) / 1e12 if scan_launches else None
+            peak_tf = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+            roofline = {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
+                        "frac": tf / peak_tf if tf else None, "peak_kind": peak_kind + " (bf16 sustained)",
+                        "frac_of_burst": tf / peaks["bf16_tflops"] if tf else None,
+                        "kernel": "scan_tc_kernel", "flops_per_launch": flops, "traffic": None,
+                        "hbm_gbs": achieved}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
@@ -331,13 +356,7 @@ def main():
                              % (corpus_bytes / 1e9) if corpus_bytes > 2.5e8 else
                              "corpus near L2 size: L2-warm figure, not an HBM number"},
             "scan_gbs": achieved, "scan_ms": scan_avg_ms, "scan_passes_per_step": passes,
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": achieved / peaks["hbm_gbs"] if achieved else None,
-                         "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / 8000.0 if achieved else None,
-                         "kernel": "scan_kernel", "bytes_per_launch": corpus_bytes,
-                         "traffic": (corpus_bytes * TRAFFIC_RATIO["scan_kernel<mma,ip>"]
-                                     if cfg.metric == "ip" and args.variant in (0, 2) and not args.tune else None),
-                         "traffic_note": "2M-row ncu capture scaled by rows; null if the kernel changed since"},
+            "roofline": roofline,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
             "gpu_launches": int(gpu_launches),

@@ -118,7 +118,7 @@ ralm_status_t ralm_search_host(ralm_index_t *idx, const void *queries_host, int3
  *   ids, scores            DEVICE int64 [s][k] / fp32 [s][k] (written), 1 <= k <= RALM_STATIC_MAX_K
  *   device_status          DEVICE int32, may be NULL: zeroed by the call, then set to a
  *                          ralm_status_t value if a device-side wait ran out
- * Results are identical to ralm_search's. L2 needs d <= 1024 (as ralm_search does).
+ * Results are identical to ralm_search's.
  * Errors: RALM_ERR_STATIC_LIMIT when s or k exceeds the limits above (nothing is launched);
  * INVALID_ARG, UNSUPPORTED, CUDA as elsewhere.
  *
@@ -165,8 +165,9 @@ ralm_status_t ralm_verify(const int64_t *speculated_ids, const int64_t *retrieve
 ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
 
 /* Pin the scan variant used by ralm_search on this index (benchmarking aid).
- *   0 = automatic, 1 = FMA scan (fp32 FMAs, any metric), 2 = warp-MMA scan (inner product,
- *   up to 8 queries per pass), 3 = tcgen05 scan (inner product, large batches).
+ *   0 = automatic, 1 = FMA scan (fp32 FMAs, d <= 1024, 4 queries per pass), 2 = warp-MMA scan
+ *   (8 queries per pass; for L2 the tensor-core value only filters and the ranked distance is
+ *   the direct sum of squared differences), 3 = tcgen05 scan (inner product, large batches).
  * UNSUPPORTED if the variant cannot serve the index's metric or dimension. */
 ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant);
 

@@ -188,6 +188,34 @@ cache_rank_kernel(const uint64_t *__restrict__ keys, int Cp, int k, int l2,
 }
 
 // ------------------------------------------------------------------------------------
+// Squared norms of the corpus rows (L2 indexes, once at creation): one warp per row, fp32.
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+row_norm_kernel(const __half *__restrict__ corpus, long long N, int d, float *__restrict__ norms) {
+    const int lane = threadIdx.x & 31;
+    const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
+    for (long long row = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); row < N;
+         row += warps) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(corpus + row * d);
+        float2 sum = make_float2(0.f, 0.f);
+        for (int piece = lane; piece * 8 < d; piece += 32) {
+            const uint4 raw = __ldg(src + piece);
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 x = __half22float2(*reinterpret_cast<const __half2 *>(&w[e]));
+                sum.x = fmaf(x.x, x.x, sum.x);
+                sum.y = fmaf(x.y, x.y, sum.y);
+            }
+        }
+        float v = sum.x + sum.y;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) norms[row] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------
 // Verification: one warp per request; lanes take speculation steps 32 at a time.
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128)

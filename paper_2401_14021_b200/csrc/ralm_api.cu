@@ -12,6 +12,7 @@
 
 #include "aux_kernels.cuh"
 #include "scan.cuh"
+#include "scan_tc.cuh"
 
 using namespace ralm;
 
@@ -28,6 +29,9 @@ struct ralm_index {
     int tune_warps, tune_depth, tune_rows;  // 0 = library default
     uint64_t *partial;   // [num_sms][max_s][max_k]
     uint64_t *cache_keys;  // [RALM_MAX_CACHE_KEYS]
+    float *norms;          // L2: squared norm of every corpus row (fp32 [N]), or null
+    uint64_t *tc_cand;     // tcgen05 scan: [num_sms][tc_cand_q][kTcCap] candidate lists, or null
+    int tc_cand_q;
     int *status;
     // staging for the host-buffer entry point
     __half *h_queries;
@@ -82,9 +86,9 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
     return true;
 }
 
-template <bool MMA, bool L2, int SQ, int DP, bool TOP1>
+template <bool MMA, bool L2, int SQ, int DP, bool TOP1, bool NRM = false>
 cudaError_t launch_scan(const ScanParams &p, int grid, int smem, cudaStream_t st) {
-    auto kern = scan_kernel<MMA, L2, SQ, DP, TOP1>;
+    auto kern = scan_kernel<MMA, L2, SQ, DP, TOP1, NRM>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     kern<<<grid, 32 * (p.nwarps + 1), smem, st>>>(p);
@@ -111,15 +115,133 @@ cudaError_t launch_fma(const ScanParams &p, int grid, int smem, cudaStream_t st)
 constexpr int kFmaMaxD = 1024;
 constexpr int kFmaQueriesPerPass = 4;
 
-// Which scan serves this index: 1 = FMA, 2 = warp-MMA.
+// Which scan serves a small batch on this index: 1 = FMA, 2 = warp-MMA (the default).
 int resolve_variant(const ralm_index *idx) {
     if (idx->variant == 1 || idx->variant == 2) return idx->variant;
-    return idx->metric == RALM_IP ? 2 : 1;
+    return 2;
 }
+
+
+// ---- tcgen05 scan (large batches, inner product) -------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The tensor-map encoder lives in the driver; it is looked up once through the runtime so that
+// the library does not link against the driver library.
+EncodeTiledFn tensor_map_encoder() {
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult res;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &res) != cudaSuccess ||
+            res != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(sym);
+    }();
+    return fn;
+}
+
+// fp16 [rows][d] row-major, tiles of box_rows x 64 elements, 128-byte swizzle, zero fill
+// outside the tensor.
+bool encode_rows_map(CUtensorMap *map, const void *base, long long rows, int d, int box_rows) {
+    EncodeTiledFn enc = tensor_map_encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(d) * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kTcChunkK), static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tc_can_serve(const ralm_index *idx, int k) {
+    return idx->metric == RALM_IP && idx->tc_cand != nullptr && k <= kTcMaxK && idx->d >= kTcChunkK;
+}
+
+bool alloc_tc_workspace(ralm_index *idx, int queries) {
+    if (idx->tc_cand && idx->tc_cand_q >= queries) return true;
+    if (idx->tc_cand) cudaFree(idx->tc_cand);
+    idx->tc_cand = nullptr;
+    idx->tc_cand_q = 0;
+    const size_t bytes = sizeof(uint64_t) * idx->num_sms * static_cast<size_t>(queries) * kTcCap;
+    if (cudaMalloc(&idx->tc_cand, bytes) != cudaSuccess) {
+        idx->tc_cand = nullptr;
+        return false;
+    }
+    idx->tc_cand_q = queries;
+    return true;
+}
+
+// One pass of up to min(512, workspace) queries.
+ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int s_total, int q0, int k,
+                             int grid, cudaStream_t st) {
+    TcParams p;
+    p.partial = idx->partial;
+    p.cand = idx->tc_cand;
+    p.cand_q = idx->tc_cand_q;
+    p.status = idx->status;
+    p.N = idx->N;
+    p.ntiles = (idx->N + kTcTileM - 1) / kTcTileM;
+    p.nchunks = (idx->d + kTcChunkK - 1) / kTcChunkK;
+    p.s = sp;
+    p.s_total = s_total;
+    p.q_base = q0;
+    p.k = k;
+    p.nb = sp > kTcMaxN ? kTcMaxN : align_up(sp, 16);
+    p.nhalves = (sp + p.nb - 1) / p.nb;
+    p.stage_bytes = kTcABytes + p.nb * 128;
+    p.off_stage = align_up(kTcOffEnd, 1024);
+    p.stages = std::min(kTcMaxStages, (idx->smem_optin - p.off_stage) / p.stage_bytes);
+    if (p.stages < 2) return RALM_ERR_UNSUPPORTED;
+    const int smem = p.off_stage + p.stages * p.stage_bytes;
+    CUtensorMap map_x, map_q;
+    if (!encode_rows_map(&map_x, idx->corpus, idx->N, idx->d, kTcTileM) ||
+        !encode_rows_map(&map_q, queries, sp, idx->d, p.nb))
+        return RALM_ERR_CUDA;
+    if (cudaFuncSetAttribute(scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return RALM_ERR_CUDA;
+    scan_tc_kernel<<<grid, kTcThreads, smem, st>>>(map_x, map_q, p);
+    return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
+}
+
+constexpr int kTcAutoMinQueries = 9;  // batches the 8-query scan cannot serve in one pass
 
 ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k, int64_t *ids,
                             float *scores, cudaStream_t st) {
     if (s == 0) return RALM_OK;
+    const bool tc = tc_can_serve(idx, k) && (idx->variant == 3 || (idx->variant == 0 && s >= kTcAutoMinQueries));
+    if (tc) {
+        const int grid = static_cast<int>(std::min<long long>(idx->num_sms, (idx->N + kTcTileM - 1) / kTcTileM));
+        const int per_pass = std::min(kTcMaxQueries, idx->tc_cand_q);
+        for (int q0 = 0; grid > 0 && q0 < s; q0 += per_pass) {
+            const int sp = std::min(per_pass, s - q0);
+            std::pair<cudaEvent_t, cudaEvent_t> ev{nullptr, nullptr};
+            if (idx->timing) {
+                if (!idx->spare.empty()) {
+                    ev = idx->spare.back();
+                    idx->spare.pop_back();
+                } else if (cudaEventCreate(&ev.first) != cudaSuccess ||
+                           cudaEventCreate(&ev.second) != cudaSuccess) {
+                    return RALM_ERR_CUDA;
+                }
+                cudaEventRecord(ev.first, st);
+            }
+            const ralm_status_t rs =
+                launch_tc_pass(idx, queries + static_cast<size_t>(q0) * idx->d, sp, s, q0, k, grid, st);
+            if (idx->timing) {
+                cudaEventRecord(ev.second, st);
+                idx->timed.push_back(ev);
+            }
+            if (rs != RALM_OK) return rs;
+            idx->launches++;
+        }
+        merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, 0, ids, scores);
+        if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
+        idx->launches++;
+        return RALM_OK;
+    }
     const int variant = resolve_variant(idx);
     const bool mma = variant == 2;
     if (!mma && idx->d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
@@ -133,6 +255,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             ScanParams p;
             p.corpus = idx->corpus;
             p.queries = queries + static_cast<size_t>(q0) * idx->d;
+            p.norms = idx->norms;
             p.partial = idx->partial;
             p.status = idx->status;
             p.N = idx->N;
@@ -151,6 +274,10 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             p.off_q = pl.off_q;
             p.off_cand = pl.off_cand;
             p.off_stage = pl.off_stage;
+            // bound on the rounding error of the tensor-core |x|^2 - 2 x.q + |q|^2 relative to
+            // |x|^2 + |q|^2: d accumulation steps of at most 2^-22 each, on terms that sum to
+            // at most twice that scale
+            p.l2_slack = static_cast<float>(idx->d) * (1.0f / 2097152.0f);
             cudaError_t e;
             std::pair<cudaEvent_t, cudaEvent_t> ev{nullptr, nullptr};
             if (idx->timing) {
@@ -163,7 +290,13 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
                 }
                 cudaEventRecord(ev.first, st);
             }
-            if (mma) {
+            if (mma && idx->metric == RALM_L2 && idx->norms) {
+                e = (k == 1) ? launch_scan<true, true, 8, 1, true, true>(p, grid, pl.smem_bytes, st)
+                             : launch_scan<true, true, 8, 1, false, true>(p, grid, pl.smem_bytes, st);
+            } else if (mma && idx->metric == RALM_L2) {
+                e = (k == 1) ? launch_scan<true, true, 8, 1, true>(p, grid, pl.smem_bytes, st)
+                             : launch_scan<true, true, 8, 1, false>(p, grid, pl.smem_bytes, st);
+            } else if (mma) {
                 e = (k == 1) ? launch_scan<true, false, 8, 1, true>(p, grid, pl.smem_bytes, st)
                              : launch_scan<true, false, 8, 1, false>(p, grid, pl.smem_bytes, st);
             } else if (idx->metric == RALM_L2) {
@@ -279,7 +412,13 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->timing = false;
     const size_t partial_bytes = sizeof(uint64_t) * idx->num_sms * max_s * static_cast<size_t>(max_k);
     const size_t sk = static_cast<size_t>(max_s) * max_k;
+    idx->tc_cand = nullptr;
+    idx->tc_cand_q = 0;
+    idx->norms = nullptr;
     bool ok = cudaMalloc(&idx->partial, partial_bytes) == cudaSuccess;
+    if (metric == RALM_L2 && N > 0) ok = ok && cudaMalloc(&idx->norms, sizeof(float) * N) == cudaSuccess;
+    if (metric == RALM_IP && max_s >= kTcAutoMinQueries && d >= kTcChunkK)
+        ok = ok && alloc_tc_workspace(idx, std::min(kTcMaxQueries, align_up(max_s, 16)));
     ok = ok && cudaMalloc(&idx->cache_keys, sizeof(uint64_t) * RALM_MAX_CACHE_KEYS) == cudaSuccess;
     ok = ok && cudaMalloc(&idx->status, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMalloc(&idx->h_queries, static_cast<size_t>(max_s) * d * 2) == cudaSuccess;
@@ -294,6 +433,15 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
         ralm_index_destroy(idx);
         return RALM_ERR_CUDA;
     }
+    if (idx->norms) {
+        // one pass over the corpus; the filter of the L2 scan reads these instead of recomputing
+        const int blocks = static_cast<int>(std::min<long long>((N + 7) / 8, 32LL * idx->num_sms));
+        row_norm_kernel<<<blocks, 256>>>(idx->corpus, N, d, idx->norms);
+        if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+            ralm_index_destroy(idx);
+            return RALM_ERR_CUDA;
+        }
+    }
     *out = idx;
     return RALM_OK;
 }
@@ -302,6 +450,8 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
     if (!idx) return RALM_OK;
     cudaFree(idx->partial);
     cudaFree(idx->cache_keys);
+    cudaFree(idx->tc_cand);
+    cudaFree(idx->norms);
     cudaFree(idx->status);
     cudaFree(idx->h_queries);
     cudaFree(idx->h_ids);
@@ -395,8 +545,10 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream) {
 ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant) {
     if (!idx || variant < 0 || variant > 3) return RALM_ERR_INVALID_ARG;
     if (variant == 1 && idx->d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
-    if (variant == 2 && idx->metric != RALM_IP) return RALM_ERR_UNSUPPORTED;
-    if (variant == 3) return RALM_ERR_UNSUPPORTED;
+    if (variant == 3) {
+        if (idx->metric != RALM_IP || idx->d < kTcChunkK || !tensor_map_encoder()) return RALM_ERR_UNSUPPORTED;
+        if (!alloc_tc_workspace(idx, std::min(kTcMaxQueries, align_up(idx->max_s, 16)))) return RALM_ERR_OOM;
+    }
     idx->variant = variant;
     return RALM_OK;
 }
@@ -436,13 +588,15 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.tune_warps = view.tune_depth = view.tune_rows = 0;
     view.partial = dev->partial;
     view.cache_keys = nullptr;
+    view.tc_cand = nullptr;
+    view.tc_cand_q = 0;
+    view.norms = nullptr;  // no index, no stored norms: the scan derives them on the tensor cores
     view.status = status;
     view.h_queries = nullptr;
     view.h_ids = nullptr;
     view.h_scores = nullptr;
     view.launches = 0;
     view.timing = false;
-    if (view.metric == RALM_L2 && d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
     return search_device(&view, static_cast<const __half *>(queries), s, k, ids, scores, st);
 }
 

@@ -12,9 +12,12 @@
 //     pairs), converts its slice of a row and issues packed fp32 FMAs; per-lane partial
 //     sums are combined with a transposing shuffle reduction. Serves both metrics (L2 in
 //     the direct sum-of-squared-differences form, which has no cancellation).
-//   warp-MMA flavour (inner product): m16n8k16 tensor-core tiles with the 16 corpus rows as
-//     M and the (up to) 8 queries as N, fp32 accumulators. The k index is permuted (the
-//     same way for rows and queries) so that each lane reads 16 contiguous bytes per row.
+//   warp-MMA flavour: m16n8k16 tensor-core tiles with the 16 corpus rows as M and the (up
+//     to) 8 queries as N, fp32 accumulators. The k index is permuted (the same way for rows
+//     and queries) so that each lane reads 16 contiguous bytes per row. For L2 the tensor
+//     cores also give the rows' squared norms (diagonals of rows x rows products) and
+//     |x|^2 - 2 x.q + |q|^2 serves as a conservative filter; every pair that passes is scored
+//     again in the direct form, and only that value is ranked and returned.
 //
 // Selection: k == 1 keeps a running best key per thread. k > 1 uses a per-query threshold
 // (the current k-th best of this CTA) and a shared-memory candidate buffer. A push that lands
@@ -37,6 +40,7 @@ constexpr int kQueryPadBytes = 64;
 struct ScanParams {
     const __half *corpus;
     const __half *queries;  // [s][d] of this pass
+    const float *norms;     // warp-MMA L2 with NRM: squared norm of every corpus row, fp32 [N]
     uint64_t *partial;      // [gridDim.x][s_total][k] sorted keys, 0 = empty
     int *status;
     long long N;
@@ -55,6 +59,7 @@ struct ScanParams {
     int off_q;  // shared-memory offsets (bytes)
     int off_cand;
     int off_stage;
+    float l2_slack;  // warp-MMA L2: filter slack per unit of (|x|^2 + |q|^2)
 };
 
 struct ScanHeader {
@@ -173,12 +178,39 @@ __device__ __forceinline__ void push_candidate(ScanHeader *hdr, uint64_t *cand, 
     if (slot >= soft) *reinterpret_cast<volatile int *>(&hdr->flag) = 1;
 }
 
+
+// Warp-MMA L2 flavour, exact part: squared distance between one corpus row (read back from
+// global memory; the tile it came with has just passed through L2) and one query (fp16 in
+// shared memory), computed by the whole warp in the direct sum-of-squared-differences form
+// (no cancellation). Every lane returns the full sum.
+__device__ __forceinline__ float warp_direct_l2(const __half *row, uint32_t q_addr, int d, int lane) {
+    float2 sum = make_float2(0.f, 0.f);
+    for (int piece = lane; piece * 8 < d; piece += 32) {
+        const uint4 xr = __ldg(reinterpret_cast<const uint4 *>(row) + piece);
+        const uint4 qr = lds128(q_addr + piece * 16);
+        const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
+        const uint32_t qw[4] = {qr.x, qr.y, qr.z, qr.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 x = h2_to_f2(xw[e]), q = h2_to_f2(qw[e]);
+            const float dx = x.x - q.x, dy = x.y - q.y;
+            sum.x = fmaf(dx, dx, sum.x);
+            sum.y = fmaf(dy, dy, sum.y);
+        }
+    }
+    float v = sum.x + sum.y;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
 // ------------------------------------------------------------------------------------
-// The kernel. MMA: warp-MMA flavour (inner product only) or FMA flavour.
-// L2: metric of the FMA flavour. SQ: queries held per lane (1 or 4; FMA flavour).
+// The kernel. MMA: warp-MMA flavour or FMA flavour. L2: metric (the warp-MMA flavour uses
+// the tensor-core value of |x|^2 - 2 x.q + |q|^2 as a filter and ranks the direct form). SQ: queries held per lane (1 or 4; FMA flavour).
 // DP: 16-byte pieces of a row per lane (d <= 256 * DP; FMA flavour). TOP1: k == 1.
+// NRM (warp-MMA L2): the rows' squared norms come from p.norms instead of extra MMAs.
 // ------------------------------------------------------------------------------------
-template <bool MMA, bool L2, int SQ, int DP, bool TOP1>
+template <bool MMA, bool L2, int SQ, int DP, bool TOP1, bool NRM = false>
 __global__ void __launch_bounds__(MMA ? kScanThreads : kScanThreads - 32, 1)
 scan_kernel(const ScanParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -310,6 +342,21 @@ scan_kernel(const ScanParams p) {
                 }
         }
 
+        // warp-MMA flavour: where the queries sit in shared memory; for L2 also the squared
+        // norms of this lane's two queries (2t, 2t+1), summed in fp32
+        const uint32_t q_pitch = static_cast<uint32_t>(d * 2 + kQueryPadBytes);
+        const uint32_t q_base_addr = smem_u32(smem + p.off_q);
+        float qn0 = 0.f, qn1 = 0.f;
+        if (MMA && L2) {
+            const __half *qa = reinterpret_cast<const __half *>(smem + p.off_q + (2 * t) * q_pitch);
+            const __half *qb = reinterpret_cast<const __half *>(smem + p.off_q + (2 * t + 1) * q_pitch);
+            for (int i = 0; i < d; ++i) {
+                const float a = __half2float(qa[i]), b = __half2float(qb[i]);
+                qn0 = fmaf(a, a, qn0);
+                qn1 = fmaf(b, b, qn1);
+            }
+        }
+
         int slot = 0;         // position in this warp's private ring
         uint32_t parity = 0;  // phase parity of the ring's current lap
         long long row0 = (static_cast<long long>(blockIdx.x) + static_cast<long long>(w) * gridDim.x) * T;
@@ -321,6 +368,11 @@ scan_kernel(const ScanParams p) {
             const int st = w + slot * W;
             const uint32_t full_bar = smem_u32(&hdr->full[st]);
             const uint32_t my_parity = parity;
+            float pn_lo = 0.f, pn_hi = 0.f;  // stored norms of rows g and g + 8, in flight during the wait
+            if (MMA && L2 && NRM) {
+                if (row0 + g < p.N) pn_lo = __ldg(p.norms + row0 + g);
+                if (row0 + g + 8 < p.N) pn_hi = __ldg(p.norms + row0 + g + 8);
+            }
             if (++slot == p.depth) {
                 slot = 0;
                 parity ^= 1;
@@ -360,11 +412,14 @@ scan_kernel(const ScanParams p) {
             const uint32_t empty_bar = smem_u32(&hdr->empty[st]);
             if (MMA) {
                 // ---- 16 rows x 8 queries on tensor cores; two accumulator sets halve the
-                // dependent chain
+                // dependent chain. For L2 two more products per step, rows x rows, put the
+                // rows' squared norms on the diagonals of nlo (rows 0..7) and nhi (rows 8..15).
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
                 float acc_b[4] = {0.f, 0.f, 0.f, 0.f};
+                float nlo[4] = {0.f, 0.f, 0.f, 0.f}, nlo_b[4] = {0.f, 0.f, 0.f, 0.f};
+                float nhi[4] = {0.f, 0.f, 0.f, 0.f}, nhi_b[4] = {0.f, 0.f, 0.f, 0.f};
                 const int nchunks = (d + 31) >> 5;
-                const uint32_t q_addr = smem_u32(smem + p.off_q) + g * (d * 2 + kQueryPadBytes);
+                const uint32_t q_addr = q_base_addr + g * q_pitch;
                 const uint32_t a_lo_addr = stage_addr + g * d * 2;
                 const uint32_t a_hi_addr = stage_addr + (g + 8) * d * 2;
 #pragma unroll 4
@@ -380,6 +435,12 @@ scan_kernel(const ScanParams p) {
                     }
                     mma_m16n8k16(acc, lo.x, hi.x, lo.y, hi.y, b.x, b.y);
                     mma_m16n8k16(acc_b, lo.z, hi.z, lo.w, hi.w, b.z, b.w);
+                    if (L2 && !NRM) {
+                        mma_m16n8k16(nlo, lo.x, hi.x, lo.y, hi.y, lo.x, lo.y);
+                        mma_m16n8k16(nhi, lo.x, hi.x, lo.y, hi.y, hi.x, hi.y);
+                        mma_m16n8k16(nlo_b, lo.z, hi.z, lo.w, hi.w, lo.z, lo.w);
+                        mma_m16n8k16(nhi_b, lo.z, hi.z, lo.w, hi.w, hi.z, hi.w);
+                    }
                 }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[i] += acc_b[i];
@@ -389,6 +450,58 @@ scan_kernel(const ScanParams p) {
                 // acc[2]: (row g+8, query 2t)   acc[3]: (row g+8, query 2t+1)
                 const long long r_lo = row0 + g, r_hi = row0 + g + 8;
                 const int q0 = 2 * t, q1 = 2 * t + 1;
+                if (L2) {
+                    // |x|^2 - 2 x.q + |q|^2 from the tensor cores is only a FILTER (it cancels):
+                    // a pair passes when it could still beat the threshold given the slack that
+                    // bounds the filter's rounding error, and is then scored again in the direct
+                    // form, which is the value that is ranked and returned.
+                    float n_lo = pn_lo, n_hi = pn_hi;
+                    if (!NRM) {
+                        // the diagonal entry of row g (and g + 8) is held by the lane with t == g / 2
+                        const float d_lo = (g & 1) ? (nlo[1] + nlo_b[1]) : (nlo[0] + nlo_b[0]);
+                        const float d_hi = (g & 1) ? (nhi[3] + nhi_b[3]) : (nhi[2] + nhi_b[2]);
+                        const int diag_lane = (lane & ~3) | (g >> 1);
+                        n_lo = __shfl_sync(0xffffffffu, d_lo, diag_lane);
+                        n_hi = __shfl_sync(0xffffffffu, d_hi, diag_lane);
+                    }
+                    float th0, th1;
+                    if (TOP1) {
+                        const unsigned long long b0 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[q0]);
+                        const unsigned long long b1 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[q1]);
+                        th0 = b0 ? key_value(b0) : -INFINITY;
+                        th1 = b1 ? key_value(b1) : -INFINITY;
+                    } else {
+                        th0 = *reinterpret_cast<volatile float *>(&hdr->thr[q0]);
+                        th1 = *reinterpret_cast<volatile float *>(&hdr->thr[q1]);
+                    }
+                    const float sl = p.l2_slack;
+                    bool pass[4];
+                    pass[0] = r_lo < p.N && q0 < p.s && (2.f * acc[0] - n_lo - qn0) + sl * (n_lo + qn0) >= th0;
+                    pass[1] = r_lo < p.N && q1 < p.s && (2.f * acc[1] - n_lo - qn1) + sl * (n_lo + qn1) >= th1;
+                    pass[2] = r_hi < p.N && q0 < p.s && (2.f * acc[2] - n_hi - qn0) + sl * (n_hi + qn0) >= th0;
+                    pass[3] = r_hi < p.N && q1 < p.s && (2.f * acc[3] - n_hi - qn1) + sl * (n_hi + qn1) >= th1;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        unsigned m = __ballot_sync(0xffffffffu, pass[i]);
+                        while (m) {
+                            const int src = __ffs(m) - 1;
+                            m &= m - 1;
+                            const int row_local = (src >> 2) + ((i & 2) ? 8 : 0);
+                            const int q = 2 * (src & 3) + (i & 1);
+                            const float dist = warp_direct_l2(p.corpus + (row0 + row_local) * d,
+                                                              q_base_addr + q * q_pitch, d, lane);
+                            if (lane == 0) {
+                                const float val = 0.0f - dist;
+                                const uint64_t key = make_key(val, static_cast<uint32_t>(row0 + row_local));
+                                if (TOP1) {
+                                    atomicMax(&hdr->best[q], static_cast<unsigned long long>(key));
+                                } else if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q])) {
+                                    push_candidate(hdr, cand, p.cap, p.soft_limit, q, key);
+                                }
+                            }
+                        }
+                    }
+                } else {
                 if (TOP1) {
                     if (r_lo < p.N) {
                         const uint64_t k0 = make_key(acc[0], static_cast<uint32_t>(r_lo));
@@ -420,6 +533,7 @@ scan_kernel(const ScanParams p) {
                             push_candidate(hdr, cand, p.cap, p.soft_limit, q1,
                                            make_key(acc[3], static_cast<uint32_t>(r_hi)));
                     }
+                }
                 }
             } else {
                 // ---- FMA flavour: RG rows at a time, RG * SQ = 16 partial sums
@@ -487,6 +601,7 @@ scan_kernel(const ScanParams p) {
         // ------------------------------------------------------------ CTA result
         if (TOP1) {
             if (MMA) {
+                // (the L2 flavour has put its keys into hdr->best as it went)
                 if (best0) atomicMax(&hdr->best[2 * t], static_cast<unsigned long long>(best0));
                 if (best1) atomicMax(&hdr->best[2 * t + 1], static_cast<unsigned long long>(best1));
             } else {

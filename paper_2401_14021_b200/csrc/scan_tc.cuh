@@ -1,0 +1,399 @@
+// Corpus scan for large query batches (inner product, up to 512 queries per pass) on the
+// fifth-generation tensor cores: scores = corpus tile [128 rows] x queries^T [up to 256] with
+// tcgen05.mma, fp16 operands, fp32 accumulators in tensor memory (TMEM), fused with the
+// per-CTA top-k selection so that the N x s score matrix never exists in memory.
+//
+// One persistent CTA per SM, 6 warps:
+//   warp 0      producer: one thread issues the TMA tile loads. A stage holds one K chunk
+//               (64 fp16 = 128 bytes per row, the 128-byte swizzle span) of 128 corpus rows
+//               and of up to 256 queries; stages form a ring guarded by full/empty mbarriers.
+//   warp 1      MMA: one thread issues tcgen05.mma (M = 128, N = 16..256, K = 16 per
+//               instruction, 4 per chunk). A work unit is (row tile, half of the queries);
+//               the two halves of TMEM (256 columns each) alternate between units, so one
+//               accumulator is drained while the next is being filled.
+//   warps 2..5  selection: each warp owns one quarter of the TMEM lanes (32 corpus rows),
+//               reads the scores with tcgen05.ld, compares each with its query's threshold
+//               (the CTA's current k-th best) and appends what passes to that query's
+//               candidate list in global memory. Lists are compacted (sorted, cut to k,
+//               threshold raised) by the same warps between units, before they can overflow.
+//
+// Every wait is bounded; when one runs out the CTA records kStatusTimeout, lets copies and
+// MMAs in flight finish, frees its TMEM and returns.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace ralm {
+
+constexpr int kTcThreads = 192;
+constexpr int kTcTileM = 128;    // corpus rows per tile = TMEM lanes
+constexpr int kTcMaxN = 256;     // queries per accumulator = TMEM columns per half
+constexpr int kTcChunkK = 64;    // fp16 per K chunk (128 bytes: one swizzle span)
+constexpr int kTcMaxQueries = 2 * kTcMaxN;
+constexpr int kTcABytes = kTcTileM * kTcChunkK * 2;
+constexpr int kTcMaxStages = 12;
+constexpr int kTcCap = 256;      // candidate slots per (CTA, query)
+constexpr int kTcSoft = 128;     // a list holding this many is compacted before the next unit
+constexpr int kTcMaxK = 64;      // k <= kTcSoft / 2 keeps compactions rare
+constexpr int kTcTmemCols = 512;
+
+struct TcParams {
+    uint64_t *partial;  // [gridDim.x][s_total][k] sorted keys, 0 = empty
+    uint64_t *cand;     // [gridDim.x][cand_q][kTcCap] candidate lists
+    int *status;
+    long long N;
+    long long ntiles;   // ceil(N / 128)
+    int nchunks;        // ceil(d / 64)
+    int s;              // queries in this pass (<= 512)
+    int s_total;
+    int q_base;
+    int k;
+    int nb;             // query rows per stage = rows of the query TMA box (16..256, multiple of 16)
+    int nhalves;        // ceil(s / nb): 1 or 2
+    int stages;
+    int stage_bytes;    // kTcABytes + nb * 128, a multiple of 1024
+    int off_stage;      // shared-memory offset of the stage ring (1024-byte aligned)
+    int cand_q;         // queries the candidate workspace was sized for (>= s)
+};
+
+struct TcHeader {
+    uint64_t full[kTcMaxStages];
+    uint64_t empty[kTcMaxStages];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    int abort;
+    int dirty;  // some candidate list reached kTcSoft during the current unit
+};
+constexpr int kTcHeaderBytes = 512;
+static_assert(sizeof(TcHeader) <= kTcHeaderBytes, "header too large");
+// shared-memory layout after the header
+constexpr int kTcOffThr = kTcHeaderBytes;                      // float [512]
+constexpr int kTcOffCnt = kTcOffThr + kTcMaxQueries * 4;       // int [512]
+constexpr int kTcOffSorted = kTcOffCnt + kTcMaxQueries * 4;    // int [512]
+constexpr int kTcOffScratch = kTcOffSorted + kTcMaxQueries * 4;  // u64 [4][256]
+constexpr int kTcOffEnd = kTcOffScratch + 4 * kTcCap * 8;
+
+// ---- tcgen05 / TMA wrappers -------------------------------------------------------------
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, fp16 x fp16 -> fp32
+__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                           uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Shared-memory operand descriptor: K-major tile, 128-byte swizzle, rows 128 bytes apart,
+// groups of 8 rows 1024 bytes apart; `addr` may be advanced by 32 bytes per K step of 16.
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr) {
+    uint64_t desc = (addr & 0x3FFFFu) >> 4;         // start address, 16-byte units
+    desc |= static_cast<uint64_t>(1) << 16;         // leading byte offset (unused with swizzle)
+    desc |= static_cast<uint64_t>(1024 >> 4) << 32; // stride byte offset: next group of 8 rows
+    desc |= static_cast<uint64_t>(1) << 46;         // descriptor version of this architecture
+    desc |= static_cast<uint64_t>(2) << 61;         // 128-byte swizzle
+    return desc;
+}
+// Instruction descriptor: fp16 A and B (both K-major), fp32 accumulator, M = 128, N = n.
+__device__ __forceinline__ uint32_t tc_idesc(int n) {
+    return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTcTileM >> 4) << 24);
+}
+// 32 consecutive columns of this thread's TMEM lane, then wait for the load.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]),
+          "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+          "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+// One selection warp sorts query q's candidate list (n <= 256 keys in global memory), keeps
+// the best k there, raises the threshold.
+__device__ inline void tc_compact_query(uint64_t *list, uint64_t *scratch, float *thr, int *cnt,
+                                        int *sorted, int q, int k, int lane) {
+    const int n = cnt[q];
+    for (int i = lane; i < kTcCap; i += 32) scratch[i] = (i < n) ? list[i] : 0ull;
+    __syncwarp();
+    bitonic_sort_desc(scratch, kTcCap, lane, 32, -2);
+    const int keep = n < k ? n : k;
+    for (int i = lane; i < keep; i += 32) list[i] = scratch[i];
+    if (lane == 0) {
+        cnt[q] = keep;
+        sorted[q] = keep;
+        thr[q] = (n >= k) ? key_value(scratch[k - 1]) : -INFINITY;
+    }
+    __syncwarp();
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_q,
+               const TcParams p) {
+    extern __shared__ __align__(1024) unsigned char tc_smem[];
+    TcHeader *hdr = reinterpret_cast<TcHeader *>(tc_smem);
+    float *thr = reinterpret_cast<float *>(tc_smem + kTcOffThr);
+    int *cnt = reinterpret_cast<int *>(tc_smem + kTcOffCnt);
+    int *sorted = reinterpret_cast<int *>(tc_smem + kTcOffSorted);
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int S = p.stages;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < S; ++i) {
+            mbar_init(smem_u32(&hdr->full[i]), 1);
+            mbar_init(smem_u32(&hdr->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&hdr->tmem_full[i]), 1);
+            mbar_init(smem_u32(&hdr->tmem_empty[i]), 4);  // one arrival per selection warp
+        }
+        mbar_init(smem_u32(&hdr->drain), 1);
+        mbar_fence_init();
+        hdr->abort = 0;
+        hdr->dirty = 0;
+    }
+    for (int q = threadIdx.x; q < kTcMaxQueries; q += kTcThreads) {
+        thr[q] = (q < p.s) ? -INFINITY : INFINITY;  // absent queries never pass
+        cnt[q] = 0;
+        sorted[q] = 0;
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(&hdr->tmem_base)),
+                     "r"(kTcTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&hdr->tmem_base);
+
+    const long long my_tiles =
+        (p.ntiles > blockIdx.x) ? (p.ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const long long my_units = my_tiles * p.nhalves;
+    volatile int *abort_flag = &hdr->abort;
+    const uint32_t stage_base = smem_u32(tc_smem + p.off_stage);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            const uint32_t stage_tx = static_cast<uint32_t>(kTcABytes + p.nb * 128);
+            int st = 0;
+            uint32_t lap = 0;
+            long long issued = 0;
+            bool ok = true, stop = false;
+            for (long long u = 0; u < my_units && !stop; ++u) {
+                const long long tile = blockIdx.x + (u / p.nhalves) * gridDim.x;
+                const int half = static_cast<int>(u % p.nhalves);
+                for (int c = 0; c < p.nchunks; ++c) {
+                    ok = mbar_wait_bounded(smem_u32(&hdr->empty[st]), (lap & 1) ^ 1);
+                    if (!ok || *abort_flag) {
+                        stop = true;
+                        break;
+                    }
+                    const uint32_t bar = smem_u32(&hdr->full[st]);
+                    const uint32_t dst = stage_base + static_cast<uint32_t>(st) * p.stage_bytes;
+                    mbar_arrive_expect_tx(bar, stage_tx);
+                    tma_load_2d(dst, &map_x, c * kTcChunkK, static_cast<int>(tile * kTcTileM), bar);
+                    tma_load_2d(dst + kTcABytes, &map_q, c * kTcChunkK, half * p.nb, bar);
+                    ++issued;
+                    if (++st == S) {
+                        st = 0;
+                        ++lap;
+                    }
+                }
+            }
+            if (!ok && !*abort_flag) {
+                atomicMax(p.status, kStatusTimeout);
+                *abort_flag = 1;
+            }
+            if (*abort_flag) {
+                // winding down early: let every copy already issued land before exit
+                const long long first = issued > S ? issued - S : 0;
+                for (long long it = first; it < issued; ++it)
+                    mbar_wait_bounded(smem_u32(&hdr->full[it % S]), static_cast<uint32_t>((it / S) & 1));
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int st = 0;
+            uint32_t lap = 0;
+            bool ok = true;
+            for (long long u = 0; u < my_units && ok; ++u) {
+                const int half = static_cast<int>(u % p.nhalves);
+                const int acc = static_cast<int>(u & 1);
+                const int nq = (p.s - half * p.nb < p.nb) ? (p.s - half * p.nb) : p.nb;
+                const uint32_t idesc = tc_idesc((nq + 15) & ~15);
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kTcMaxN);
+                // the selection warps must have drained this accumulator's previous unit
+                ok = mbar_wait_bounded(smem_u32(&hdr->tmem_empty[acc]), static_cast<uint32_t>(((u >> 1) & 1) ^ 1));
+                if (!ok || *abort_flag) break;
+                tc_fence_after();
+                for (int c = 0; c < p.nchunks; ++c) {
+                    ok = mbar_wait_bounded(smem_u32(&hdr->full[st]), lap & 1);
+                    if (!ok || *abort_flag) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = stage_base + static_cast<uint32_t>(st) * p.stage_bytes;
+                    const uint32_t b_addr = a_addr + kTcABytes;
+#pragma unroll
+                    for (int kk = 0; kk < kTcChunkK / 16; ++kk)
+                        tc_mma_f16(d_tmem, tc_smem_desc(a_addr + kk * 32), tc_smem_desc(b_addr + kk * 32),
+                                   idesc, (c | kk) != 0 ? 1u : 0u);
+                    tc_commit(smem_u32(&hdr->empty[st]));  // stage reusable once these MMAs are done
+                    if (++st == S) {
+                        st = 0;
+                        ++lap;
+                    }
+                }
+                if (!ok || *abort_flag) break;
+                tc_commit(smem_u32(&hdr->tmem_full[acc]));
+            }
+            if (!ok && !*abort_flag) {
+                atomicMax(p.status, kStatusTimeout);
+                *abort_flag = 1;
+            }
+            // every MMA issued above must have completed before the TMEM is given back
+            tc_commit(smem_u32(&hdr->drain));
+            mbar_wait_bounded(smem_u32(&hdr->drain), 0);
+        }
+    } else {
+        // ------------------------------------------------------------------ selection
+        const int ew = warp - 2;        // 0..3
+        const int quarter = warp & 3;   // the TMEM lanes this warp may read: 32 * quarter ..
+        uint64_t *my_cand = p.cand + static_cast<size_t>(blockIdx.x) * p.cand_q * kTcCap;
+        uint64_t *scratch = reinterpret_cast<uint64_t *>(tc_smem + kTcOffScratch) + ew * kTcCap;
+        volatile int *dirty = &hdr->dirty;
+        bool ok = true;
+        for (long long u = 0; u < my_units; ++u) {
+            const long long tile = blockIdx.x + (u / p.nhalves) * gridDim.x;
+            const int half = static_cast<int>(u % p.nhalves);
+            const int acc = static_cast<int>(u & 1);
+            const int qb = half * p.nb;
+            const int nq = (p.s - qb < p.nb) ? (p.s - qb) : p.nb;
+            if (ok && !*abort_flag) {
+                int got = 0;
+                if (lane == 0)
+                    got = mbar_wait_bounded(smem_u32(&hdr->tmem_full[acc]), static_cast<uint32_t>((u >> 1) & 1)) ? 1 : 0;
+                got = __shfl_sync(0xffffffffu, got, 0);
+                if (!got) {
+                    ok = false;
+                    if (lane == 0) {
+                        atomicMax(p.status, kStatusTimeout);
+                        *abort_flag = 1;
+                    }
+                }
+            }
+            const bool live = ok && !*abort_flag;
+            if (live) {
+                tc_fence_after();
+                const long long row = tile * kTcTileM + quarter * 32 + lane;
+                const bool row_ok = row < p.N;
+                const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                       static_cast<uint32_t>(acc * kTcMaxN);
+                for (int j = 0; j * 32 < nq; ++j) {
+                    uint32_t v[32];
+                    tmem_ld32(t_row + j * 32, v);
+                    const float4 *t4 = reinterpret_cast<const float4 *>(thr + qb + j * 32);
+                    uint32_t hit = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 th = t4[i];
+                        hit |= (__uint_as_float(v[4 * i + 0]) >= th.x ? 1u : 0u) << (4 * i + 0);
+                        hit |= (__uint_as_float(v[4 * i + 1]) >= th.y ? 1u : 0u) << (4 * i + 1);
+                        hit |= (__uint_as_float(v[4 * i + 2]) >= th.z ? 1u : 0u) << (4 * i + 2);
+                        hit |= (__uint_as_float(v[4 * i + 3]) >= th.w ? 1u : 0u) << (4 * i + 3);
+                    }
+                    if (row_ok && hit) {
+#pragma unroll
+                        for (int b = 0; b < 32; ++b) {
+                            if (hit & (1u << b)) {
+                                const int q = qb + j * 32 + b;
+                                const int slot = atomicAdd(&cnt[q], 1);
+                                my_cand[static_cast<size_t>(q) * kTcCap + slot] =
+                                    make_key(__uint_as_float(v[b]), static_cast<uint32_t>(row));
+                                if (slot + 1 >= kTcSoft) *dirty = 1;
+                            }
+                        }
+                    }
+                }
+                // accumulator drained: hand it back to the MMA warp
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&hdr->tmem_empty[acc]));
+            }
+            // All four warps meet after every unit (also when winding down, so that nobody is
+            // left waiting): first so that every push of the unit is visible, then, having all
+            // read the same value of the flag, to compact the lists that asked for it.
+            named_barrier(1, 128);
+            const int need = *dirty;
+            named_barrier(1, 128);
+            if (need) {
+                for (int base = 0; base < p.s; base += 128) {
+                    const int q = base + ew * 32 + lane;
+                    unsigned m = __ballot_sync(0xffffffffu, q < p.s && cnt[q] >= kTcSoft);
+                    while (m) {
+                        const int b = __ffs(m) - 1;
+                        m &= m - 1;
+                        const int qq = base + ew * 32 + b;
+                        tc_compact_query(my_cand + static_cast<size_t>(qq) * kTcCap, scratch, thr, cnt, sorted,
+                                         qq, p.k, lane);
+                    }
+                }
+                if (threadIdx.x == 64) *dirty = 0;
+                named_barrier(1, 128);
+            }
+        }
+        // ---- CTA result: every list sorted and cut to k, written as this CTA's partial lists
+        for (int base = 0; base < p.s; base += 128) {
+            const int q0 = base + ew * 32;
+            for (int b = 0; b < 32 && q0 + b < p.s; ++b) {
+                const int q = q0 + b;
+                uint64_t *list = my_cand + static_cast<size_t>(q) * kTcCap;
+                if (cnt[q] != sorted[q]) tc_compact_query(list, scratch, thr, cnt, sorted, q, p.k, lane);
+                const int n = cnt[q];
+                uint64_t *dst = p.partial + (static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
+                for (int i = lane; i < p.k; i += 32) dst[i] = (i < n) ? list[i] : 0ull;
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTcTmemCols)
+                     : "memory");
+    }
+}
+
+}  // namespace ralm

@@ -29,20 +29,23 @@ def _run(corpus, queries, metric, k, variant=0):
     return ids, scores
 
 
-VARIANTS = {oracle.IP: (2, 1), oracle.L2: (1,)}
+VARIANTS = {oracle.IP: (2, 1), oracle.L2: (2, 1)}
 
 
 # ------------------------------------------------------------------ exact integer cases
 @pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
 @pytest.mark.parametrize("N,d,s,k", [(1, 8, 1, 1), (15, 8, 3, 4), (16, 16, 8, 1), (17, 64, 5, 20),
                                      (33, 40, 2, 40), (1000, 72, 8, 7), (5000, 768, 4, 5),
-                                     (3001, 1024, 4, 1024), (257, 264, 9, 3), (64, 8, 17, 64)])
+                                     (3001, 1024, 4, 1024), (257, 264, 9, 3), (64, 8, 17, 64),
+                                     (700, 2048, 3, 9)])
 def test_integer_inputs_are_bit_exact(metric, N, d, s, k):
     """Small-integer rows: every score is an integer that fp32 holds exactly, and ties abound,
     so ids (tie-break included) and scores must equal the oracle's bit for bit."""
     x = workloads.integer_valued((N, d), seed=100 + N, lo=-3, hi=3, device=DEV)
     q = workloads.integer_valued((s, d), seed=200 + N, lo=-3, hi=3, device=DEV)
     for variant in VARIANTS[metric]:
+        if variant == 1 and d > 1024:
+            continue                       # the FMA scan keeps a whole query slice in registers
         ids, scores = _run(x, q, metric, k, variant)
         check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), metric, k, exact=True)
 
@@ -116,8 +119,9 @@ def test_adversarial_row_order_sorted_by_score():
     for variant in (2, 1):
         ids, scores = _run(x, q, oracle.IP, 100, variant)
         check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 100, exact=True)
-    ids, scores = _run(x, q[:1].contiguous(), oracle.L2, 1024)
-    check_search(ids, scores, x.cpu().numpy(), q[:1].cpu().numpy(), oracle.L2, 1024, exact=True)
+    for variant in (2, 1):
+        ids, scores = _run(x, q[:1].contiguous(), oracle.L2, 1024, variant)
+        check_search(ids, scores, x.cpu().numpy(), q[:1].cpu().numpy(), oracle.L2, 1024, exact=True)
 
 
 def test_clustered_row_order():
@@ -169,7 +173,52 @@ def test_argument_errors():
         idx.set_variant(7)
     l2 = ralm.Index(x, oracle.L2, 2, 5)
     with pytest.raises(ralm.RalmError):
-        l2.set_variant(2)                 # warp-MMA scan cannot serve L2
+        l2.set_variant(3)                 # the tcgen05 scan cannot serve L2
+
+
+# ------------------------------------------------------------------ large batches (tcgen05 scan)
+@pytest.mark.parametrize("N,d,s,k", [(1, 64, 1, 1), (129, 72, 3, 1), (300, 128, 9, 64), (1000, 64, 16, 5),
+                                     (5000, 768, 100, 20), (257, 64, 257, 2), (3000, 256, 600, 7),
+                                     (40_000, 768, 512, 20)])
+def test_tcgen05_scan_integer_inputs_are_bit_exact(N, d, s, k):
+    """The large-batch scan pinned explicitly (variant 3), including shapes with a ragged last
+    K chunk (d % 64 != 0), a ragged row tile, a second query half and a second pass."""
+    x = workloads.integer_valued((N, d), seed=400 + N, lo=-3, hi=3, device=DEV)
+    q = workloads.integer_valued((s, d), seed=500 + N, lo=-3, hi=3, device=DEV)
+    ids, scores = _run(x, q, oracle.IP, k, 3)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+
+
+@pytest.mark.parametrize("N,d,s,k", [(100_003, 768, 300, 20), (250_000, 128, 64, 1), (20_000, 1024, 512, 33)])
+def test_tcgen05_scan_parity(N, d, s, k):
+    """Real-valued mixture rows; s >= 9 takes the large-batch scan by itself (variant 0)."""
+    x, _ = workloads.mixture_corpus(N, d, 64, seed=600 + d, device=DEV)
+    q, src = workloads.noisy_copy_queries(x, s, seed=601 + d)
+    ids, scores = _run(x, q, oracle.IP, k)
+    strict, band = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k)
+    assert ids[:, 0].tolist() == src.tolist()
+    ids8, scores8 = _run(x, q, oracle.IP, k, 2)          # the 8-queries-per-pass scan on the same batch
+    assert torch.equal(ids[:, 0], ids8[:, 0])
+    torch.testing.assert_close(scores, scores8, rtol=1e-4, atol=1e-5)
+
+
+def test_tcgen05_scan_adversarial_row_order():
+    """Scores increase along the corpus: every row passes every threshold, so every unit ends
+    in a compaction of every list."""
+    N, d = 30_000, 64
+    x = torch.zeros((N, d), dtype=torch.float16, device=DEV)
+    x[:, 0] = (torch.arange(N, device=DEV) // 16).to(torch.float16)
+    q = torch.zeros((12, d), dtype=torch.float16, device=DEV)
+    q[:, 0] = torch.tensor([1, -1, 2, -2, 1, 1, -1, 3, 0, 1, -3, 2], dtype=torch.float16)
+    ids, scores = _run(x, q, oracle.IP, 64, 3)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 64, exact=True)
+
+
+def test_large_k_falls_back_from_the_tcgen05_scan():
+    x, _ = workloads.mixture_corpus(30_000, 128, 16, seed=71, device=DEV)
+    q, _ = workloads.noisy_copy_queries(x, 20, seed=72)
+    ids, scores = _run(x, q, oracle.IP, 200)             # k beyond the large-batch scan's limit
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 200)
 
 
 # ------------------------------------------------------------------ the configs
@@ -207,7 +256,8 @@ def test_knn_lm_shape_l2_k1024():
     x, _ = workloads.mixture_corpus(1_000_000, 1024, 4096, workloads.seed_for(4), device=DEV,
                                     normalise=False, lognormal_sigma=0.3)
     q, src = workloads.noisy_copy_queries(x, 4, workloads.seed_for(4, "queries"))
-    ids, scores = _run(x, q, oracle.L2, 1024)
-    strict, band = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, 1024)
-    assert ids[:, 0].tolist() == src.tolist()
-    print("C4/50 strict=%d band=%d" % (strict, band))
+    for variant in (2, 1):
+        ids, scores = _run(x, q, oracle.L2, 1024, variant)
+        strict, band = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, 1024)
+        assert ids[:, 0].tolist() == src.tolist()
+        print("C4/50 variant=%d strict=%d band=%d" % (variant, strict, band))
