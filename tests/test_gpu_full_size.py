@@ -1,0 +1,157 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle cannot rank 21 M or 50 M rows in seconds, so the check is sampled, in a way that
+still catches a missed row: the oracle ranks a SUB-CORPUS made of (a) seeded random chunks of
+rows, the first rows and the ragged tail and (b) every row the GPU returned. If the GPU's
+lists are the top-k of the whole corpus they are also the top-k of any sub-corpus that contains
+them, so the oracle's ranking of the sub-corpus must reproduce them (ids by the near-tie rule,
+scores within tolerance); a sampled row that the GPU wrongly left out shows up as a mismatch.
+Rank 0 must also be the row each query was copied from.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+from parity import check_lists
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _ralm():
+    import paper_2401_14021_b200 as ralm
+    return ralm
+
+
+def _sampled_parity(x, q, ids, scores, metric, k, n_chunks, chunk_rows, seed, query_sel=None):
+    N = x.shape[0]
+    sel = list(range(q.shape[0])) if query_sel is None else list(query_sel)
+    g = torch.Generator().manual_seed(seed)
+    starts = (torch.randint(0, max(1, N // chunk_rows), (n_chunks,), generator=g) * chunk_rows).tolist()
+    starts += [0, max(0, N - chunk_rows + 1)]
+    rows = torch.cat([torch.arange(s0, min(N, s0 + chunk_rows)) for s0 in sorted(set(starts))])
+    gi, gs = ids.cpu(), scores.cpu().numpy()
+    returned = gi[sel].flatten()
+    sub_rows = torch.unique(torch.cat([rows, returned[returned >= 0]]))     # ascending: id order is kept
+    xs = x[sub_rows.to(x.device)].cpu().numpy()
+    qn = q.cpu().numpy()[sel]
+    o_local, o_scores = oracle.search(xs, qn, metric, k)
+    o_ids = np.where(o_local >= 0, sub_rows.numpy()[np.maximum(o_local, 0)], -1)
+    pos = {int(r): i for i, r in enumerate(sub_rows.tolist())}
+    max_norm = float(np.linalg.norm(xs.astype(np.float64), axis=1).max())
+    strict = band = 0
+    for n, i in enumerate(sel):
+        scale = max_norm * float(np.linalg.norm(qn[n].astype(np.float64)))
+        a, b = check_lists(gi[i].numpy(), gs[i], o_ids[n], o_scores[n],
+                           lambda j, n=n: oracle.pair_score(xs[pos[j]], qn[n], metric), metric,
+                           scale=scale, n_valid=N)
+        strict += a
+        band += b
+    return strict, band, sub_rows.numel()
+
+
+@pytest.fixture(scope="module")
+def c3_corpus():
+    c = workloads.CONFIGS["C3"]
+    x, assign = workloads.mixture_corpus(c.N, c.d, c.n_centres, workloads.seed_for(3), device=DEV)
+    yield x, assign
+    del x, assign
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("k", [1, 20])
+def test_c3_full_size_s8(c3_corpus, k):
+    """The headline configuration: 21 M x 768, inner product, s = 8."""
+    ralm = _ralm()
+    x, _ = c3_corpus
+    q, src = workloads.noisy_copy_queries(x, 8, workloads.seed_for(3, "queries"))
+    idx = ralm.Index(x, oracle.IP, max_s=8, max_k=k)
+    ids, scores = ralm.search(idx, q, k)
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    assert ids[:, 0].tolist() == src.tolist()
+    strict, band, n_sub = _sampled_parity(x, q, ids, scores, oracle.IP, k, 30, 16_384, seed=3300 + k)
+    print("C3 k=%d: strict=%d band=%d over a %d-row sub-corpus" % (k, strict, band, n_sub))
+    # every s in 1..8 returns the same rows for the queries it shares with the full batch
+    for s in (1, 3, 5):
+        ids_s, _ = ralm.search(idx, q[:s].contiguous(), k)
+        assert torch.equal(ids_s, ids[:s])
+    idx.close()
+
+
+def test_c3_serving_step_cache_and_verify(c3_corpus):
+    """8 concurrent requests x 512-entry caches x stride 8 on the full corpus: cache lookup and
+    first-mismatch positions against the oracle (which only needs the cached rows)."""
+    ralm = _ralm()
+    x, assign = c3_corpus
+    c = workloads.CONFIGS["C3"]
+    R, stride, C = c.requests, c.stride, c.cache_entries
+    q, src = workloads.noisy_copy_queries(x, R * stride, workloads.seed_for(3, "queries"))
+    cache = workloads.speculation_cache_ids(assign, c.N, src.reshape(R, stride), C,
+                                            workloads.seed_for(3, "caches"), n_centres=c.n_centres)
+    idx = ralm.Index(x, oracle.IP, max_s=R * stride, max_k=1)
+    qr = q.reshape(R, stride, c.d).contiguous()
+    spec, spec_scores = ralm.cache_search(idx, cache, qr, 1)
+    retr, _ = ralm.search(idx, q, 1)
+    m = ralm.verify(spec.reshape(R, stride).contiguous(), retr.reshape(R, stride, 1).contiguous())
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    assert retr[:, 0].tolist() == src.tolist()
+    # oracle on the cached rows only: gather them, rank locally, map back
+    cache_h = cache.cpu()
+    uniq = torch.unique(cache_h[cache_h >= 0])
+    xs = x[uniq.to(DEV)].cpu().numpy()
+    local = torch.searchsorted(uniq, cache_h.clamp_min(0))
+    local = torch.where(cache_h >= 0, local, torch.full_like(local, -1)).numpy()
+    o_local, o_scores = oracle.cache_search(xs, local, qr.cpu().numpy(), oracle.IP, 1)
+    o_spec = np.where(o_local >= 0, uniq.numpy()[np.maximum(o_local, 0)], -1)
+    assert np.array_equal(spec.cpu().numpy(), o_spec)
+    np.testing.assert_allclose(spec_scores.cpu().numpy(), o_scores, rtol=2e-3, atol=1e-5)
+    o_m = oracle.verify(o_spec.reshape(R, stride), retr.cpu().numpy().reshape(R, stride, 1))
+    assert np.array_equal(m.cpu().numpy(), o_m)
+    print("C3 first-mismatch positions:", m.cpu().tolist())
+    idx.close()
+
+
+def test_c5_full_size_512_queries(c3_corpus):
+    """The high-concurrency configuration: 512 queries, k = 20, on the tcgen05 scan."""
+    ralm = _ralm()
+    x, _ = c3_corpus
+    q, src = workloads.noisy_copy_queries(x, 512, workloads.seed_for(3, "queries"))
+    idx = ralm.Index(x, oracle.IP, max_s=512, max_k=20)
+    ids, scores = ralm.search(idx, q, 20)
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    assert ids[:, 0].tolist() == src.tolist()
+    strict, band, n_sub = _sampled_parity(x, q, ids, scores, oracle.IP, 20, 6, 16_384, seed=3500,
+                                          query_sel=range(0, 512, 8))
+    print("C5: strict=%d band=%d over a %d-row sub-corpus, 64 of 512 queries" % (strict, band, n_sub))
+    # the first 8 queries through the small-batch scan give the same rows
+    ids8, scores8 = ralm.search(idx, q[:8].contiguous(), 20)
+    assert torch.equal(ids8[:, 0], ids[:8, 0])
+    torch.testing.assert_close(scores8, scores[:8], rtol=1e-4, atol=1e-5)
+    idx.close()
+
+
+def test_c4_full_size_l2_k1024():
+    """The KNN-LM datastore: 50 M x 1024 (102.4 GB), L2, s = 4, k = 1024."""
+    ralm = _ralm()
+    c = workloads.CONFIGS["C4"]
+    free, _ = torch.cuda.mem_get_info()
+    if free < c.N * c.d * 2 + (8 << 30):
+        pytest.skip("needs %.0f GB of free device memory" % ((c.N * c.d * 2 + (8 << 30)) / 1e9))
+    x, _ = workloads.mixture_corpus(c.N, c.d, c.n_centres, workloads.seed_for(4), device=DEV,
+                                    normalise=False, lognormal_sigma=c.lognormal_sigma)
+    q, src = workloads.noisy_copy_queries(x, 4, workloads.seed_for(4, "queries"))
+    idx = ralm.Index(x, oracle.L2, max_s=4, max_k=1024)
+    ids, scores = ralm.search(idx, q, 1024)
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    assert ids[:, 0].tolist() == src.tolist()
+    strict, band, n_sub = _sampled_parity(x, q, ids, scores, oracle.L2, 1024, 14, 16_384, seed=3400)
+    print("C4: strict=%d band=%d over a %d-row sub-corpus" % (strict, band, n_sub))
+    idx.close()
+    del x
+    torch.cuda.empty_cache()
