@@ -29,7 +29,10 @@ struct ralm_index {
     int tune_warps, tune_depth, tune_rows;  // 0 = library default
     uint64_t *partial;   // [num_sms][max_s][max_k]
     uint64_t *cache_keys;  // [RALM_MAX_CACHE_KEYS]
+    uint64_t *spill;       // large k: candidate lists of the small-batch scan, [num_sms][8][spill_cap]
+    int spill_cap;
     float *norms;          // L2: squared norm of every corpus row (fp32 [N]), or null
+    int tc_clusters;       // CTA pairs the device runs at once (-1 = not asked yet)
     uint64_t *tc_cand;     // tcgen05 scan: [num_sms][tc_cand_q][kTcCap] candidate lists, or null
     int tc_cand_q;
     int *status;
@@ -48,7 +51,10 @@ namespace {
 
 struct ScanPlan {
     int nwarps, depth, tile_rows, stage_bytes, cap, soft_limit, off_q, off_cand, off_stage, smem_bytes;
+    bool spill;  // candidate lists in global memory, one sort scratch in shared memory
 };
+
+constexpr int kSmemCandBytes = 32 * 1024;  // candidate lists larger than this leave shared memory
 
 int align_up(int v, int a) { return (v + a - 1) / a * a; }
 
@@ -69,11 +75,15 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
     pl->off_cand = off;
     pl->cap = 0;
     pl->soft_limit = 0;
+    pl->spill = false;
     if (k > 1) {
         // after the flag is raised every warp may still finish the tile it is on
         pl->cap = std::max(512, 2 * next_pow2(k));
         pl->soft_limit = pl->cap - (kMaxConsumerWarps + 1) * pl->tile_rows;
-        off += s_pass * pl->cap * 8;
+        // the stage ring needs the room more than large lists do: those go to global memory
+        // (they are touched rarely) and only the scratch they are sorted in stays here
+        pl->spill = s_pass * pl->cap * 8 > kSmemCandBytes && idx->spill && pl->cap <= idx->spill_cap;
+        off += (pl->spill ? 1 : s_pass) * pl->cap * 8;
     }
     pl->off_stage = align_up(off, 128);
     const int room = idx->smem_optin - pl->off_stage;
@@ -174,36 +184,77 @@ bool alloc_tc_workspace(ralm_index *idx, int queries) {
     return true;
 }
 
-// One pass of up to min(512, workspace) queries.
+// One pass of up to min(512, workspace) queries. `pair`: clusters of two CTAs that share each
+// MMA (half the query bytes staged per CTA); falls back to single CTAs when no cluster fits.
 ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int s_total, int q0, int k,
-                             int grid, cudaStream_t st) {
+                             bool pair, int *grid_out, cudaStream_t st) {
     TcParams p;
     p.partial = idx->partial;
     p.cand = idx->tc_cand;
     p.cand_q = idx->tc_cand_q;
     p.status = idx->status;
     p.N = idx->N;
-    p.ntiles = (idx->N + kTcTileM - 1) / kTcTileM;
     p.nchunks = (idx->d + kTcChunkK - 1) / kTcChunkK;
     p.s = sp;
     p.s_total = s_total;
     p.q_base = q0;
     p.k = k;
-    p.nb = sp > kTcMaxN ? kTcMaxN : align_up(sp, 16);
-    p.nhalves = (sp + p.nb - 1) / p.nb;
-    p.stage_bytes = kTcABytes + p.nb * 128;
     p.off_stage = align_up(kTcOffEnd, 1024);
-    p.stages = std::min(kTcMaxStages, (idx->smem_optin - p.off_stage) / p.stage_bytes);
-    if (p.stages < 2) return RALM_ERR_UNSUPPORTED;
-    const int smem = p.off_stage + p.stages * p.stage_bytes;
     CUtensorMap map_x, map_q;
-    if (!encode_rows_map(&map_x, idx->corpus, idx->N, idx->d, kTcTileM) ||
-        !encode_rows_map(&map_q, queries, sp, idx->d, p.nb))
-        return RALM_ERR_CUDA;
-    if (cudaFuncSetAttribute(scan_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-        return RALM_ERR_CUDA;
-    scan_tc_kernel<<<grid, kTcThreads, smem, st>>>(map_x, map_q, p);
-    return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
+    if (!encode_rows_map(&map_x, idx->corpus, idx->N, idx->d, kTcTileM)) return RALM_ERR_CUDA;
+    for (;;) {
+        const int group_rows = pair ? 2 * kTcTileM : kTcTileM;
+        p.ntiles = (idx->N + group_rows - 1) / group_rows;
+        p.nb = sp > kTcMaxN ? kTcMaxN : align_up(sp, pair ? 32 : 16);
+        p.nhalves = (sp + p.nb - 1) / p.nb;
+        const int nb_cta = pair ? p.nb / 2 : p.nb;
+        p.stage_bytes = kTcABytes + nb_cta * 128;
+        p.stages = std::min(kTcMaxStages, (idx->smem_optin - p.off_stage) / p.stage_bytes);
+        if (p.stages < 2) return RALM_ERR_UNSUPPORTED;
+        const int smem = p.off_stage + p.stages * p.stage_bytes;
+        if (!encode_rows_map(&map_q, queries, sp, idx->d, nb_cta)) return RALM_ERR_CUDA;
+        if (!pair) {
+            const int grid = static_cast<int>(std::min<long long>(idx->num_sms, p.ntiles));
+            if (cudaFuncSetAttribute(scan_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+                cudaSuccess)
+                return RALM_ERR_CUDA;
+            scan_tc_kernel<false><<<grid, kTcThreads, smem, st>>>(map_x, map_q, p);
+            *grid_out = grid;
+            return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
+        }
+        if (cudaFuncSetAttribute(scan_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
+            cudaSuccess)
+            return RALM_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.gridDim = dim3(2, 1, 1);
+        cfg.blockDim = dim3(kTcThreads, 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (idx->tc_clusters < 0) {
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, scan_tc_kernel<true>, &cfg) != cudaSuccess) {
+                cudaGetLastError();
+                n = 0;
+            }
+            idx->tc_clusters = std::min(n, idx->num_sms / 2);
+        }
+        if (idx->tc_clusters < 1) {  // no room for a pair on this device: single CTAs
+            pair = false;
+            continue;
+        }
+        const int clusters = static_cast<int>(std::min<long long>(idx->tc_clusters, p.ntiles));
+        cfg.gridDim = dim3(2 * clusters, 1, 1);
+        *grid_out = 2 * clusters;
+        return cudaLaunchKernelEx(&cfg, scan_tc_kernel<true>, map_x, map_q, p) == cudaSuccess ? RALM_OK
+                                                                                              : RALM_ERR_CUDA;
+    }
 }
 
 constexpr int kTcAutoMinQueries = 9;  // batches the 8-query scan cannot serve in one pass
@@ -211,9 +262,10 @@ constexpr int kTcAutoMinQueries = 9;  // batches the 8-query scan cannot serve i
 ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k, int64_t *ids,
                             float *scores, cudaStream_t st) {
     if (s == 0) return RALM_OK;
-    const bool tc = tc_can_serve(idx, k) && (idx->variant == 3 || (idx->variant == 0 && s >= kTcAutoMinQueries));
+    const bool tc = tc_can_serve(idx, k) &&
+                    (idx->variant == 3 || idx->variant == 4 || (idx->variant == 0 && s >= kTcAutoMinQueries));
     if (tc) {
-        const int grid = static_cast<int>(std::min<long long>(idx->num_sms, (idx->N + kTcTileM - 1) / kTcTileM));
+        int grid = idx->N > 0 ? 1 : 0;  // set by the passes (the same for all of them)
         const int per_pass = std::min(kTcMaxQueries, idx->tc_cand_q);
         for (int q0 = 0; grid > 0 && q0 < s; q0 += per_pass) {
             const int sp = std::min(per_pass, s - q0);
@@ -229,7 +281,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
                 cudaEventRecord(ev.first, st);
             }
             const ralm_status_t rs =
-                launch_tc_pass(idx, queries + static_cast<size_t>(q0) * idx->d, sp, s, q0, k, grid, st);
+                launch_tc_pass(idx, queries + static_cast<size_t>(q0) * idx->d, sp, s, q0, k,
+                               idx->variant != 4, &grid, st);
             if (idx->timing) {
                 cudaEventRecord(ev.second, st);
                 idx->timed.push_back(ev);
@@ -256,6 +309,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             p.corpus = idx->corpus;
             p.queries = queries + static_cast<size_t>(q0) * idx->d;
             p.norms = idx->norms;
+            p.spill = pl.spill ? idx->spill : nullptr;
             p.partial = idx->partial;
             p.status = idx->status;
             p.N = idx->N;
@@ -414,8 +468,16 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     const size_t sk = static_cast<size_t>(max_s) * max_k;
     idx->tc_cand = nullptr;
     idx->tc_cand_q = 0;
+    idx->tc_clusters = -1;
     idx->norms = nullptr;
+    idx->spill = nullptr;
+    idx->spill_cap = 0;
     bool ok = cudaMalloc(&idx->partial, partial_bytes) == cudaSuccess;
+    if (max_k > 1 && std::max(512, 2 * next_pow2(max_k)) * 8 > kSmemCandBytes / kScanMaxQueries) {
+        idx->spill_cap = std::max(512, 2 * next_pow2(max_k));
+        ok = ok && cudaMalloc(&idx->spill, sizeof(uint64_t) * idx->num_sms * kScanMaxQueries *
+                                               static_cast<size_t>(idx->spill_cap)) == cudaSuccess;
+    }
     if (metric == RALM_L2 && N > 0) ok = ok && cudaMalloc(&idx->norms, sizeof(float) * N) == cudaSuccess;
     if (metric == RALM_IP && max_s >= kTcAutoMinQueries && d >= kTcChunkK)
         ok = ok && alloc_tc_workspace(idx, std::min(kTcMaxQueries, align_up(max_s, 16)));
@@ -452,6 +514,7 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
     cudaFree(idx->cache_keys);
     cudaFree(idx->tc_cand);
     cudaFree(idx->norms);
+    cudaFree(idx->spill);
     cudaFree(idx->status);
     cudaFree(idx->h_queries);
     cudaFree(idx->h_ids);
@@ -543,9 +606,9 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream) {
 }
 
 ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant) {
-    if (!idx || variant < 0 || variant > 3) return RALM_ERR_INVALID_ARG;
+    if (!idx || variant < 0 || variant > 4) return RALM_ERR_INVALID_ARG;
     if (variant == 1 && idx->d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
-    if (variant == 3) {
+    if (variant == 3 || variant == 4) {
         if (idx->metric != RALM_IP || idx->d < kTcChunkK || !tensor_map_encoder()) return RALM_ERR_UNSUPPORTED;
         if (!alloc_tc_workspace(idx, std::min(kTcMaxQueries, align_up(idx->max_s, 16)))) return RALM_ERR_OOM;
     }
@@ -590,6 +653,9 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.cache_keys = nullptr;
     view.tc_cand = nullptr;
     view.tc_cand_q = 0;
+    view.tc_clusters = -1;
+    view.spill = nullptr;
+    view.spill_cap = 0;
     view.norms = nullptr;  // no index, no stored norms: the scan derives them on the tensor cores
     view.status = status;
     view.h_queries = nullptr;

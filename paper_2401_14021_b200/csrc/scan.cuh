@@ -42,6 +42,8 @@ struct ScanParams {
     const __half *queries;  // [s][d] of this pass
     const float *norms;     // warp-MMA L2 with NRM: squared norm of every corpus row, fp32 [N]
     uint64_t *partial;      // [gridDim.x][s_total][k] sorted keys, 0 = empty
+    uint64_t *spill;        // large k: candidate lists in global memory, [gridDim.x][8][cap]; the
+                            // shared-memory candidate area then holds one sort scratch of cap keys
     int *status;
     long long N;
     long long ntiles;
@@ -76,15 +78,25 @@ constexpr int kScanHeaderBytes = 1024;
 static_assert(sizeof(ScanHeader) <= kScanHeaderBytes, "header too large");
 
 // Sort query q's candidates, keep the best k, raise the threshold. Called by a group of
-// `nthr` threads with ranks `tid`, synchronised through group_sync(bar_id).
-__device__ inline void compact_query(ScanHeader *hdr, uint64_t *cand, int cap, int q, int k,
-                                     int tid, int nthr, int bar_id) {
-    uint64_t *a = cand + static_cast<size_t>(q) * cap;
+// `nthr` threads with ranks `tid`, synchronised through group_sync(bar_id). With a scratch
+// area the list (which then lives in global memory) is sorted there and its head copied back.
+__device__ inline void compact_query(ScanHeader *hdr, uint64_t *cand, uint64_t *scratch, int cap, int q,
+                                     int k, int tid, int nthr, int bar_id) {
+    uint64_t *list = cand + static_cast<size_t>(q) * cap;
+    uint64_t *a = scratch ? scratch : list;
     const int n = hdr->cnt[q];
     const int P = next_pow2(n > 1 ? n : 2);
-    for (int i = n + tid; i < P; i += nthr) a[i] = 0;
+    if (scratch) {
+        for (int i = tid; i < P; i += nthr) a[i] = (i < n) ? list[i] : 0ull;
+    } else {
+        for (int i = n + tid; i < P; i += nthr) a[i] = 0;
+    }
     group_sync(bar_id, nthr);
     bitonic_sort_desc(a, P, tid, nthr, bar_id);
+    if (scratch) {
+        const int keep = n < k ? n : k;
+        for (int i = tid; i < keep; i += nthr) list[i] = a[i];
+    }
     if (tid == 0) {
         hdr->cnt[q] = n < k ? n : k;
         hdr->thr[q] = (n >= k) ? key_value(a[k - 1]) : -INFINITY;
@@ -95,8 +107,8 @@ __device__ inline void compact_query(ScanHeader *hdr, uint64_t *cand, int cap, i
 // All W consumer warps (this one is w) compact every query that holds more than `min_count`
 // candidates; the queries are spread over groups of warps that sort in parallel. Must be
 // called by all W * 32 consumer threads, with no push in flight.
-__device__ inline void compact_all(ScanHeader *hdr, uint64_t *cand, int cap, int s, int k,
-                                   int min_count, int w, int lane, int W) {
+__device__ inline void compact_all(ScanHeader *hdr, uint64_t *cand, uint64_t *scratch, int cap, int s,
+                                   int k, int min_count, int w, int lane, int W) {
     int list[kScanMaxQueries];
     int nq = 0;
 #pragma unroll
@@ -105,7 +117,8 @@ __device__ inline void compact_all(ScanHeader *hdr, uint64_t *cand, int cap, int
     // nobody may start rewriting cnt[] before everybody has taken the same snapshot of it
     named_barrier(1, W * 32);
     if (nq == 0) return;
-    const int ngroups = nq < W ? nq : W;
+    // one scratch area: one group, the queries one after the other
+    const int ngroups = scratch ? 1 : (nq < W ? nq : W);
     const int G = W / ngroups;  // warps per group
     const int group = w / G;
     if (group >= ngroups) return;
@@ -116,16 +129,16 @@ __device__ inline void compact_all(ScanHeader *hdr, uint64_t *cand, int cap, int
 #pragma unroll
         for (int j = 0; j < kScanMaxQueries; ++j)
             if (j == i) q = list[j];
-        compact_query(hdr, cand, cap, q, k, tid, G * 32, bar_id);
+        compact_query(hdr, cand, scratch, cap, q, k, tid, G * 32, bar_id);
     }
 }
 
 // The meeting itself: barrier, compact, lower the flag, barrier.
-__device__ __forceinline__ void compaction_meeting(ScanHeader *hdr, uint64_t *cand,
+__device__ __forceinline__ void compaction_meeting(ScanHeader *hdr, uint64_t *cand, uint64_t *scratch,
                                                    const int cap, const int s, const int k, int w,
                                                    int lane, int W) {
     named_barrier(1, W * 32);
-    compact_all(hdr, cand, cap, s, k, k, w, lane, W);
+    compact_all(hdr, cand, scratch, cap, s, k, k, w, lane, W);
     if (w == 0 && lane == 0) *reinterpret_cast<volatile int *>(&hdr->flag) = 0;
     named_barrier(1, W * 32);
 }
@@ -179,14 +192,13 @@ __device__ __forceinline__ void push_candidate(ScanHeader *hdr, uint64_t *cand, 
 }
 
 
-// Warp-MMA L2 flavour, exact part: squared distance between one corpus row (read back from
-// global memory; the tile it came with has just passed through L2) and one query (fp16 in
-// shared memory), computed by the whole warp in the direct sum-of-squared-differences form
-// (no cancellation). Every lane returns the full sum.
-__device__ __forceinline__ float warp_direct_l2(const __half *row, uint32_t q_addr, int d, int lane) {
+// Warp-MMA L2 flavour, exact part: squared distance between one staged corpus row and one
+// query (both fp16 in shared memory), computed by the whole warp in the direct
+// sum-of-squared-differences form (no cancellation). Every lane returns the full sum.
+__device__ __forceinline__ float warp_direct_l2(uint32_t row_addr, uint32_t q_addr, int d, int lane) {
     float2 sum = make_float2(0.f, 0.f);
     for (int piece = lane; piece * 8 < d; piece += 32) {
-        const uint4 xr = __ldg(reinterpret_cast<const uint4 *>(row) + piece);
+        const uint4 xr = lds128(row_addr + piece * 16);
         const uint4 qr = lds128(q_addr + piece * 16);
         const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
         const uint32_t qw[4] = {qr.x, qr.y, qr.z, qr.w};
@@ -215,7 +227,9 @@ __global__ void __launch_bounds__(MMA ? kScanThreads : kScanThreads - 32, 1)
 scan_kernel(const ScanParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     ScanHeader *hdr = reinterpret_cast<ScanHeader *>(smem);
-    uint64_t *cand = reinterpret_cast<uint64_t *>(smem + p.off_cand);
+    uint64_t *scratch = p.spill ? reinterpret_cast<uint64_t *>(smem + p.off_cand) : nullptr;
+    uint64_t *cand = p.spill ? p.spill + static_cast<size_t>(blockIdx.x) * kScanMaxQueries * p.cap
+                             : reinterpret_cast<uint64_t *>(smem + p.off_cand);
     const int W = p.nwarps;
     const int S = W * p.depth;
     const int T = p.tile_rows;
@@ -396,7 +410,7 @@ scan_kernel(const ScanParams p) {
                         while (!mbar_try_wait(full_bar, my_parity)) {}  // completed: returns at once
                         have_tile = true;
                     } else if (state == 2) {
-                        compaction_meeting(hdr, cand, p.cap, p.s, p.k, w, lane, W);
+                        compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W);
                     } else if (state == 3) {
                         if (lane == 0) {
                             atomicMax(p.status, kStatusTimeout);
@@ -444,8 +458,10 @@ scan_kernel(const ScanParams p) {
                 }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[i] += acc_b[i];
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar);
+                if (!L2) {  // the L2 flavour still needs the rows: it hands the stage back below
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_bar);
+                }
                 // acc[0]: (row g, query 2t)     acc[1]: (row g, query 2t+1)
                 // acc[2]: (row g+8, query 2t)   acc[3]: (row g+8, query 2t+1)
                 const long long r_lo = row0 + g, r_hi = row0 + g + 8;
@@ -488,7 +504,7 @@ scan_kernel(const ScanParams p) {
                             m &= m - 1;
                             const int row_local = (src >> 2) + ((i & 2) ? 8 : 0);
                             const int q = 2 * (src & 3) + (i & 1);
-                            const float dist = warp_direct_l2(p.corpus + (row0 + row_local) * d,
+                            const float dist = warp_direct_l2(stage_addr + row_local * d * 2,
                                                               q_base_addr + q * q_pitch, d, lane);
                             if (lane == 0) {
                                 const float val = 0.0f - dist;
@@ -501,6 +517,8 @@ scan_kernel(const ScanParams p) {
                             }
                         }
                     }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_bar);
                 } else {
                 if (TOP1) {
                     if (r_lo < p.N) {
@@ -631,11 +649,11 @@ scan_kernel(const ScanParams p) {
                     }
                 }
                 state = __shfl_sync(0xffffffffu, state, 0);
-                if (state == 1) compaction_meeting(hdr, cand, p.cap, p.s, p.k, w, lane, W);
+                if (state == 1) compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W);
                 else if (state == 2) break;
             }
             named_barrier(1, cthreads);
-            compact_all(hdr, cand, p.cap, p.s, p.k, 0, w, lane, W);
+            compact_all(hdr, cand, scratch, p.cap, p.s, p.k, 0, w, lane, W);
             named_barrier(1, cthreads);
             for (int q = 0; q < p.s; ++q) {
                 const int n = hdr->cnt[q];

@@ -17,8 +17,13 @@
 //               candidate list in global memory. Lists are compacted (sorted, cut to k,
 //               threshold raised) by the same warps between units, before they can overflow.
 //
+// The kernel is bound by the bytes it stages per MMA, so by default it runs as clusters of two
+// CTAs (cta_group::2): a row tile is then 256 rows, each CTA stages its own 128 rows but only
+// half of the queries of a chunk, the pair's leader issues one M = 256 MMA for both, and each
+// CTA selects from the 128 rows that land in its own TMEM. No load is multicast.
+//
 // Every wait is bounded; when one runs out the CTA records kStatusTimeout, lets copies and
-// MMAs in flight finish, frees its TMEM and returns.
+// MMAs in flight finish, frees its TMEM and returns (a pair leaves through a cluster barrier).
 #pragma once
 
 #include <cuda.h>
@@ -50,10 +55,11 @@ struct TcParams {
     int s_total;
     int q_base;
     int k;
-    int nb;             // query rows per stage = rows of the query TMA box (16..256, multiple of 16)
+    int nb;             // queries per accumulator (16..256; a multiple of 16, of 32 for CTA pairs);
+                        // a CTA stages nb query rows per chunk, nb / 2 in a pair
     int nhalves;        // ceil(s / nb): 1 or 2
     int stages;
-    int stage_bytes;    // kTcABytes + nb * 128, a multiple of 1024
+    int stage_bytes;    // kTcABytes + (staged query rows) * 128, a multiple of 1024
     int off_stage;      // shared-memory offset of the stage ring (1024-byte aligned)
     int cand_q;         // queries the candidate workspace was sized for (>= s)
 };
@@ -116,9 +122,9 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr) {
     desc |= static_cast<uint64_t>(2) << 61;         // 128-byte swizzle
     return desc;
 }
-// Instruction descriptor: fp16 A and B (both K-major), fp32 accumulator, M = 128, N = n.
-__device__ __forceinline__ uint32_t tc_idesc(int n) {
-    return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTcTileM >> 4) << 24);
+// Instruction descriptor: fp16 A and B (both K-major), fp32 accumulator, M = m, N = n.
+__device__ __forceinline__ uint32_t tc_idesc(int n, int m) {
+    return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
 // 32 consecutive columns of this thread's TMEM lane, then wait for the load.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
@@ -154,6 +160,56 @@ __device__ inline void tc_compact_query(uint64_t *list, uint64_t *scratch, float
     __syncwarp();
 }
 
+// ---- CTA-pair helpers (PAIR = true: two CTAs of a cluster work as one MMA unit) -----------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Tile load whose completion is signalled on an mbarrier that may live in the other CTA of the pair.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int x, int y,
+                                                 uint32_t cluster_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(cluster_bar)
+        : "memory");
+}
+// Arrive on the barrier at this offset in both CTAs of the pair once the MMAs issued so far are done.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+        "h"(static_cast<uint16_t>(3))
+        : "memory");
+}
+__device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                                uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// PAIR = false: every CTA is on its own (M = 128 rows per MMA).
+// PAIR = true: clusters of two CTAs. A row tile is 256 rows; CTA r of the pair stages rows
+// 128 r .. 128 r + 127 and half of the query rows of each K chunk, the leader (rank 0) issues
+// one M = 256 MMA for both, and each CTA finds the scores of its own 128 rows in its own
+// TMEM. Per CTA and chunk this stages 16 KB + nb/2 query rows instead of 16 KB + nb.
+template <bool PAIR>
 __global__ void __launch_bounds__(kTcThreads, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_q,
                const TcParams p) {
@@ -165,6 +221,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int S = p.stages;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // 0 = leader of the pair
+    const bool leader = rank == 0;
+    const int group = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+    const int ngroups = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
+    constexpr int kGroupRows = PAIR ? 2 * kTcTileM : kTcTileM;
+    const int nb_cta = PAIR ? p.nb / 2 : p.nb;             // query rows this CTA stages per chunk
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < S; ++i) {
@@ -173,7 +235,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&hdr->tmem_full[i]), 1);
-            mbar_init(smem_u32(&hdr->tmem_empty[i]), 4);  // one arrival per selection warp
+            // one arrival per selection warp (of both CTAs for a pair)
+            mbar_init(smem_u32(&hdr->tmem_empty[i]), PAIR ? 8 : 4);
         }
         mbar_init(smem_u32(&hdr->drain), 1);
         mbar_fence_init();
@@ -186,19 +249,27 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         sorted[q] = 0;
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                         smem_u32(&hdr->tmem_base)),
-                     "r"(kTcTmemCols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                             smem_u32(&hdr->tmem_base)),
+                         "r"(kTcTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                             smem_u32(&hdr->tmem_base)),
+                         "r"(kTcTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_barrier();  // the partner's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&hdr->tmem_base);
 
-    const long long my_tiles =
-        (p.ntiles > blockIdx.x) ? (p.ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+    const long long my_tiles = (p.ntiles > group) ? (p.ntiles - group + ngroups - 1) / ngroups : 0;
     const long long my_units = my_tiles * p.nhalves;
     volatile int *abort_flag = &hdr->abort;
     const uint32_t stage_base = smem_u32(tc_smem + p.off_stage);
@@ -206,14 +277,21 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
         if (lane == 0) {
-            const uint32_t stage_tx = static_cast<uint32_t>(kTcABytes + p.nb * 128);
+            // bytes that land per stage and phase on the barrier the MMA thread waits on: a
+            // pair's loads all report to the leader's barrier
+            const uint32_t stage_tx = static_cast<uint32_t>(kTcABytes + nb_cta * 128) * (PAIR ? 2u : 1u);
             int st = 0;
             uint32_t lap = 0;
             long long issued = 0;
             bool ok = true, stop = false;
             for (long long u = 0; u < my_units && !stop; ++u) {
-                const long long tile = blockIdx.x + (u / p.nhalves) * gridDim.x;
+                const long long tile = group + (u / p.nhalves) * ngroups;
                 const int half = static_cast<int>(u % p.nhalves);
+                const int row_y = static_cast<int>(tile * kGroupRows + rank * kTcTileM);
+                // a pair splits the N of this unit's MMA, not nb: the follower supplies the upper
+                // half of the (rounded) queries this half really has
+                const int nq_u = (p.s - half * p.nb < p.nb) ? (p.s - half * p.nb) : p.nb;
+                const int query_y = half * p.nb + (PAIR ? static_cast<int>(rank) * (((nq_u + 31) & ~31) / 2) : 0);
                 for (int c = 0; c < p.nchunks; ++c) {
                     ok = mbar_wait_bounded(smem_u32(&hdr->empty[st]), (lap & 1) ^ 1);
                     if (!ok || *abort_flag) {
@@ -222,9 +300,16 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     }
                     const uint32_t bar = smem_u32(&hdr->full[st]);
                     const uint32_t dst = stage_base + static_cast<uint32_t>(st) * p.stage_bytes;
-                    mbar_arrive_expect_tx(bar, stage_tx);
-                    tma_load_2d(dst, &map_x, c * kTcChunkK, static_cast<int>(tile * kTcTileM), bar);
-                    tma_load_2d(dst + kTcABytes, &map_q, c * kTcChunkK, half * p.nb, bar);
+                    if (PAIR) {
+                        const uint32_t lead_bar = map_to_cta(bar, 0);
+                        if (leader) mbar_arrive_expect_tx(bar, stage_tx);
+                        tma_load_2d_pair(dst, &map_x, c * kTcChunkK, row_y, lead_bar);
+                        tma_load_2d_pair(dst + kTcABytes, &map_q, c * kTcChunkK, query_y, lead_bar);
+                    } else {
+                        mbar_arrive_expect_tx(bar, stage_tx);
+                        tma_load_2d(dst, &map_x, c * kTcChunkK, row_y, bar);
+                        tma_load_2d(dst + kTcABytes, &map_q, c * kTcChunkK, query_y, bar);
+                    }
                     ++issued;
                     if (++st == S) {
                         st = 0;
@@ -236,8 +321,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 atomicMax(p.status, kStatusTimeout);
                 *abort_flag = 1;
             }
-            if (*abort_flag) {
-                // winding down early: let every copy already issued land before exit
+            if (*abort_flag && (!PAIR || leader)) {
+                // winding down early: let every copy already issued land before exit (a pair's
+                // follower cannot watch the leader's barrier; its copies land in its own shared
+                // memory, which stays allocated until both CTAs have passed the final barrier,
+                // and a wait has already run out by then)
                 const long long first = issued > S ? issued - S : 0;
                 for (long long it = first; it < issued; ++it)
                     mbar_wait_bounded(smem_u32(&hdr->full[it % S]), static_cast<uint32_t>((it / S) & 1));
@@ -245,7 +333,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (lane == 0 && leader) {
             int st = 0;
             uint32_t lap = 0;
             bool ok = true;
@@ -253,7 +341,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const int half = static_cast<int>(u % p.nhalves);
                 const int acc = static_cast<int>(u & 1);
                 const int nq = (p.s - half * p.nb < p.nb) ? (p.s - half * p.nb) : p.nb;
-                const uint32_t idesc = tc_idesc((nq + 15) & ~15);
+                const int n_mma = PAIR ? ((nq + 31) & ~31) : ((nq + 15) & ~15);
+                const uint32_t idesc = tc_idesc(n_mma, kGroupRows);
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kTcMaxN);
                 // the selection warps must have drained this accumulator's previous unit
                 ok = mbar_wait_bounded(smem_u32(&hdr->tmem_empty[acc]), static_cast<uint32_t>(((u >> 1) & 1) ^ 1));
@@ -266,24 +355,33 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     const uint32_t a_addr = stage_base + static_cast<uint32_t>(st) * p.stage_bytes;
                     const uint32_t b_addr = a_addr + kTcABytes;
 #pragma unroll
-                    for (int kk = 0; kk < kTcChunkK / 16; ++kk)
-                        tc_mma_f16(d_tmem, tc_smem_desc(a_addr + kk * 32), tc_smem_desc(b_addr + kk * 32),
-                                   idesc, (c | kk) != 0 ? 1u : 0u);
-                    tc_commit(smem_u32(&hdr->empty[st]));  // stage reusable once these MMAs are done
+                    for (int kk = 0; kk < kTcChunkK / 16; ++kk) {
+                        if (PAIR)
+                            tc_mma_f16_pair(d_tmem, tc_smem_desc(a_addr + kk * 32), tc_smem_desc(b_addr + kk * 32),
+                                            idesc, (c | kk) != 0 ? 1u : 0u);
+                        else
+                            tc_mma_f16(d_tmem, tc_smem_desc(a_addr + kk * 32), tc_smem_desc(b_addr + kk * 32),
+                                       idesc, (c | kk) != 0 ? 1u : 0u);
+                    }
+                    // stage reusable (in both CTAs of a pair) once these MMAs are done
+                    if (PAIR) tc_commit_pair(smem_u32(&hdr->empty[st]));
+                    else tc_commit(smem_u32(&hdr->empty[st]));
                     if (++st == S) {
                         st = 0;
                         ++lap;
                     }
                 }
                 if (!ok || *abort_flag) break;
-                tc_commit(smem_u32(&hdr->tmem_full[acc]));
+                if (PAIR) tc_commit_pair(smem_u32(&hdr->tmem_full[acc]));
+                else tc_commit(smem_u32(&hdr->tmem_full[acc]));
             }
             if (!ok && !*abort_flag) {
                 atomicMax(p.status, kStatusTimeout);
                 *abort_flag = 1;
             }
             // every MMA issued above must have completed before the TMEM is given back
-            tc_commit(smem_u32(&hdr->drain));
+            if (PAIR) tc_commit_pair(smem_u32(&hdr->drain));
+            else tc_commit(smem_u32(&hdr->drain));
             mbar_wait_bounded(smem_u32(&hdr->drain), 0);
         }
     } else {
@@ -295,7 +393,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         volatile int *dirty = &hdr->dirty;
         bool ok = true;
         for (long long u = 0; u < my_units; ++u) {
-            const long long tile = blockIdx.x + (u / p.nhalves) * gridDim.x;
+            const long long tile = group + (u / p.nhalves) * ngroups;
             const int half = static_cast<int>(u % p.nhalves);
             const int acc = static_cast<int>(u & 1);
             const int qb = half * p.nb;
@@ -316,7 +414,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             const bool live = ok && !*abort_flag;
             if (live) {
                 tc_fence_after();
-                const long long row = tile * kTcTileM + quarter * 32 + lane;
+                const long long row = tile * kGroupRows + rank * kTcTileM + quarter * 32 + lane;
                 const bool row_ok = row < p.N;
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                        static_cast<uint32_t>(acc * kTcMaxN);
@@ -346,10 +444,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         }
                     }
                 }
-                // accumulator drained: hand it back to the MMA warp
+                // accumulator drained: hand it back to the MMA thread (the pair's leader)
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&hdr->tmem_empty[acc]));
+                if (lane == 0) {
+                    if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&hdr->tmem_empty[acc]), 0));
+                    else mbar_arrive(smem_u32(&hdr->tmem_empty[acc]));
+                }
             }
             // All four warps meet after every unit (also when winding down, so that nobody is
             // left waiting): first so that every push of the unit is visible, then, having all
@@ -389,10 +490,17 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 
     tc_fence_before();
     __syncthreads();
+    // a pair leaves together: the leader's MMAs read the follower's shared memory and its
+    // commits arrive on the follower's barriers
+    if (PAIR) cluster_barrier();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTcTmemCols)
-                     : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTcTmemCols)
+                         : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTcTmemCols)
+                         : "memory");
     }
 }
 

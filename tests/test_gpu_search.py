@@ -37,7 +37,7 @@ VARIANTS = {oracle.IP: (2, 1), oracle.L2: (2, 1)}
 @pytest.mark.parametrize("N,d,s,k", [(1, 8, 1, 1), (15, 8, 3, 4), (16, 16, 8, 1), (17, 64, 5, 20),
                                      (33, 40, 2, 40), (1000, 72, 8, 7), (5000, 768, 4, 5),
                                      (3001, 1024, 4, 1024), (257, 264, 9, 3), (64, 8, 17, 64),
-                                     (700, 2048, 3, 9)])
+                                     (700, 2048, 3, 9), (9000, 128, 8, 1024), (5000, 64, 7, 300)])
 def test_integer_inputs_are_bit_exact(metric, N, d, s, k):
     """Small-integer rows: every score is an integer that fp32 holds exactly, and ties abound,
     so ids (tie-break included) and scores must equal the oracle's bit for bit."""
@@ -179,14 +179,16 @@ def test_argument_errors():
 # ------------------------------------------------------------------ large batches (tcgen05 scan)
 @pytest.mark.parametrize("N,d,s,k", [(1, 64, 1, 1), (129, 72, 3, 1), (300, 128, 9, 64), (1000, 64, 16, 5),
                                      (5000, 768, 100, 20), (257, 64, 257, 2), (3000, 256, 600, 7),
+                                     (2000, 128, 300, 5), (700, 64, 40, 3),
                                      (40_000, 768, 512, 20)])
 def test_tcgen05_scan_integer_inputs_are_bit_exact(N, d, s, k):
     """The large-batch scan pinned explicitly (variant 3), including shapes with a ragged last
     K chunk (d % 64 != 0), a ragged row tile, a second query half and a second pass."""
     x = workloads.integer_valued((N, d), seed=400 + N, lo=-3, hi=3, device=DEV)
     q = workloads.integer_valued((s, d), seed=500 + N, lo=-3, hi=3, device=DEV)
-    ids, scores = _run(x, q, oracle.IP, k, 3)
-    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+    for variant in (3, 4):                 # CTA pairs, single CTAs
+        ids, scores = _run(x, q, oracle.IP, k, variant)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
 
 
 @pytest.mark.parametrize("N,d,s,k", [(100_003, 768, 300, 20), (250_000, 128, 64, 1), (20_000, 1024, 512, 33)])
@@ -200,6 +202,9 @@ def test_tcgen05_scan_parity(N, d, s, k):
     ids8, scores8 = _run(x, q, oracle.IP, k, 2)          # the 8-queries-per-pass scan on the same batch
     assert torch.equal(ids[:, 0], ids8[:, 0])
     torch.testing.assert_close(scores, scores8, rtol=1e-4, atol=1e-5)
+    ids1, scores1 = _run(x, q, oracle.IP, k, 4)          # single CTAs instead of pairs
+    assert torch.equal(ids1[:, 0], ids[:, 0])
+    torch.testing.assert_close(scores1, scores, rtol=1e-5, atol=1e-6)
 
 
 def test_tcgen05_scan_adversarial_row_order():
@@ -210,8 +215,9 @@ def test_tcgen05_scan_adversarial_row_order():
     x[:, 0] = (torch.arange(N, device=DEV) // 16).to(torch.float16)
     q = torch.zeros((12, d), dtype=torch.float16, device=DEV)
     q[:, 0] = torch.tensor([1, -1, 2, -2, 1, 1, -1, 3, 0, 1, -3, 2], dtype=torch.float16)
-    ids, scores = _run(x, q, oracle.IP, 64, 3)
-    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 64, exact=True)
+    for variant in (3, 4):
+        ids, scores = _run(x, q, oracle.IP, 64, variant)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 64, exact=True)
 
 
 def test_large_k_falls_back_from_the_tcgen05_scan():
