@@ -159,6 +159,28 @@ ralm_status_t ralm_verify(const int64_t *speculated_ids, const int64_t *retrieve
                           int32_t stride, int32_t ld, int32_t cmp_k, int32_t *first_mismatch,
                           void *stream);
 
+/* Cache update after a verification step (Section 3, "Speculative retrieval": the local cache is
+ * populated with the documents retrieved during verification, the top-ranked one per query or
+ * the first `top` of them (top-k update, prefetching; Fig. 3); Section 5.3: for KNN-LM the next n
+ * entries after each retrieved item go in instead of the items themselves).
+ * Request r's cache is a set of corpus ids in C slots (-1 = empty) used as a ring: a new id is
+ * written at cursor[r], which then advances modulo C, so a full cache drops its oldest entry
+ * (the paper does not name an eviction rule; first-in first-out is this library's). For request r,
+ * in this order: steps i = 0 .. steps[r]-1, ranks j = 0 .. top-1, id = retrieved_ids[r][i][j]
+ * (negative ids are skipped); candidates are id itself (next_n == 0) or id+1 .. id+next_n
+ * (next_n > 0), cut at N; a candidate already in the cache is skipped, any other is inserted.
+ *   cache_ids     DEVICE int64 [R][C] (read and written)   1 <= C <= RALM_MAX_CACHE
+ *   cursor        DEVICE int32 [R] (read and written), values in [0, C)
+ *   retrieved_ids DEVICE int64 [R][stride][ld], 1 <= top <= ld
+ *   steps         DEVICE int32 [R] or NULL (= stride for every request); values are clamped to
+ *                 [0, stride]. Passing min(first_mismatch + 1, stride) inserts what was confirmed
+ *                 plus the correcting document.
+ *   N             number of corpus rows (candidates >= N are never inserted)
+ * Needs no index. Asynchronous on `stream`. R == 0 or stride == 0 are no-ops. */
+ralm_status_t ralm_cache_update(int64_t *cache_ids, int32_t *cursor, int32_t R, int32_t C,
+                                const int64_t *retrieved_ids, int32_t stride, int32_t ld, int32_t top,
+                                const int32_t *steps, int32_t next_n, int64_t N, void *stream);
+
 /* Synchronise `stream`, read and clear the index's sticky device status word. Returns
  * RALM_OK, RALM_ERR_TIMEOUT, RALM_ERR_BAD_CACHE_ID, or RALM_ERR_CUDA if the stream itself
  * reports an error. */
@@ -190,6 +212,31 @@ ralm_status_t ralm_index_set_timing(ralm_index_t *idx, int32_t enabled);
 /* Wait for the scan launches timed since the last read, return the sum of their durations in
  * milliseconds and how many there were, and forget them. HOST pointers. */
 ralm_status_t ralm_index_read_timing(ralm_index_t *idx, double *total_ms, int64_t *launches);
+
+/* ---- Optimal speculation stride scheduler (OS^3): host arithmetic, no device work ---------
+ * Section 4 ("Optimal speculation stride scheduler") and Appendix A.2. `a` is the latency of one
+ * speculation step, `b` of one verification step (any one unit, e.g. the milliseconds that CUDA
+ * events around ralm_cache_search and ralm_search report), gamma the probability that one
+ * speculated document matches.
+ *
+ * ralm_os3_expected_verified: (1 - gamma^s) / (1 - gamma), the expected number of documents one
+ *   verification step of stride s confirms (Appendix A.2); s for gamma = 1, 0 for s <= 0.
+ * ralm_os3_objective: expected verified documents per unit time for stride s. Synchronous
+ *   verification: latency s a + b. Asynchronous (async_verify != 0): with probability gamma^s
+ *   the latency is (s - 1) a + max(a, b), otherwise s a + b.
+ * ralm_os3_gamma: the windowed estimate sum(M) / (sum(M) + #{t : M(t) < s(t)}) over the last w
+ *   verification steps, truncated at gamma_max (the evaluation uses w = 5, gamma_max = 0.6).
+ *   matched[t] = the first_mismatch value ralm_verify returned for a step of stride strides[t]
+ *   (HOST arrays, 0 <= matched[t] <= strides[t], strides[t] >= 1). No history (w = 0) gives 0.
+ * ralm_os3_stride: the stride in 1..s_max that maximises the objective for the estimated gamma
+ *   (the smaller stride on ties). With no history this is 1, where the scheduler starts.
+ * Errors: INVALID_ARG for null pointers, negative latencies, values out of the stated ranges. */
+double ralm_os3_expected_verified(double gamma, int32_t s);
+double ralm_os3_objective(double gamma, double a, double b, int32_t s, int32_t async_verify);
+ralm_status_t ralm_os3_gamma(const int32_t *matched, const int32_t *strides, int32_t w, double gamma_max,
+                             double *gamma_out);
+ralm_status_t ralm_os3_stride(const int32_t *matched, const int32_t *strides, int32_t w, double gamma_max,
+                              double a, double b, int32_t s_max, int32_t async_verify, int32_t *s_out);
 
 /* Static description of a status code. */
 const char *ralm_status_string(ralm_status_t status);

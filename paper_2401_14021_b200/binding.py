@@ -50,6 +50,8 @@ def load_library() -> ctypes.CDLL:
     lib.ralm_cache_search.argtypes = [p, p, i32, i32, p, i32, i32, p, p, p]
     lib.ralm_verify.restype = i32
     lib.ralm_verify.argtypes = [p, p, i32, i32, i32, i32, p, p]
+    lib.ralm_cache_update.restype = i32
+    lib.ralm_cache_update.argtypes = [p, p, i32, i32, p, i32, i32, i32, p, i32, i64, p]
     lib.ralm_device_status.restype = i32
     lib.ralm_device_status.argtypes = [p, p]
     lib.ralm_index_set_variant.restype = i32
@@ -62,6 +64,16 @@ def load_library() -> ctypes.CDLL:
     lib.ralm_index_set_timing.argtypes = [p, i32]
     lib.ralm_index_read_timing.restype = i32
     lib.ralm_index_read_timing.argtypes = [p, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
+    f64 = ctypes.c_double
+    lib.ralm_os3_expected_verified.restype = f64
+    lib.ralm_os3_expected_verified.argtypes = [f64, i32]
+    lib.ralm_os3_objective.restype = f64
+    lib.ralm_os3_objective.argtypes = [f64, f64, f64, i32, i32]
+    lib.ralm_os3_gamma.restype = i32
+    lib.ralm_os3_gamma.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(i32), i32, f64, ctypes.POINTER(f64)]
+    lib.ralm_os3_stride.restype = i32
+    lib.ralm_os3_stride.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(i32), i32, f64, f64, f64, i32, i32,
+                                    ctypes.POINTER(i32)]
     lib.ralm_status_string.restype = ctypes.c_char_p
     lib.ralm_status_string.argtypes = [i32]
     _lib = lib
@@ -219,3 +231,48 @@ def verify(speculated_ids: torch.Tensor, retrieved_ids: torch.Tensor, cmp_k: int
     fp = _dev(first_mismatch, torch.int32, "first_mismatch") if R else 0
     _check(_lib.ralm_verify(sp, rp, R, stride, ld, cmp_k, fp, _stream_ptr(stream)), "ralm_verify")
     return first_mismatch
+
+
+def cache_update(cache_ids: torch.Tensor, cursor: torch.Tensor, retrieved_ids: torch.Tensor, top: int,
+                 N: int, steps: torch.Tensor = None, next_n: int = 0, stream=None):
+    """ralm_cache_update: insert the ids retrieved by a verification step into the requests' caches
+    (in place). cache_ids int64 [R][C], cursor int32 [R], retrieved_ids int64 [R][stride][ld],
+    steps int32 [R] or None."""
+    lib = load_library()
+    R, C = cache_ids.shape
+    stride, ld = retrieved_ids.shape[1], retrieved_ids.shape[2]
+    _check(lib.ralm_cache_update(_dev(cache_ids, torch.int64, "cache_ids") if R else 0,
+                                 _dev(cursor, torch.int32, "cursor") if R else 0, R, C,
+                                 _dev(retrieved_ids, torch.int64, "retrieved_ids") if retrieved_ids.numel() else 0,
+                                 stride, ld, top, _dev(steps, torch.int32, "steps") if steps is not None else 0,
+                                 next_n, N, _stream_ptr(stream)), "ralm_cache_update")
+    return cache_ids, cursor
+
+
+def _i32_array(values):
+    values = [int(v) for v in values]
+    return (ctypes.c_int32 * max(len(values), 1))(*values), len(values)
+
+
+def os3_gamma(matched, strides, gamma_max: float = 0.6) -> float:
+    """ralm_os3_gamma: windowed estimate of the speculation accuracy from the first_mismatch values
+    (`matched`) and strides of the most recent verification steps."""
+    lib = load_library()
+    m, w = _i32_array(matched)
+    s, _ = _i32_array(strides)
+    out = ctypes.c_double()
+    _check(lib.ralm_os3_gamma(m, s, w, gamma_max, ctypes.byref(out)), "ralm_os3_gamma")
+    return out.value
+
+
+def os3_stride(matched, strides, a: float, b: float, s_max: int = 16, async_verify: bool = False,
+               gamma_max: float = 0.6) -> int:
+    """ralm_os3_stride: the speculation stride in 1..s_max that maximises the expected number of
+    verified documents per unit time, given speculation-step latency a and verification latency b."""
+    lib = load_library()
+    m, w = _i32_array(matched)
+    s, _ = _i32_array(strides)
+    out = ctypes.c_int32()
+    _check(lib.ralm_os3_stride(m, s, w, gamma_max, a, b, s_max, int(async_verify), ctypes.byref(out)),
+           "ralm_os3_stride")
+    return out.value

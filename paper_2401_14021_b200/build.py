@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libralm.so")
-SOURCES = ["ralm_api.cu"]
+SOURCES = ["ralm_api.cu", "os3.cpp"]
 HEADERS = ["common.cuh", "scan.cuh", "aux_kernels.cuh", os.path.join("..", "..", "include", "ralm.h")]
 
 

@@ -188,6 +188,53 @@ cache_rank_kernel(const uint64_t *__restrict__ keys, int Cp, int k, int l2,
 }
 
 // ------------------------------------------------------------------------------------
+// Cache update after a verification step: one CTA per request. The request's slots sit in
+// shared memory; candidates are taken strictly in order (step, rank, offset), each tested
+// against all slots by the whole CTA and, if absent, written at the request's ring cursor.
+// The order is part of the result (what a full ring evicts depends on it), so the loop over
+// candidates is sequential and only the membership test is parallel.
+// ------------------------------------------------------------------------------------
+constexpr int kCacheUpdateThreads = 256;
+
+__global__ void __launch_bounds__(kCacheUpdateThreads)
+cache_update_kernel(int64_t *__restrict__ cache_ids, int *__restrict__ cursor, int C,
+                    const int64_t *__restrict__ retrieved, int stride, int ld, int top,
+                    const int *__restrict__ steps, int next_n, long long N) {
+    extern __shared__ __align__(16) unsigned char cu_smem[];
+    int64_t *slots = reinterpret_cast<int64_t *>(cu_smem);
+    const int r = blockIdx.x;
+    const int tid = threadIdx.x;
+    int64_t *mine = cache_ids + static_cast<size_t>(r) * C;
+    for (int i = tid; i < C; i += kCacheUpdateThreads) slots[i] = mine[i];
+    int cur = cursor[r] % C;
+    if (cur < 0) cur += C;
+    int n_steps = steps ? steps[r] : stride;
+    n_steps = n_steps < 0 ? 0 : (n_steps > stride ? stride : n_steps);
+    __syncthreads();
+    const int first = next_n > 0 ? 1 : 0, last = next_n > 0 ? next_n : 0;
+    for (int i = 0; i < n_steps; ++i) {
+        for (int j = 0; j < top; ++j) {
+            const long long doc = retrieved[(static_cast<size_t>(r) * stride + i) * ld + j];
+            if (doc < 0) continue;
+            for (int o = first; o <= last; ++o) {
+                const long long c = doc + o;
+                if (c >= N) break;
+                int found = 0;
+                for (int sidx = tid; sidx < C; sidx += kCacheUpdateThreads) found |= (slots[sidx] == c);
+                if (!__syncthreads_or(found)) {
+                    if (tid == 0) slots[cur] = c;
+                    cur = (cur + 1 == C) ? 0 : cur + 1;
+                    __syncthreads();
+                }
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < C; i += kCacheUpdateThreads) mine[i] = slots[i];
+    if (tid == 0) cursor[r] = cur;
+}
+
+// ------------------------------------------------------------------------------------
 // Squared norms of the corpus rows (L2 indexes, once at creation): one warp per row, fp32.
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)

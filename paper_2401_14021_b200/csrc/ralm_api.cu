@@ -592,6 +592,19 @@ ralm_status_t ralm_verify(const int64_t *speculated_ids, const int64_t *retrieve
     return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
 }
 
+ralm_status_t ralm_cache_update(int64_t *cache_ids, int32_t *cursor, int32_t R, int32_t C,
+                                const int64_t *retrieved_ids, int32_t stride, int32_t ld, int32_t top,
+                                const int32_t *steps, int32_t next_n, int64_t N, void *stream) {
+    if (R < 0 || C < 1 || C > RALM_MAX_CACHE || stride < 0 || top < 1 || ld < top || next_n < 0 || N < 0)
+        return RALM_ERR_INVALID_ARG;
+    if (R == 0 || stride == 0) return RALM_OK;
+    if (!cache_ids || !cursor || !retrieved_ids) return RALM_ERR_INVALID_ARG;
+    cache_update_kernel<<<R, kCacheUpdateThreads, static_cast<size_t>(C) * sizeof(int64_t),
+                          static_cast<cudaStream_t>(stream)>>>(cache_ids, cursor, C, retrieved_ids, stride, ld,
+                                                               top, steps, next_n, N);
+    return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
+}
+
 ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream) {
     if (!idx) return RALM_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

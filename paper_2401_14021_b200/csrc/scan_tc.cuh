@@ -40,8 +40,10 @@ constexpr int kTcMaxQueries = 2 * kTcMaxN;
 constexpr int kTcABytes = kTcTileM * kTcChunkK * 2;
 constexpr int kTcMaxStages = 12;
 constexpr int kTcCap = 256;      // candidate slots per (CTA, query)
-constexpr int kTcSoft = 128;     // a list holding this many is compacted before the next unit
-constexpr int kTcMaxK = 64;      // k <= kTcSoft / 2 keeps compactions rare
+constexpr int kTcSoft = 120;     // a list holding this many is compacted before the next unit (at most
+                                 // 128 more arrive in a unit; just under 128 so that the usual sort is
+                                 // one of 128 keys)
+constexpr int kTcMaxK = 64;      // k <= about kTcSoft / 2 keeps compactions rare
 constexpr int kTcTmemCols = 512;
 
 struct TcParams {
@@ -80,8 +82,7 @@ static_assert(sizeof(TcHeader) <= kTcHeaderBytes, "header too large");
 constexpr int kTcOffThr = kTcHeaderBytes;                      // float [512]
 constexpr int kTcOffCnt = kTcOffThr + kTcMaxQueries * 4;       // int [512]
 constexpr int kTcOffSorted = kTcOffCnt + kTcMaxQueries * 4;    // int [512]
-constexpr int kTcOffScratch = kTcOffSorted + kTcMaxQueries * 4;  // u64 [4][256]
-constexpr int kTcOffEnd = kTcOffScratch + 4 * kTcCap * 8;
+constexpr int kTcOffEnd = kTcOffSorted + kTcMaxQueries * 4;
 
 // ---- tcgen05 / TMA wrappers -------------------------------------------------------------
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
@@ -142,22 +143,76 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         : "memory");
 }
 
-// One selection warp sorts query q's candidate list (n <= 256 keys in global memory), keeps
+// Bitonic sort (descending) of 32 * E keys held by one warp in registers: key i lives in
+// x[i / 32] of lane i % 32. Exchanges at distance >= 32 stay inside a lane, the others are
+// shuffles; nothing touches memory.
+template <int E>
+__device__ __forceinline__ void warp_sort_desc(uint64_t (&x)[E], int lane) {
+#pragma unroll
+    for (int size = 2; size <= 32 * E; size <<= 1) {
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            if (stride >= 32) {
+                const int es = stride >> 5;
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    if ((e & es) == 0) {
+                        const bool desc = ((e << 5) & size) == 0;
+                        const uint64_t a = x[e], b = x[e | es];
+                        const bool swap = desc ? (a < b) : (a > b);
+                        x[e] = swap ? b : a;
+                        x[e | es] = swap ? a : b;
+                    }
+                }
+            } else {
+                const bool lower = (lane & stride) == 0;
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    const bool desc = (((e << 5) | lane) & size) == 0;
+                    const uint64_t other = __shfl_xor_sync(0xffffffffu, x[e], stride);
+                    const bool keep_max = lower == desc;
+                    const bool mine_larger = x[e] > other;
+                    x[e] = (keep_max == mine_larger) ? x[e] : other;
+                }
+            }
+        }
+    }
+}
+
+// One selection warp sorts query q's candidate list (n <= 32 * E keys in global memory), keeps
 // the best k there, raises the threshold.
-__device__ inline void tc_compact_query(uint64_t *list, uint64_t *scratch, float *thr, int *cnt,
-                                        int *sorted, int q, int k, int lane) {
-    const int n = cnt[q];
-    for (int i = lane; i < kTcCap; i += 32) scratch[i] = (i < n) ? list[i] : 0ull;
-    __syncwarp();
-    bitonic_sort_desc(scratch, kTcCap, lane, 32, -2);
+template <int E>
+__device__ __forceinline__ void tc_compact_sorted(uint64_t *list, float *thr, int *cnt, int *sorted, int q,
+                                                  int n, int k, int lane) {
+    uint64_t x[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) x[e] = (e * 32 + lane < n) ? list[e * 32 + lane] : 0ull;
+    warp_sort_desc<E>(x, lane);
     const int keep = n < k ? n : k;
-    for (int i = lane; i < keep; i += 32) list[i] = scratch[i];
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (e * 32 + lane < keep) list[e * 32 + lane] = x[e];
+    // the k-th best key sits in x[(k - 1) / 32] of lane (k - 1) % 32
+    uint64_t kth = 0;
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (e == ((k - 1) >> 5)) kth = x[e];
+    kth = __shfl_sync(0xffffffffu, kth, (k - 1) & 31);
     if (lane == 0) {
         cnt[q] = keep;
         sorted[q] = keep;
-        thr[q] = (n >= k) ? key_value(scratch[k - 1]) : -INFINITY;
+        thr[q] = (n >= k) ? key_value(kth) : -INFINITY;
     }
     __syncwarp();
+}
+
+__device__ __forceinline__ void tc_compact_query(uint64_t *list, float *thr, int *cnt, int *sorted, int q,
+                                                 int k, int lane) {
+    const int n = cnt[q];
+    if (n <= 32) tc_compact_sorted<1>(list, thr, cnt, sorted, q, n, k, lane);
+    else if (n <= 64) tc_compact_sorted<2>(list, thr, cnt, sorted, q, n, k, lane);
+    else if (n <= 128) tc_compact_sorted<4>(list, thr, cnt, sorted, q, n, k, lane);
+    else tc_compact_sorted<8>(list, thr, cnt, sorted, q, n, k, lane);
 }
 
 // ---- CTA-pair helpers (PAIR = true: two CTAs of a cluster work as one MMA unit) -----------
@@ -389,7 +444,6 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const int ew = warp - 2;        // 0..3
         const int quarter = warp & 3;   // the TMEM lanes this warp may read: 32 * quarter ..
         uint64_t *my_cand = p.cand + static_cast<size_t>(blockIdx.x) * p.cand_q * kTcCap;
-        uint64_t *scratch = reinterpret_cast<uint64_t *>(tc_smem + kTcOffScratch) + ew * kTcCap;
         volatile int *dirty = &hdr->dirty;
         bool ok = true;
         for (long long u = 0; u < my_units; ++u) {
@@ -431,15 +485,37 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         hit |= (__uint_as_float(v[4 * i + 2]) >= th.z ? 1u : 0u) << (4 * i + 2);
                         hit |= (__uint_as_float(v[4 * i + 3]) >= th.w ? 1u : 0u) << (4 * i + 3);
                     }
-                    if (row_ok && hit) {
+                    if (!row_ok) hit = 0;
+                    // Rows that pass are appended by the warp as a whole: lane L learns which rows
+                    // pass column L (one ballot per column that has any), reserves that many slots
+                    // of query L's list with ONE atomic instruction (32 different lists), and
+                    // every passing row then stores its key at its rank within the reservation.
+                    const uint32_t any_col = __reduce_or_sync(0xffffffffu, hit);
+                    if (any_col) {
+                        uint32_t mine = 0;
 #pragma unroll
                         for (int b = 0; b < 32; ++b) {
-                            if (hit & (1u << b)) {
-                                const int q = qb + j * 32 + b;
-                                const int slot = atomicAdd(&cnt[q], 1);
-                                my_cand[static_cast<size_t>(q) * kTcCap + slot] =
-                                    make_key(__uint_as_float(v[b]), static_cast<uint32_t>(row));
-                                if (slot + 1 >= kTcSoft) *dirty = 1;
+                            if (any_col & (1u << b)) {
+                                const uint32_t m = __ballot_sync(0xffffffffu, (hit >> b) & 1u);
+                                if (lane == b) mine = m;
+                            }
+                        }
+                        int base = 0;
+                        if (mine) {
+                            base = atomicAdd(&cnt[qb + j * 32 + lane], __popc(mine));
+                            if (base + __popc(mine) >= kTcSoft) *dirty = 1;
+                        }
+                        const uint32_t below = (1u << lane) - 1u;
+#pragma unroll
+                        for (int b = 0; b < 32; ++b) {
+                            if (any_col & (1u << b)) {
+                                const int base_b = __shfl_sync(0xffffffffu, base, b);
+                                const uint32_t rows_b = __shfl_sync(0xffffffffu, mine, b);
+                                if ((hit >> b) & 1u) {
+                                    const int q = qb + j * 32 + b;
+                                    my_cand[static_cast<size_t>(q) * kTcCap + base_b + __popc(rows_b & below)] =
+                                        make_key(__uint_as_float(v[b]), static_cast<uint32_t>(row));
+                                }
                             }
                         }
                     }
@@ -466,8 +542,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         const int b = __ffs(m) - 1;
                         m &= m - 1;
                         const int qq = base + ew * 32 + b;
-                        tc_compact_query(my_cand + static_cast<size_t>(qq) * kTcCap, scratch, thr, cnt, sorted,
-                                         qq, p.k, lane);
+                        tc_compact_query(my_cand + static_cast<size_t>(qq) * kTcCap, thr, cnt, sorted, qq, p.k, lane);
                     }
                 }
                 if (threadIdx.x == 64) *dirty = 0;
@@ -480,7 +555,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             for (int b = 0; b < 32 && q0 + b < p.s; ++b) {
                 const int q = q0 + b;
                 uint64_t *list = my_cand + static_cast<size_t>(q) * kTcCap;
-                if (cnt[q] != sorted[q]) tc_compact_query(list, scratch, thr, cnt, sorted, q, p.k, lane);
+                if (cnt[q] != sorted[q]) tc_compact_query(list, thr, cnt, sorted, q, p.k, lane);
                 const int n = cnt[q];
                 uint64_t *dst = p.partial + (static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
                 for (int i = lane; i < p.k; i += 32) dst[i] = (i < n) ? list[i] : 0ull;

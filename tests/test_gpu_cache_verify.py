@@ -167,3 +167,54 @@ def test_speculate_search_verify_chain():
     assert np.array_equal(m.cpu().numpy(), o_m)
     assert 0 < (o_m < stride).sum() and o_m.max() >= 1     # mismatches and matches both occur
     assert idx.device_status() == 0
+
+
+# ------------------------------------------------------------------ cache update
+@pytest.mark.parametrize("R,C,stride,ld,top,next_n", [(1, 4, 4, 2, 1, 0), (8, 512, 8, 20, 1, 0), (8, 512, 8, 20, 20, 0),
+                                                      (3, 37, 5, 6, 4, 0), (4, 64, 8, 4, 2, 10), (2, 4096, 3, 64, 64, 0),
+                                                      (5, 1, 2, 3, 3, 0), (2, 16, 4, 1024, 1024, 0)])
+def test_cache_update_is_bit_exact(R, C, stride, ld, top, next_n):
+    from oracle.cache_update import cache_update as oracle_update
+    ralm = _ralm()
+    g = torch.Generator().manual_seed(1000 * R + C + stride)
+    N = 3 * C + 50
+    cache = torch.stack([torch.randperm(N, generator=g)[:C] for _ in range(R)]).to(torch.int64)
+    cache[torch.rand(cache.shape, generator=g) < 0.3] = -1
+    cursor = torch.randint(0, C, (R,), generator=g, dtype=torch.int32)
+    retrieved = torch.randint(-1, N, (R, stride, ld), generator=g, dtype=torch.int64)
+    steps = torch.randint(0, stride + 2, (R,), generator=g, dtype=torch.int32)      # also beyond stride: clamped
+    for use_steps in (True, False):
+        want_cache, want_cur = oracle_update(cache.numpy(), cursor.numpy(), retrieved.numpy(), top,
+                                             steps.numpy() if use_steps else None, next_n, N)
+        d_cache, d_cur = cache.to(DEV), cursor.to(DEV)
+        ralm.cache_update(d_cache, d_cur, retrieved.to(DEV), top, N, steps.to(DEV) if use_steps else None, next_n)
+        torch.cuda.synchronize()
+        assert np.array_equal(d_cache.cpu().numpy(), want_cache)
+        assert np.array_equal(d_cur.cpu().numpy(), want_cur)
+
+
+def test_cache_update_closes_the_speculation_loop():
+    """After the retrieved documents enter the caches, speculating the same queries again finds
+    them: every step matches and first_mismatch equals the stride."""
+    ralm = _ralm()
+    N, d, R, stride, C = 80_000, 256, 4, 8, 128
+    x, assign = workloads.mixture_corpus(N, d, 64, seed=81, device=DEV)
+    q, src = workloads.noisy_copy_queries(x, R * stride, seed=82)
+    idx = ralm.Index(x, oracle.IP, R * stride, 5)
+    cache = torch.full((R, C), -1, dtype=torch.int64, device=DEV)
+    cursor = torch.zeros((R,), dtype=torch.int32, device=DEV)
+    qr = q.reshape(R, stride, d).contiguous()
+    spec, _ = ralm.cache_search(idx, cache, qr, 1)
+    retr, _ = ralm.search(idx, q, 5)
+    retr = retr.reshape(R, stride, 5).contiguous()
+    m = ralm.verify(spec.reshape(R, stride).contiguous(), retr)
+    assert m.tolist() == [0] * R                                    # empty caches: nothing matches
+    ralm.cache_update(cache, cursor, retr, 5, N)                    # top-k update with all steps
+    spec, _ = ralm.cache_search(idx, cache, qr, 1)
+    m = ralm.verify(spec.reshape(R, stride).contiguous(), retr)
+    torch.cuda.synchronize()
+    assert m.tolist() == [stride] * R
+    assert cursor.tolist() == [int((cache[r] >= 0).sum()) % C for r in range(R)]
+    # argument errors
+    with pytest.raises(ralm.RalmError):
+        ralm.cache_update(cache, cursor, retr, 6, N)                # top > ld
