@@ -25,20 +25,28 @@ __device__ __forceinline__ void write_result(uint64_t key, bool l2, int64_t *id_
 // Merge: one CTA per query. `partial` holds B lists of k keys, each sorted descending and
 // padded with 0, laid out [B][s][k]. Writes ids [s][k] (int64) and scores [s][k] (fp32).
 // ------------------------------------------------------------------------------------
+// extra_slot >= 0: one more list takes part, stored at that block index of `partial`.
+// With keys_out the merged list is written as keys [s][k] instead (and the k-th value, or -inf
+// when there are fewer than k rows, to thr_out[q]): the result of scanning a sample of the
+// corpus, which seeds the thresholds of the main scan and rejoins the final merge as one more
+// partial list.
 __global__ void __launch_bounds__(kMergeThreads, 1)
 merge_kernel(const uint64_t *__restrict__ partial, int B, int s, int k, int l2,
-             int64_t *__restrict__ ids, float *__restrict__ scores) {
+             int64_t *__restrict__ ids, float *__restrict__ scores, uint64_t *__restrict__ keys_out = nullptr,
+             float *__restrict__ thr_out = nullptr, int extra_slot = -1) {
     __shared__ uint64_t buf[kMergeSortMax];
     const int q = blockIdx.x;
     const int tid = threadIdx.x;
-    const long long total = static_cast<long long>(B) * k;
+    const int lists = B + (extra_slot >= 0 ? 1 : 0);
+    const long long total = static_cast<long long>(lists) * k;
     if (total <= kMergeSortMax) {
         const int P = next_pow2(total > 1 ? static_cast<int>(total) : 2);
         for (int i = tid; i < P; i += kMergeThreads) {
             uint64_t key = 0;
             if (i < total) {
                 const int b = i / k, j = i - b * k;
-                key = partial[(static_cast<size_t>(b) * s + q) * k + j];
+                const int slot = b < B ? b : extra_slot;
+                key = partial[(static_cast<size_t>(slot) * s + q) * k + j];
             }
             buf[i] = key;
         }
@@ -49,11 +57,12 @@ merge_kernel(const uint64_t *__restrict__ partial, int B, int s, int k, int l2,
         // of a descending list and a reversed descending list holds the best P keys of both
         // and is bitonic
         const int P = next_pow2(k);
+        const int slot0 = B > 0 ? 0 : extra_slot;
         for (int i = tid; i < P; i += kMergeThreads)
-            buf[i] = (i < k) ? partial[(static_cast<size_t>(q)) * k + i] : 0ull;
+            buf[i] = (i < k) ? partial[(static_cast<size_t>(slot0) * s + q) * k + i] : 0ull;
         __syncthreads();
-        for (int b = 1; b < B; ++b) {
-            const uint64_t *list = partial + (static_cast<size_t>(b) * s + q) * k;
+        for (int b = 1; b < lists; ++b) {
+            const uint64_t *list = partial + (static_cast<size_t>(b < B ? b : extra_slot) * s + q) * k;
             for (int i = tid; i < P; i += kMergeThreads) {
                 const int j = P - 1 - i;
                 const uint64_t other = (j < k) ? list[j] : 0ull;
@@ -66,8 +75,13 @@ merge_kernel(const uint64_t *__restrict__ partial, int B, int s, int k, int l2,
     }
     for (int i = tid; i < k; i += kMergeThreads) {
         const uint64_t key = (i < total) ? buf[i] : 0ull;
-        write_result(key, l2 != 0, ids + static_cast<size_t>(q) * k + i,
-                     scores + static_cast<size_t>(q) * k + i);
+        if (keys_out) {
+            keys_out[static_cast<size_t>(q) * k + i] = key;
+            if (i == k - 1) thr_out[q] = key ? key_value(key) : -INFINITY;
+        } else {
+            write_result(key, l2 != 0, ids + static_cast<size_t>(q) * k + i,
+                         scores + static_cast<size_t>(q) * k + i);
+        }
     }
 }
 

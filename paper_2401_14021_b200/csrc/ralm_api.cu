@@ -32,6 +32,8 @@ struct ralm_index {
     uint64_t *spill;       // large k: candidate lists of the small-batch scan, [num_sms][8][spill_cap]
     int spill_cap;
     float *norms;          // L2: squared norm of every corpus row (fp32 [N]), or null
+    float *tc_thr;         // tcgen05 scan: thresholds from the sample phase, [max_s]
+    bool tc_two_phase;     // sample phase enabled (tuning aid)
     int tc_clusters;       // CTA pairs the device runs at once (-1 = not asked yet)
     uint64_t *tc_cand;     // tcgen05 scan: [num_sms][tc_cand_q][kTcCap] candidate lists, or null
     int tc_cand_q;
@@ -176,6 +178,10 @@ bool alloc_tc_workspace(ralm_index *idx, int queries) {
     idx->tc_cand = nullptr;
     idx->tc_cand_q = 0;
     const size_t bytes = sizeof(uint64_t) * idx->num_sms * static_cast<size_t>(queries) * kTcCap;
+    if (!idx->tc_thr && cudaMalloc(&idx->tc_thr, sizeof(float) * idx->max_s) != cudaSuccess) {
+        idx->tc_thr = nullptr;
+        return false;
+    }
     if (cudaMalloc(&idx->tc_cand, bytes) != cudaSuccess) {
         idx->tc_cand = nullptr;
         return false;
@@ -187,13 +193,15 @@ bool alloc_tc_workspace(ralm_index *idx, int queries) {
 // One pass of up to min(512, workspace) queries. `pair`: clusters of two CTAs that share each
 // MMA (half the query bytes staged per CTA); falls back to single CTAs when no cluster fits.
 ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int s_total, int q0, int k,
-                             bool pair, int *grid_out, cudaStream_t st) {
+                             bool pair, long long row_begin, long long row_end, const float *thr_init,
+                             int *grid_out, cudaStream_t st) {
     TcParams p;
     p.partial = idx->partial;
     p.cand = idx->tc_cand;
     p.cand_q = idx->tc_cand_q;
     p.status = idx->status;
-    p.N = idx->N;
+    p.N = row_end;
+    p.thr_init = thr_init;
     p.nchunks = (idx->d + kTcChunkK - 1) / kTcChunkK;
     p.s = sp;
     p.s_total = s_total;
@@ -204,7 +212,8 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
     if (!encode_rows_map(&map_x, idx->corpus, idx->N, idx->d, kTcTileM)) return RALM_ERR_CUDA;
     for (;;) {
         const int group_rows = pair ? 2 * kTcTileM : kTcTileM;
-        p.ntiles = (idx->N + group_rows - 1) / group_rows;
+        p.tile0 = row_begin / group_rows;  // row_begin is a multiple of 256
+        p.ntiles = (row_end - row_begin + group_rows - 1) / group_rows;
         p.nb = sp > kTcMaxN ? kTcMaxN : align_up(sp, pair ? 32 : 16);
         p.nhalves = (sp + p.nb - 1) / p.nb;
         const int nb_cta = pair ? p.nb / 2 : p.nb;
@@ -265,10 +274,19 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     const bool tc = tc_can_serve(idx, k) &&
                     (idx->variant == 3 || idx->variant == 4 || (idx->variant == 0 && s >= kTcAutoMinQueries));
     if (tc) {
-        int grid = idx->N > 0 ? 1 : 0;  // set by the passes (the same for all of them)
+        // Large corpora are scanned in two phases: a small sample first, whose merged top-k gives
+        // every query a score that k rows are known to reach; the rest then starts from those
+        // thresholds, so that hardly any score passes and the selection stays off the critical
+        // path. The sample's list rejoins the final merge (block index num_sms of `partial`).
+        const long long group_rows = 2 * kTcTileM;
+        long long sample = std::max<long long>(idx->N / 64, 4LL * idx->num_sms * kTcTileM);
+        sample = (sample + group_rows - 1) / group_rows * group_rows;
+        const bool two_phase = sample * 8 <= idx->N && idx->tc_two_phase;
+        int grid = 0;
         const int per_pass = std::min(kTcMaxQueries, idx->tc_cand_q);
-        for (int q0 = 0; grid > 0 && q0 < s; q0 += per_pass) {
+        for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
             const int sp = std::min(per_pass, s - q0);
+            const __half *qp = queries + static_cast<size_t>(q0) * idx->d;
             std::pair<cudaEvent_t, cudaEvent_t> ev{nullptr, nullptr};
             if (idx->timing) {
                 if (!idx->spare.empty()) {
@@ -280,9 +298,23 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
                 }
                 cudaEventRecord(ev.first, st);
             }
-            const ralm_status_t rs =
-                launch_tc_pass(idx, queries + static_cast<size_t>(q0) * idx->d, sp, s, q0, k,
-                               idx->variant != 4, &grid, st);
+            ralm_status_t rs = RALM_OK;
+            if (two_phase) {
+                int grid1 = 0;
+                rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, sample, nullptr, &grid1, st);
+                if (rs == RALM_OK) {
+                    merge_kernel<<<sp, kMergeThreads, 0, st>>>(
+                        idx->partial + static_cast<size_t>(q0) * k, grid1, s, k, 0, nullptr, nullptr,
+                        idx->partial + (static_cast<size_t>(idx->num_sms) * s + q0) * k, idx->tc_thr + q0);
+                    if (cudaGetLastError() != cudaSuccess) rs = RALM_ERR_CUDA;
+                }
+                if (rs == RALM_OK)
+                    rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, sample, idx->N, idx->tc_thr,
+                                        &grid, st);
+                idx->launches += 2;
+            } else {
+                rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, idx->N, nullptr, &grid, st);
+            }
             if (idx->timing) {
                 cudaEventRecord(ev.second, st);
                 idx->timed.push_back(ev);
@@ -290,7 +322,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             if (rs != RALM_OK) return rs;
             idx->launches++;
         }
-        merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, 0, ids, scores);
+        merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, 0, ids, scores, nullptr, nullptr,
+                                                  two_phase ? idx->num_sms : -1);
         if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
         idx->launches++;
         return RALM_OK;
@@ -464,11 +497,14 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->tune_warps = idx->tune_depth = idx->tune_rows = 0;
     idx->launches = 0;
     idx->timing = false;
-    const size_t partial_bytes = sizeof(uint64_t) * idx->num_sms * max_s * static_cast<size_t>(max_k);
+    // one list per scan CTA and query, plus one more block for the list of a sample phase
+    const size_t partial_bytes = sizeof(uint64_t) * (idx->num_sms + 1) * max_s * static_cast<size_t>(max_k);
     const size_t sk = static_cast<size_t>(max_s) * max_k;
     idx->tc_cand = nullptr;
     idx->tc_cand_q = 0;
     idx->tc_clusters = -1;
+    idx->tc_thr = nullptr;
+    idx->tc_two_phase = true;
     idx->norms = nullptr;
     idx->spill = nullptr;
     idx->spill_cap = 0;
@@ -513,6 +549,7 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
     cudaFree(idx->partial);
     cudaFree(idx->cache_keys);
     cudaFree(idx->tc_cand);
+    cudaFree(idx->tc_thr);
     cudaFree(idx->norms);
     cudaFree(idx->spill);
     cudaFree(idx->status);
@@ -667,6 +704,8 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.tc_cand = nullptr;
     view.tc_cand_q = 0;
     view.tc_clusters = -1;
+    view.tc_thr = nullptr;
+    view.tc_two_phase = false;
     view.spill = nullptr;
     view.spill_cap = 0;
     view.norms = nullptr;  // no index, no stored norms: the scan derives them on the tensor cores

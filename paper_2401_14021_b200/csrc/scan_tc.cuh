@@ -50,8 +50,10 @@ struct TcParams {
     uint64_t *partial;  // [gridDim.x][s_total][k] sorted keys, 0 = empty
     uint64_t *cand;     // [gridDim.x][cand_q][kTcCap] candidate lists
     int *status;
-    long long N;
-    long long ntiles;   // ceil(N / 128)
+    long long N;        // rows of this launch end here (the whole corpus, or the end of a sample)
+    long long tile0;    // first row tile (of 128 rows, 256 for pairs) of this launch
+    const float *thr_init;  // [s_total] starting thresholds (scores that k rows are known to reach), or null
+    long long ntiles;   // row tiles of this launch
     int nchunks;        // ceil(d / 64)
     int s;              // queries in this pass (<= 512)
     int s_total;
@@ -74,7 +76,7 @@ struct TcHeader {
     uint64_t drain;
     uint32_t tmem_base;
     int abort;
-    int dirty;  // some candidate list reached kTcSoft during the current unit
+    int dirty[3];  // [u % 3]: some candidate list reached kTcSoft during unit u
 };
 constexpr int kTcHeaderBytes = 512;
 static_assert(sizeof(TcHeader) <= kTcHeaderBytes, "header too large");
@@ -215,6 +217,55 @@ __device__ __forceinline__ void tc_compact_query(uint64_t *list, float *thr, int
     else tc_compact_sorted<8>(list, thr, cnt, sorted, q, n, k, lane);
 }
 
+// The rare part of the selection: some score of this warp's 32 rows x 32 columns passes its
+// threshold. Out of line, and re-reading the scores from TMEM, so that the common path (no score
+// passes) stays a short loop with few live registers. The warp appends as a whole: lane L
+// learns which rows pass column L (one ballot per column that has any), reserves that many
+// slots of query L's list with ONE atomic instruction (32 different lists), and every passing
+// row then stores its key at its rank within the reservation.
+__device__ __noinline__ void tc_append_chunk(uint32_t taddr, const float *thr_chunk, int *cnt_chunk,
+                                             uint64_t *cand_chunk, uint32_t row, bool row_ok,
+                                             volatile int *dirty, int lane) {
+    uint32_t v[32];
+    tmem_ld32(taddr, v);
+    const float4 *t4 = reinterpret_cast<const float4 *>(thr_chunk);
+    uint32_t hit = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float4 th = t4[i];
+        hit |= (__uint_as_float(v[4 * i + 0]) >= th.x ? 1u : 0u) << (4 * i + 0);
+        hit |= (__uint_as_float(v[4 * i + 1]) >= th.y ? 1u : 0u) << (4 * i + 1);
+        hit |= (__uint_as_float(v[4 * i + 2]) >= th.z ? 1u : 0u) << (4 * i + 2);
+        hit |= (__uint_as_float(v[4 * i + 3]) >= th.w ? 1u : 0u) << (4 * i + 3);
+    }
+    if (!row_ok) hit = 0;
+    const uint32_t any_col = __reduce_or_sync(0xffffffffu, hit);
+    uint32_t mine = 0;
+#pragma unroll
+    for (int b = 0; b < 32; ++b) {
+        if (any_col & (1u << b)) {
+            const uint32_t m = __ballot_sync(0xffffffffu, (hit >> b) & 1u);
+            if (lane == b) mine = m;
+        }
+    }
+    int base = 0;
+    if (mine) {
+        base = atomicAdd(&cnt_chunk[lane], __popc(mine));
+        if (base + __popc(mine) >= kTcSoft) *dirty = 1;
+    }
+    const uint32_t below = (1u << lane) - 1u;
+#pragma unroll
+    for (int b = 0; b < 32; ++b) {
+        if (any_col & (1u << b)) {
+            const int base_b = __shfl_sync(0xffffffffu, base, b);
+            const uint32_t rows_b = __shfl_sync(0xffffffffu, mine, b);
+            if ((hit >> b) & 1u)
+                cand_chunk[static_cast<size_t>(b) * kTcCap + base_b + __popc(rows_b & below)] =
+                    make_key(__uint_as_float(v[b]), row);
+        }
+    }
+}
+
 // ---- CTA-pair helpers (PAIR = true: two CTAs of a cluster work as one MMA unit) -----------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -296,10 +347,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         mbar_init(smem_u32(&hdr->drain), 1);
         mbar_fence_init();
         hdr->abort = 0;
-        hdr->dirty = 0;
+        hdr->dirty[0] = hdr->dirty[1] = hdr->dirty[2] = 0;
     }
     for (int q = threadIdx.x; q < kTcMaxQueries; q += kTcThreads) {
-        thr[q] = (q < p.s) ? -INFINITY : INFINITY;  // absent queries never pass
+        // absent queries never pass; the others start at a score that k rows are already known
+        // to reach, when the caller has one
+        thr[q] = (q < p.s) ? (p.thr_init ? p.thr_init[p.q_base + q] : -INFINITY) : INFINITY;
         cnt[q] = 0;
         sorted[q] = 0;
     }
@@ -340,7 +393,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             long long issued = 0;
             bool ok = true, stop = false;
             for (long long u = 0; u < my_units && !stop; ++u) {
-                const long long tile = group + (u / p.nhalves) * ngroups;
+                const long long tile = p.tile0 + group + (u / p.nhalves) * ngroups;
                 const int half = static_cast<int>(u % p.nhalves);
                 const int row_y = static_cast<int>(tile * kGroupRows + rank * kTcTileM);
                 // a pair splits the N of this unit's MMA, not nb: the follower supplies the upper
@@ -444,14 +497,14 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const int ew = warp - 2;        // 0..3
         const int quarter = warp & 3;   // the TMEM lanes this warp may read: 32 * quarter ..
         uint64_t *my_cand = p.cand + static_cast<size_t>(blockIdx.x) * p.cand_q * kTcCap;
-        volatile int *dirty = &hdr->dirty;
         bool ok = true;
         for (long long u = 0; u < my_units; ++u) {
-            const long long tile = group + (u / p.nhalves) * ngroups;
+            const long long tile = p.tile0 + group + (u / p.nhalves) * ngroups;
             const int half = static_cast<int>(u % p.nhalves);
             const int acc = static_cast<int>(u & 1);
             const int qb = half * p.nb;
             const int nq = (p.s - qb < p.nb) ? (p.s - qb) : p.nb;
+            volatile int *dirty = &hdr->dirty[u % 3];
             if (ok && !*abort_flag) {
                 int got = 0;
                 if (lane == 0)
@@ -476,49 +529,20 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     uint32_t v[32];
                     tmem_ld32(t_row + j * 32, v);
                     const float4 *t4 = reinterpret_cast<const float4 *>(thr + qb + j * 32);
-                    uint32_t hit = 0;
+                    // common case: nothing passes. Four independent predicate chains.
+                    bool p0 = false, p1 = false, p2 = false, p3 = false;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const float4 th = t4[i];
-                        hit |= (__uint_as_float(v[4 * i + 0]) >= th.x ? 1u : 0u) << (4 * i + 0);
-                        hit |= (__uint_as_float(v[4 * i + 1]) >= th.y ? 1u : 0u) << (4 * i + 1);
-                        hit |= (__uint_as_float(v[4 * i + 2]) >= th.z ? 1u : 0u) << (4 * i + 2);
-                        hit |= (__uint_as_float(v[4 * i + 3]) >= th.w ? 1u : 0u) << (4 * i + 3);
+                        p0 |= __uint_as_float(v[4 * i + 0]) >= th.x;
+                        p1 |= __uint_as_float(v[4 * i + 1]) >= th.y;
+                        p2 |= __uint_as_float(v[4 * i + 2]) >= th.z;
+                        p3 |= __uint_as_float(v[4 * i + 3]) >= th.w;
                     }
-                    if (!row_ok) hit = 0;
-                    // Rows that pass are appended by the warp as a whole: lane L learns which rows
-                    // pass column L (one ballot per column that has any), reserves that many slots
-                    // of query L's list with ONE atomic instruction (32 different lists), and
-                    // every passing row then stores its key at its rank within the reservation.
-                    const uint32_t any_col = __reduce_or_sync(0xffffffffu, hit);
-                    if (any_col) {
-                        uint32_t mine = 0;
-#pragma unroll
-                        for (int b = 0; b < 32; ++b) {
-                            if (any_col & (1u << b)) {
-                                const uint32_t m = __ballot_sync(0xffffffffu, (hit >> b) & 1u);
-                                if (lane == b) mine = m;
-                            }
-                        }
-                        int base = 0;
-                        if (mine) {
-                            base = atomicAdd(&cnt[qb + j * 32 + lane], __popc(mine));
-                            if (base + __popc(mine) >= kTcSoft) *dirty = 1;
-                        }
-                        const uint32_t below = (1u << lane) - 1u;
-#pragma unroll
-                        for (int b = 0; b < 32; ++b) {
-                            if (any_col & (1u << b)) {
-                                const int base_b = __shfl_sync(0xffffffffu, base, b);
-                                const uint32_t rows_b = __shfl_sync(0xffffffffu, mine, b);
-                                if ((hit >> b) & 1u) {
-                                    const int q = qb + j * 32 + b;
-                                    my_cand[static_cast<size_t>(q) * kTcCap + base_b + __popc(rows_b & below)] =
-                                        make_key(__uint_as_float(v[b]), static_cast<uint32_t>(row));
-                                }
-                            }
-                        }
-                    }
+                    if (__any_sync(0xffffffffu, row_ok && (p0 | p1 | p2 | p3)))
+                        tc_append_chunk(t_row + j * 32, thr + qb + j * 32, cnt + qb + j * 32,
+                                        my_cand + static_cast<size_t>(qb + j * 32) * kTcCap,
+                                        static_cast<uint32_t>(row), row_ok, dirty, lane);
                 }
                 // accumulator drained: hand it back to the MMA thread (the pair's leader)
                 tc_fence_before();
@@ -529,11 +553,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 }
             }
             // All four warps meet after every unit (also when winding down, so that nobody is
-            // left waiting): first so that every push of the unit is visible, then, having all
-            // read the same value of the flag, to compact the lists that asked for it.
+            // left waiting) so that every push of the unit is visible; each then reads the
+            // unit's flag. Three flags in rotation make one barrier enough: unit u's flag is
+            // written during unit u, read between the barriers that end units u and u + 1, and
+            // cleared after the barrier that ends unit u + 1, well before unit u + 3 writes it.
             named_barrier(1, 128);
             const int need = *dirty;
-            named_barrier(1, 128);
+            if (threadIdx.x == 64) *reinterpret_cast<volatile int *>(&hdr->dirty[(u + 2) % 3]) = 0;
             if (need) {
                 for (int base = 0; base < p.s; base += 128) {
                     const int q = base + ew * 32 + lane;
@@ -545,8 +571,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         tc_compact_query(my_cand + static_cast<size_t>(qq) * kTcCap, thr, cnt, sorted, qq, p.k, lane);
                     }
                 }
-                if (threadIdx.x == 64) *dirty = 0;
-                named_barrier(1, 128);
+                named_barrier(1, 128);  // thresholds and counts settled before the next unit's pushes
             }
         }
         // ---- CTA result: every list sorted and cut to k, written as this CTA's partial lists

@@ -207,6 +207,19 @@ def test_tcgen05_scan_parity(N, d, s, k):
     torch.testing.assert_close(scores1, scores, rtol=1e-5, atol=1e-6)
 
 
+def test_tcgen05_scan_two_phases_integer_inputs():
+    """Corpora of 8 sample-sizes or more are scanned sample first (its merged top-k seeds the
+    thresholds of the rest): ties abound in integer data, so any row lost at the seam, or to a
+    threshold that is too tight, would show. Also a query batch that needs two passes."""
+    N, d = 700_001, 64
+    x = workloads.integer_valued((N, d), seed=77, lo=-2, hi=2, device=DEV)
+    for s, k in ((40, 5), (530, 2)):
+        q = workloads.integer_valued((s, d), seed=78 + s, lo=-2, hi=2, device=DEV)
+        for variant in (3, 4):
+            ids, scores = _run(x, q, oracle.IP, k, variant)
+            check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+
+
 def test_tcgen05_scan_adversarial_row_order():
     """Scores increase along the corpus: every row passes every threshold, so every unit ends
     in a compaction of every list."""
