@@ -32,7 +32,7 @@ struct ralm_index {
     uint64_t *spill;       // large k: candidate lists of the small-batch scan, [num_sms][8][spill_cap]
     int spill_cap;
     float *norms;          // L2: squared norm of every corpus row (fp32 [N]), or null
-    float *tc_thr;         // tcgen05 scan: thresholds from the sample phase, [max_s]
+    float *tc_thr;         // thresholds from the sample phase of a two-phase scan, [max_s]
     bool tc_two_phase;     // sample phase enabled (tuning aid)
     int tc_clusters;       // CTA pairs the device runs at once (-1 = not asked yet)
     uint64_t *tc_cand;     // tcgen05 scan: [num_sms][tc_cand_q][kTcCap] candidate lists, or null
@@ -332,75 +332,97 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     const bool mma = variant == 2;
     if (!mma && idx->d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
     const int per_pass = mma ? kScanMaxQueries : kFmaQueriesPerPass;
-    const int grid = static_cast<int>(std::min<long long>(idx->num_sms, (idx->N + 15) / 16));
-    if (grid > 0) {
-        for (int q0 = 0; q0 < s; q0 += per_pass) {
-            const int sp = std::min(per_pass, s - q0);
-            ScanPlan pl;
-            if (!plan_scan(idx, mma, sp, k, &pl)) return RALM_ERR_UNSUPPORTED;
-            ScanParams p;
-            p.corpus = idx->corpus;
-            p.queries = queries + static_cast<size_t>(q0) * idx->d;
-            p.norms = idx->norms;
-            p.spill = pl.spill ? idx->spill : nullptr;
-            p.partial = idx->partial;
-            p.status = idx->status;
-            p.N = idx->N;
-            p.ntiles = (idx->N + pl.tile_rows - 1) / pl.tile_rows;
-            p.d = idx->d;
-            p.s = sp;
-            p.s_total = s;
-            p.q_base = q0;
-            p.k = k;
-            p.cap = pl.cap;
-            p.soft_limit = pl.soft_limit;
-            p.tile_rows = pl.tile_rows;
-            p.nwarps = pl.nwarps;
-            p.depth = pl.depth;
-            p.stage_bytes = pl.stage_bytes;
-            p.off_q = pl.off_q;
-            p.off_cand = pl.off_cand;
-            p.off_stage = pl.off_stage;
-            // bound on the rounding error of the tensor-core |x|^2 - 2 x.q + |q|^2 relative to
-            // |x|^2 + |q|^2: d accumulation steps of at most 2^-22 each, on terms that sum to
-            // at most twice that scale
-            p.l2_slack = static_cast<float>(idx->d) * (1.0f / 2097152.0f);
-            cudaError_t e;
-            std::pair<cudaEvent_t, cudaEvent_t> ev{nullptr, nullptr};
-            if (idx->timing) {
-                if (!idx->spare.empty()) {
-                    ev = idx->spare.back();
-                    idx->spare.pop_back();
-                } else if (cudaEventCreate(&ev.first) != cudaSuccess ||
-                           cudaEventCreate(&ev.second) != cudaSuccess) {
-                    return RALM_ERR_CUDA;
-                }
-                cudaEventRecord(ev.first, st);
+    // k > 1 on a large corpus: scan a sample first and start the rest from the sample's merged
+    // k-th scores (see the large-batch path above); the sample's list is block num_sms of `partial`
+    long long sample = std::max<long long>(idx->N / 64, 4LL * idx->num_sms * kTcTileM);
+    sample = (sample + 255) / 256 * 256;
+    const bool two_phase = k > 1 && idx->tc_thr && idx->tc_two_phase && sample * 8 <= idx->N;
+    int grid = 0;
+    for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
+        const int sp = std::min(per_pass, s - q0);
+        ScanPlan pl;
+        if (!plan_scan(idx, mma, sp, k, &pl)) return RALM_ERR_UNSUPPORTED;
+        ScanParams p;
+        p.corpus = idx->corpus;
+        p.queries = queries + static_cast<size_t>(q0) * idx->d;
+        p.norms = idx->norms;
+        p.spill = pl.spill ? idx->spill : nullptr;
+        p.partial = idx->partial;
+        p.status = idx->status;
+        p.d = idx->d;
+        p.s = sp;
+        p.s_total = s;
+        p.q_base = q0;
+        p.k = k;
+        p.cap = pl.cap;
+        p.soft_limit = pl.soft_limit;
+        p.tile_rows = pl.tile_rows;
+        p.nwarps = pl.nwarps;
+        p.depth = pl.depth;
+        p.stage_bytes = pl.stage_bytes;
+        p.off_q = pl.off_q;
+        p.off_cand = pl.off_cand;
+        p.off_stage = pl.off_stage;
+        // bound on the rounding error of the tensor-core |x|^2 - 2 x.q + |q|^2 relative to
+        // |x|^2 + |q|^2: d accumulation steps of at most 2^-22 each, on terms that sum to
+        // at most twice that scale
+        p.l2_slack = static_cast<float>(idx->d) * (1.0f / 2097152.0f);
+        // one launch over rows [begin, end) starting from the given thresholds
+        auto scan_rows = [&](long long begin, long long end, const float *thr_init, int *grid_out) -> cudaError_t {
+            p.row_begin = begin;
+            p.N = end;
+            p.thr_init = thr_init;
+            p.ntiles = (end - begin + pl.tile_rows - 1) / pl.tile_rows;
+            // the same grid whatever the tile height of the pass: the merge reads one list per CTA
+            const int g = static_cast<int>(std::min<long long>(idx->num_sms, (end - begin + 15) / 16));
+            *grid_out = g;
+            if (mma && idx->metric == RALM_L2 && idx->norms)
+                return (k == 1) ? launch_scan<true, true, 8, 1, true, true>(p, g, pl.smem_bytes, st)
+                                : launch_scan<true, true, 8, 1, false, true>(p, g, pl.smem_bytes, st);
+            if (mma && idx->metric == RALM_L2)
+                return (k == 1) ? launch_scan<true, true, 8, 1, true>(p, g, pl.smem_bytes, st)
+                                : launch_scan<true, true, 8, 1, false>(p, g, pl.smem_bytes, st);
+            if (mma)
+                return (k == 1) ? launch_scan<true, false, 8, 1, true>(p, g, pl.smem_bytes, st)
+                                : launch_scan<true, false, 8, 1, false>(p, g, pl.smem_bytes, st);
+            return idx->metric == RALM_L2 ? launch_fma<true>(p, g, pl.smem_bytes, st)
+                                          : launch_fma<false>(p, g, pl.smem_bytes, st);
+        };
+        cudaError_t e;
+        std::pair<cudaEvent_t, cudaEvent_t> ev{nullptr, nullptr};
+        if (idx->timing) {
+            if (!idx->spare.empty()) {
+                ev = idx->spare.back();
+                idx->spare.pop_back();
+            } else if (cudaEventCreate(&ev.first) != cudaSuccess ||
+                       cudaEventCreate(&ev.second) != cudaSuccess) {
+                return RALM_ERR_CUDA;
             }
-            if (mma && idx->metric == RALM_L2 && idx->norms) {
-                e = (k == 1) ? launch_scan<true, true, 8, 1, true, true>(p, grid, pl.smem_bytes, st)
-                             : launch_scan<true, true, 8, 1, false, true>(p, grid, pl.smem_bytes, st);
-            } else if (mma && idx->metric == RALM_L2) {
-                e = (k == 1) ? launch_scan<true, true, 8, 1, true>(p, grid, pl.smem_bytes, st)
-                             : launch_scan<true, true, 8, 1, false>(p, grid, pl.smem_bytes, st);
-            } else if (mma) {
-                e = (k == 1) ? launch_scan<true, false, 8, 1, true>(p, grid, pl.smem_bytes, st)
-                             : launch_scan<true, false, 8, 1, false>(p, grid, pl.smem_bytes, st);
-            } else if (idx->metric == RALM_L2) {
-                e = launch_fma<true>(p, grid, pl.smem_bytes, st);
-            } else {
-                e = launch_fma<false>(p, grid, pl.smem_bytes, st);
-            }
-            if (idx->timing) {
-                cudaEventRecord(ev.second, st);
-                idx->timed.push_back(ev);
-            }
-            if (e != cudaSuccess) return RALM_ERR_CUDA;
-            idx->launches++;
+            cudaEventRecord(ev.first, st);
         }
+        if (two_phase) {
+            int grid1 = 0;
+            e = scan_rows(0, sample, nullptr, &grid1);
+            if (e == cudaSuccess) {
+                merge_kernel<<<sp, kMergeThreads, 0, st>>>(
+                    idx->partial + static_cast<size_t>(q0) * k, grid1, s, k, idx->metric == RALM_L2, nullptr,
+                    nullptr, idx->partial + (static_cast<size_t>(idx->num_sms) * s + q0) * k, idx->tc_thr + q0);
+                e = cudaGetLastError();
+            }
+            if (e == cudaSuccess) e = scan_rows(sample, idx->N, idx->tc_thr, &grid);
+            idx->launches += 2;
+        } else {
+            e = scan_rows(0, idx->N, nullptr, &grid);
+        }
+        if (idx->timing) {
+            cudaEventRecord(ev.second, st);
+            idx->timed.push_back(ev);
+        }
+        if (e != cudaSuccess) return RALM_ERR_CUDA;
+        idx->launches++;
     }
-    merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, idx->metric == RALM_L2, ids,
-                                              scores);
+    merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, idx->metric == RALM_L2, ids, scores,
+                                              nullptr, nullptr, two_phase ? idx->num_sms : -1);
     if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
     idx->launches++;
     return RALM_OK;
@@ -509,6 +531,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->spill = nullptr;
     idx->spill_cap = 0;
     bool ok = cudaMalloc(&idx->partial, partial_bytes) == cudaSuccess;
+    ok = ok && cudaMalloc(&idx->tc_thr, sizeof(float) * max_s) == cudaSuccess;
     if (max_k > 1 && std::max(512, 2 * next_pow2(max_k)) * 8 > kSmemCandBytes / kScanMaxQueries) {
         idx->spill_cap = std::max(512, 2 * next_pow2(max_k));
         ok = ok && cudaMalloc(&idx->spill, sizeof(uint64_t) * idx->num_sms * kScanMaxQueries *

@@ -45,8 +45,11 @@ struct ScanParams {
     uint64_t *spill;        // large k: candidate lists in global memory, [gridDim.x][8][cap]; the
                             // shared-memory candidate area then holds one sort scratch of cap keys
     int *status;
-    long long N;
-    long long ntiles;
+    long long N;        // rows of this launch end here (the whole corpus, or the end of a sample)
+    long long row_begin;  // first row of this launch (a multiple of tile_rows)
+    const float *thr_init;  // k > 1: [s_total] starting thresholds (rank values that k rows are
+                            // known to reach), or null
+    long long ntiles;   // tiles of this launch
     int d;
     int s;        // queries in this pass (<= 8)
     int s_total;  // queries of the whole call (layout of `partial`)
@@ -248,7 +251,7 @@ scan_kernel(const ScanParams p) {
         hdr->done = 0;
     }
     if (threadIdx.x < kScanMaxQueries) {
-        hdr->thr[threadIdx.x] = -INFINITY;
+        hdr->thr[threadIdx.x] = (p.thr_init && threadIdx.x < p.s) ? p.thr_init[p.q_base + threadIdx.x] : -INFINITY;
         hdr->cnt[threadIdx.x] = 0;
         hdr->best[threadIdx.x] = 0ull;
     }
@@ -281,7 +284,7 @@ scan_kernel(const ScanParams p) {
             // use-th time. The counters advance incrementally: no division on this path.
             int cw = 0, slot = 0;
             uint32_t use = 0;
-            long long row0 = static_cast<long long>(blockIdx.x) * T;
+            long long row0 = p.row_begin + static_cast<long long>(blockIdx.x) * T;
             const long long row_step = static_cast<long long>(gridDim.x) * T;
             const uint32_t stage_base = smem_u32(smem + p.off_stage);
             for (long long it = 0; it < my_tiles; ++it) {
@@ -373,7 +376,8 @@ scan_kernel(const ScanParams p) {
 
         int slot = 0;         // position in this warp's private ring
         uint32_t parity = 0;  // phase parity of the ring's current lap
-        long long row0 = (static_cast<long long>(blockIdx.x) + static_cast<long long>(w) * gridDim.x) * T;
+        long long row0 =
+            p.row_begin + (static_cast<long long>(blockIdx.x) + static_cast<long long>(w) * gridDim.x) * T;
         const long long row_step = static_cast<long long>(gridDim.x) * W * T;
         for (long long it = w; it < my_tiles; it += W, row0 += row_step) {
             if (*abort_flag) continue;

@@ -220,6 +220,18 @@ def test_tcgen05_scan_two_phases_integer_inputs():
             check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
 
 
+@pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
+def test_small_batch_scan_two_phases_integer_inputs(metric):
+    """The same sample-first scheme in the small-batch scans (k > 1 on a large corpus)."""
+    N, d = 650_003, 40
+    x = workloads.integer_valued((N, d), seed=87, lo=-2, hi=2, device=DEV)
+    q = workloads.integer_valued((5, d), seed=88, lo=-2, hi=2, device=DEV)
+    for variant in VARIANTS[metric]:
+        for k in (7, 300):
+            ids, scores = _run(x, q, metric, k, variant)
+            check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), metric, k, exact=True)
+
+
 def test_tcgen05_scan_adversarial_row_order():
     """Scores increase along the corpus: every row passes every threshold, so every unit ends
     in a compaction of every list."""
