@@ -336,7 +336,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     // k-th scores (see the large-batch path above); the sample's list is block num_sms of `partial`
     long long sample = std::max<long long>(idx->N / 64, 4LL * idx->num_sms * kTcTileM);
     sample = (sample + 255) / 256 * 256;
-    const bool two_phase = k > 1 && idx->tc_thr && idx->tc_two_phase && sample * 8 <= idx->N;
+    // (two more launches: only worth it when the scan itself takes a millisecond or more)
+    const bool two_phase = k > 1 && idx->tc_thr && idx->tc_two_phase && sample * 32 <= idx->N;
     int grid = 0;
     for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
         const int sp = std::min(per_pass, s - q0);

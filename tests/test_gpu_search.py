@@ -223,7 +223,7 @@ def test_tcgen05_scan_two_phases_integer_inputs():
 @pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
 def test_small_batch_scan_two_phases_integer_inputs(metric):
     """The same sample-first scheme in the small-batch scans (k > 1 on a large corpus)."""
-    N, d = 650_003, 40
+    N, d = 2_500_003, 16
     x = workloads.integer_valued((N, d), seed=87, lo=-2, hi=2, device=DEV)
     q = workloads.integer_valued((5, d), seed=88, lo=-2, hi=2, device=DEV)
     for variant in VARIANTS[metric]:
