@@ -81,7 +81,9 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
     if (k > 1) {
         // after the flag is raised every warp may still finish the tile it is on
         pl->cap = std::max(512, 2 * next_pow2(k));
-        pl->soft_limit = pl->cap - (kMaxConsumerWarps + 1) * pl->tile_rows;
+        // compact before the buffer is full, and already at about 4 k entries: a threshold only
+        // rises when its list is compacted, and until then every push costs a shared atomic
+        pl->soft_limit = std::min(pl->cap - (kMaxConsumerWarps + 1) * pl->tile_rows, std::max(4 * k, 64));
         // the stage ring needs the room more than large lists do: those go to global memory
         // (they are touched rarely) and only the scratch they are sorted in stays here
         pl->spill = s_pass * pl->cap * 8 > kSmemCandBytes && idx->spill && pl->cap <= idx->spill_cap;
@@ -133,6 +135,26 @@ int resolve_variant(const ralm_index *idx) {
     return 2;
 }
 
+
+using TimedEvents = std::pair<cudaEvent_t, cudaEvent_t>;
+
+// Optional timing of the scan launches of one pass: a pair of events recorded on the caller's
+// stream directly around them, kept until ralm_index_read_timing collects the durations.
+bool timing_begin(ralm_index *idx, cudaStream_t st, TimedEvents *ev) {
+    if (!idx->timing) return true;
+    if (!idx->spare.empty()) {
+        *ev = idx->spare.back();
+        idx->spare.pop_back();
+    } else if (cudaEventCreate(&ev->first) != cudaSuccess || cudaEventCreate(&ev->second) != cudaSuccess) {
+        return false;
+    }
+    return cudaEventRecord(ev->first, st) == cudaSuccess;
+}
+void timing_end(ralm_index *idx, cudaStream_t st, const TimedEvents &ev) {
+    if (!idx->timing) return;
+    cudaEventRecord(ev.second, st);
+    idx->timed.push_back(ev);
+}
 
 // ---- tcgen05 scan (large batches, inner product) -------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
@@ -287,17 +309,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
         for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
             const int sp = std::min(per_pass, s - q0);
             const __half *qp = queries + static_cast<size_t>(q0) * idx->d;
-            std::pair<cudaEvent_t, cudaEvent_t> ev{nullptr, nullptr};
-            if (idx->timing) {
-                if (!idx->spare.empty()) {
-                    ev = idx->spare.back();
-                    idx->spare.pop_back();
-                } else if (cudaEventCreate(&ev.first) != cudaSuccess ||
-                           cudaEventCreate(&ev.second) != cudaSuccess) {
-                    return RALM_ERR_CUDA;
-                }
-                cudaEventRecord(ev.first, st);
-            }
+            TimedEvents ev{nullptr, nullptr};
+            if (!timing_begin(idx, st, &ev)) return RALM_ERR_CUDA;
             ralm_status_t rs = RALM_OK;
             if (two_phase) {
                 int grid1 = 0;
@@ -315,10 +328,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             } else {
                 rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, idx->N, nullptr, &grid, st);
             }
-            if (idx->timing) {
-                cudaEventRecord(ev.second, st);
-                idx->timed.push_back(ev);
-            }
+            timing_end(idx, st, ev);
             if (rs != RALM_OK) return rs;
             idx->launches++;
         }
@@ -390,17 +400,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
                                           : launch_fma<false>(p, g, pl.smem_bytes, st);
         };
         cudaError_t e;
-        std::pair<cudaEvent_t, cudaEvent_t> ev{nullptr, nullptr};
-        if (idx->timing) {
-            if (!idx->spare.empty()) {
-                ev = idx->spare.back();
-                idx->spare.pop_back();
-            } else if (cudaEventCreate(&ev.first) != cudaSuccess ||
-                       cudaEventCreate(&ev.second) != cudaSuccess) {
-                return RALM_ERR_CUDA;
-            }
-            cudaEventRecord(ev.first, st);
-        }
+        TimedEvents ev{nullptr, nullptr};
+        if (!timing_begin(idx, st, &ev)) return RALM_ERR_CUDA;
         if (two_phase) {
             int grid1 = 0;
             e = scan_rows(0, sample, nullptr, &grid1);
@@ -415,10 +416,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
         } else {
             e = scan_rows(0, idx->N, nullptr, &grid);
         }
-        if (idx->timing) {
-            cudaEventRecord(ev.second, st);
-            idx->timed.push_back(ev);
-        }
+        timing_end(idx, st, ev);
         if (e != cudaSuccess) return RALM_ERR_CUDA;
         idx->launches++;
     }
