@@ -238,6 +238,20 @@ ralm_status_t ralm_os3_gamma(const int32_t *matched, const int32_t *strides, int
 ralm_status_t ralm_os3_stride(const int32_t *matched, const int32_t *strides, int32_t w, double gamma_max,
                               double a, double b, int32_t s_max, int32_t async_verify, int32_t *s_out);
 
+/* Testing aids for the failure paths (neither is needed in normal use).
+ *
+ * ralm_debug_fail_allocation: the nth device allocation the library makes from now on (1 = the
+ *   next one) fails as if the device were out of memory; 0 switches the injection off. Lets a
+ *   test see ralm_index_create return RALM_ERR_OOM and give back what it had already allocated.
+ *   Process-wide; not for concurrent use with real work.
+ * ralm_selftest_wait_timeout: runs the library's bounded wait on a barrier that nothing ever
+ *   completes, with a limit of `limit_cycles` SM clock cycles (1 .. 2e9). The kernel must return
+ *   by itself and set *device_status (DEVICE int32, zeroed by the caller) to RALM_ERR_TIMEOUT,
+ *   which is how every pipeline wait of the scan kernels ends when its partner never arrives.
+ *   Asynchronous on `stream`. */
+ralm_status_t ralm_debug_fail_allocation(int32_t nth);
+ralm_status_t ralm_selftest_wait_timeout(int64_t limit_cycles, int32_t *device_status, void *stream);
+
 /* Static description of a status code. */
 const char *ralm_status_string(ralm_status_t status);
 

@@ -52,6 +52,10 @@ def load_library() -> ctypes.CDLL:
     lib.ralm_verify.argtypes = [p, p, i32, i32, i32, i32, p, p]
     lib.ralm_cache_update.restype = i32
     lib.ralm_cache_update.argtypes = [p, p, i32, i32, p, i32, i32, i32, p, i32, i64, p]
+    lib.ralm_debug_fail_allocation.restype = i32
+    lib.ralm_debug_fail_allocation.argtypes = [i32]
+    lib.ralm_selftest_wait_timeout.restype = i32
+    lib.ralm_selftest_wait_timeout.argtypes = [i64, p, p]
     lib.ralm_device_status.restype = i32
     lib.ralm_device_status.argtypes = [p, p]
     lib.ralm_index_set_variant.restype = i32

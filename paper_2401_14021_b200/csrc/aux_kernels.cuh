@@ -249,6 +249,22 @@ cache_update_kernel(int64_t *__restrict__ cache_ids, int *__restrict__ cursor, i
 }
 
 // ------------------------------------------------------------------------------------
+// Self-test of the bounded waits: a wait on a barrier that nothing ever completes must give up
+// after `limit_cycles`, record the time-out in the status word and return normally.
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(32)
+wait_timeout_selftest_kernel(long long limit_cycles, int *status) {
+    __shared__ uint64_t never;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&never), 1);
+        mbar_fence_init();
+    }
+    __syncwarp();
+    if (threadIdx.x == 0 && !mbar_wait_bounded_for(smem_u32(&never), 0, limit_cycles))
+        atomicMax(status, kStatusTimeout);
+}
+
+// ------------------------------------------------------------------------------------
 // Squared norms of the corpus rows (L2 indexes, once at creation): one warp per row, fp32.
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)

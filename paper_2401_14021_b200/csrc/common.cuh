@@ -69,15 +69,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Every wait is bounded: about two seconds of SM clock, after which the caller records
 // kStatusTimeout and winds down instead of spinning forever.
 constexpr long long kWaitCycleLimit = 4000000000LL;
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_bounded_for(uint32_t bar, uint32_t parity, long long limit_cycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > kWaitCycleLimit) return false;
+        if (clock64() - t0 > limit_cycles) return false;
     }
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    return mbar_wait_bounded_for(bar, parity, kWaitCycleLimit);
 }
 // 1-D bulk copy global -> shared, completion signalled on an mbarrier (no multicast).
 // Both addresses 16-byte aligned, bytes a multiple of 16.

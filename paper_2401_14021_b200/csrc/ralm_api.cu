@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 #include <new>
 #include <utility>
@@ -59,6 +60,20 @@ struct ScanPlan {
 constexpr int kSmemCandBytes = 32 * 1024;  // candidate lists larger than this leave shared memory
 
 int align_up(int v, int a) { return (v + a - 1) / a * a; }
+
+// Every device allocation of the library goes through here, so that a test can make the n-th
+// one fail (ralm_debug_fail_allocation) and check that creation reports it and frees the rest.
+std::atomic<int> g_fail_allocation_in{0};
+template <typename T>
+cudaError_t device_alloc(T **ptr, size_t bytes) {
+    int n = g_fail_allocation_in.load();
+    while (n > 0 && !g_fail_allocation_in.compare_exchange_weak(n, n - 1)) {}
+    if (n == 1) {
+        *ptr = nullptr;
+        return cudaErrorMemoryAllocation;
+    }
+    return cudaMalloc(reinterpret_cast<void **>(ptr), bytes);
+}
 
 // Shared-memory layout of one scan CTA. Returns false if not even two stages fit.
 bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl) {
@@ -200,11 +215,11 @@ bool alloc_tc_workspace(ralm_index *idx, int queries) {
     idx->tc_cand = nullptr;
     idx->tc_cand_q = 0;
     const size_t bytes = sizeof(uint64_t) * idx->num_sms * static_cast<size_t>(queries) * kTcCap;
-    if (!idx->tc_thr && cudaMalloc(&idx->tc_thr, sizeof(float) * idx->max_s) != cudaSuccess) {
+    if (!idx->tc_thr && device_alloc(&idx->tc_thr, sizeof(float) * idx->max_s) != cudaSuccess) {
         idx->tc_thr = nullptr;
         return false;
     }
-    if (cudaMalloc(&idx->tc_cand, bytes) != cudaSuccess) {
+    if (device_alloc(&idx->tc_cand, bytes) != cudaSuccess) {
         idx->tc_cand = nullptr;
         return false;
     }
@@ -529,25 +544,29 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->norms = nullptr;
     idx->spill = nullptr;
     idx->spill_cap = 0;
-    bool ok = cudaMalloc(&idx->partial, partial_bytes) == cudaSuccess;
-    ok = ok && cudaMalloc(&idx->tc_thr, sizeof(float) * max_s) == cudaSuccess;
+    cudaError_t first_error = cudaSuccess;
+    auto alloc = [&first_error](auto **ptr, size_t bytes) {
+        if (first_error == cudaSuccess) first_error = device_alloc(ptr, bytes);
+    };
+    alloc(&idx->partial, partial_bytes);
+    alloc(&idx->tc_thr, sizeof(float) * max_s);
     if (max_k > 1 && std::max(512, 2 * next_pow2(max_k)) * 8 > kSmemCandBytes / kScanMaxQueries) {
         idx->spill_cap = std::max(512, 2 * next_pow2(max_k));
-        ok = ok && cudaMalloc(&idx->spill, sizeof(uint64_t) * idx->num_sms * kScanMaxQueries *
-                                               static_cast<size_t>(idx->spill_cap)) == cudaSuccess;
+        alloc(&idx->spill, sizeof(uint64_t) * idx->num_sms * kScanMaxQueries * static_cast<size_t>(idx->spill_cap));
     }
-    if (metric == RALM_L2 && N > 0) ok = ok && cudaMalloc(&idx->norms, sizeof(float) * N) == cudaSuccess;
-    if (metric == RALM_IP && max_s >= kTcAutoMinQueries && d >= kTcChunkK)
-        ok = ok && alloc_tc_workspace(idx, std::min(kTcMaxQueries, align_up(max_s, 16)));
-    ok = ok && cudaMalloc(&idx->cache_keys, sizeof(uint64_t) * RALM_MAX_CACHE_KEYS) == cudaSuccess;
-    ok = ok && cudaMalloc(&idx->status, sizeof(int)) == cudaSuccess;
-    ok = ok && cudaMalloc(&idx->h_queries, static_cast<size_t>(max_s) * d * 2) == cudaSuccess;
-    ok = ok && cudaMalloc(&idx->h_ids, sk * sizeof(int64_t)) == cudaSuccess;
-    ok = ok && cudaMalloc(&idx->h_scores, sk * sizeof(float)) == cudaSuccess;
-    if (!ok) {
-        const bool oom = cudaGetLastError() == cudaErrorMemoryAllocation;
+    if (metric == RALM_L2 && N > 0) alloc(&idx->norms, sizeof(float) * N);
+    if (metric == RALM_IP && max_s >= kTcAutoMinQueries && d >= kTcChunkK && first_error == cudaSuccess &&
+        !alloc_tc_workspace(idx, std::min(kTcMaxQueries, align_up(max_s, 16))))
+        first_error = cudaErrorMemoryAllocation;
+    alloc(&idx->cache_keys, sizeof(uint64_t) * RALM_MAX_CACHE_KEYS);
+    alloc(&idx->status, sizeof(int));
+    alloc(&idx->h_queries, static_cast<size_t>(max_s) * d * 2);
+    alloc(&idx->h_ids, sk * sizeof(int64_t));
+    alloc(&idx->h_scores, sk * sizeof(float));
+    if (first_error != cudaSuccess) {
+        cudaGetLastError();  // clear the runtime's sticky copy of an allocation failure
         ralm_index_destroy(idx);
-        return oom ? RALM_ERR_OOM : RALM_ERR_CUDA;
+        return first_error == cudaErrorMemoryAllocation ? RALM_ERR_OOM : RALM_ERR_CUDA;
     }
     if (cudaMemset(idx->status, 0, sizeof(int)) != cudaSuccess) {
         ralm_index_destroy(idx);
@@ -661,6 +680,18 @@ ralm_status_t ralm_cache_update(int64_t *cache_ids, int32_t *cursor, int32_t R, 
     cache_update_kernel<<<R, kCacheUpdateThreads, static_cast<size_t>(C) * sizeof(int64_t),
                           static_cast<cudaStream_t>(stream)>>>(cache_ids, cursor, C, retrieved_ids, stride, ld,
                                                                top, steps, next_n, N);
+    return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
+}
+
+ralm_status_t ralm_debug_fail_allocation(int32_t nth) {
+    if (nth < 0) return RALM_ERR_INVALID_ARG;
+    g_fail_allocation_in.store(nth);
+    return RALM_OK;
+}
+
+ralm_status_t ralm_selftest_wait_timeout(int64_t limit_cycles, int32_t *device_status, void *stream) {
+    if (!device_status || limit_cycles < 1 || limit_cycles > 2000000000LL) return RALM_ERR_INVALID_ARG;
+    wait_timeout_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(limit_cycles, device_status);
     return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
 }
 

@@ -179,7 +179,7 @@ def test_argument_errors():
 # ------------------------------------------------------------------ large batches (tcgen05 scan)
 @pytest.mark.parametrize("N,d,s,k", [(1, 64, 1, 1), (129, 72, 3, 1), (300, 128, 9, 64), (1000, 64, 16, 5),
                                      (5000, 768, 100, 20), (257, 64, 257, 2), (3000, 256, 600, 7),
-                                     (2000, 128, 300, 5), (700, 64, 40, 3),
+                                     (2000, 128, 300, 5), (700, 64, 40, 3), (300, 4096, 12, 3),
                                      (40_000, 768, 512, 20)])
 def test_tcgen05_scan_integer_inputs_are_bit_exact(N, d, s, k):
     """The large-batch scan pinned explicitly (variant 3), including shapes with a ragged last
