@@ -238,6 +238,21 @@ ralm_status_t ralm_os3_gamma(const int32_t *matched, const int32_t *strides, int
 ralm_status_t ralm_os3_stride(const int32_t *matched, const int32_t *strides, int32_t w, double gamma_max,
                               double a, double b, int32_t s_max, int32_t async_verify, int32_t *s_out);
 
+/* Row-sharded retrieval (a corpus split by rows over several indexes, on one GPU or one per
+ * GPU): every shard answers the same batch with ralm_search over its own rows; this call merges
+ * the G answers into the answer of C.retrieve over the whole corpus (Algorithm 1, batched
+ * verification step), with the same total order, so the result equals the unsharded search.
+ *   ids        DEVICE int64 [G][s][k]  shard-local row ids as ralm_search wrote them (-1 = padding)
+ *   scores     DEVICE fp32  [G][s][k]
+ *   row_offset DEVICE int64 [G]        global id of each shard's first row
+ *   out_ids    DEVICE int64 [s][k], out_scores DEVICE fp32 [s][k] (written)
+ *   G >= 1, 1 <= k <= RALM_MAX_K; global ids must stay below 2^32. s == 0 is a no-op.
+ * Between GPUs the [G][s][k] arrays are what an all-gather of each rank's [s][k] answer
+ * produces: G * s * k * 12 bytes in all. Needs no index. Asynchronous on `stream`. */
+ralm_status_t ralm_merge_lists(const int64_t *ids, const float *scores, const int64_t *row_offset, int32_t G,
+                               int32_t s, int32_t k, ralm_metric_t metric, int64_t *out_ids, float *out_scores,
+                               void *stream);
+
 /* Testing aids for the failure paths (neither is needed in normal use).
  *
  * ralm_debug_fail_allocation: the nth device allocation the library makes from now on (1 = the

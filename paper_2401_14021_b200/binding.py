@@ -52,6 +52,8 @@ def load_library() -> ctypes.CDLL:
     lib.ralm_verify.argtypes = [p, p, i32, i32, i32, i32, p, p]
     lib.ralm_cache_update.restype = i32
     lib.ralm_cache_update.argtypes = [p, p, i32, i32, p, i32, i32, i32, p, i32, i64, p]
+    lib.ralm_merge_lists.restype = i32
+    lib.ralm_merge_lists.argtypes = [p, p, p, i32, i32, i32, i32, p, p, p]
     lib.ralm_debug_fail_allocation.restype = i32
     lib.ralm_debug_fail_allocation.argtypes = [i32]
     lib.ralm_selftest_wait_timeout.restype = i32
@@ -251,6 +253,25 @@ def cache_update(cache_ids: torch.Tensor, cursor: torch.Tensor, retrieved_ids: t
                                  stride, ld, top, _dev(steps, torch.int32, "steps") if steps is not None else 0,
                                  next_n, N, _stream_ptr(stream)), "ralm_cache_update")
     return cache_ids, cursor
+
+
+def merge_lists(ids: torch.Tensor, scores: torch.Tensor, row_offset: torch.Tensor, metric: int,
+                out_ids: torch.Tensor = None, out_scores: torch.Tensor = None, stream=None):
+    """ralm_merge_lists: ids int64 [G][s][k] (shard-local), scores fp32 [G][s][k], row_offset int64 [G]
+    -> (ids int64 [s][k] global, scores fp32 [s][k])."""
+    lib = load_library()
+    G, s, k = ids.shape
+    if out_ids is None:
+        out_ids = torch.empty((s, k), dtype=torch.int64, device=ids.device)
+    if out_scores is None:
+        out_scores = torch.empty((s, k), dtype=torch.float32, device=ids.device)
+    _check(lib.ralm_merge_lists(_dev(ids, torch.int64, "ids") if s else 0,
+                                _dev(scores, torch.float32, "scores") if s else 0,
+                                _dev(row_offset, torch.int64, "row_offset"), G, s, k, metric,
+                                _dev(out_ids, torch.int64, "out_ids") if s else 0,
+                                _dev(out_scores, torch.float32, "out_scores") if s else 0,
+                                _stream_ptr(stream)), "ralm_merge_lists")
+    return out_ids, out_scores
 
 
 def _i32_array(values):

@@ -86,6 +86,52 @@ merge_kernel(const uint64_t *__restrict__ partial, int B, int s, int k, int l2,
 }
 
 // ------------------------------------------------------------------------------------
+// Merge of G result lists of a row-sharded search: shard g searched its own rows and reports,
+// per query, k (id, score) pairs sorted by the ranking order, ids local to the shard (-1 =
+// padding); row_offset[g] is the global id of the shard's first row. One CTA per query turns
+// the pairs back into ranking keys with global ids and merges them exactly like merge_kernel.
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kMergeThreads, 1)
+merge_lists_kernel(const int64_t *__restrict__ ids, const float *__restrict__ scores,
+                   const int64_t *__restrict__ row_offset, int G, int s, int k, int l2,
+                   int64_t *__restrict__ out_ids, float *__restrict__ out_scores) {
+    __shared__ uint64_t buf[kMergeSortMax];
+    const int q = blockIdx.x;
+    const int tid = threadIdx.x;
+    auto load = [&](int g, int j) -> uint64_t {
+        const size_t at = (static_cast<size_t>(g) * s + q) * k + j;
+        const int64_t id = ids[at];
+        if (id < 0) return 0ull;
+        const float v = l2 ? (0.0f - scores[at]) : scores[at];
+        return make_key(v, static_cast<uint32_t>(id + row_offset[g]));
+    };
+    const long long total = static_cast<long long>(G) * k;
+    if (total <= kMergeSortMax) {
+        const int P = next_pow2(total > 1 ? static_cast<int>(total) : 2);
+        for (int i = tid; i < P; i += kMergeThreads) buf[i] = (i < total) ? load(i / k, i % k) : 0ull;
+        __syncthreads();
+        bitonic_sort_desc(buf, P, tid, kMergeThreads, -1);
+    } else {
+        const int P = next_pow2(k);
+        for (int i = tid; i < P; i += kMergeThreads) buf[i] = (i < k) ? load(0, i) : 0ull;
+        __syncthreads();
+        for (int g = 1; g < G; ++g) {
+            for (int i = tid; i < P; i += kMergeThreads) {
+                const int j = P - 1 - i;
+                const uint64_t other = (j < k) ? load(g, j) : 0ull;
+                const uint64_t mine = buf[i];
+                buf[i] = mine > other ? mine : other;
+            }
+            __syncthreads();
+            bitonic_merge_desc(buf, P, tid, kMergeThreads, -1);
+        }
+    }
+    for (int i = tid; i < k; i += kMergeThreads)
+        write_result((i < total) ? buf[i] : 0ull, l2 != 0, out_ids + static_cast<size_t>(q) * k + i,
+                     out_scores + static_cast<size_t>(q) * k + i);
+}
+
+// ------------------------------------------------------------------------------------
 // Cache lookup, step 1: score. One warp per (request, cache slot); the warp scores its
 // cached corpus row against up to 8 of the request's queries at a time and stores one key
 // per query in keys[r][u][c] (Cp = C rounded up to a power of two; slots >= C hold 0).

@@ -683,6 +683,18 @@ ralm_status_t ralm_cache_update(int64_t *cache_ids, int32_t *cursor, int32_t R, 
     return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
 }
 
+ralm_status_t ralm_merge_lists(const int64_t *ids, const float *scores, const int64_t *row_offset, int32_t G,
+                               int32_t s, int32_t k, ralm_metric_t metric, int64_t *out_ids, float *out_scores,
+                               void *stream) {
+    if (G < 1 || s < 0 || k < 1 || k > RALM_MAX_K || (metric != RALM_IP && metric != RALM_L2))
+        return RALM_ERR_INVALID_ARG;
+    if (s == 0) return RALM_OK;
+    if (!ids || !scores || !row_offset || !out_ids || !out_scores) return RALM_ERR_INVALID_ARG;
+    merge_lists_kernel<<<s, kMergeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        ids, scores, row_offset, G, s, k, metric == RALM_L2, out_ids, out_scores);
+    return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
+}
+
 ralm_status_t ralm_debug_fail_allocation(int32_t nth) {
     if (nth < 0) return RALM_ERR_INVALID_ARG;
     g_fail_allocation_in.store(nth);
