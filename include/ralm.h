@@ -192,7 +192,8 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
  *   the direct sum of squared differences), 3 = tcgen05 scan (inner product, up to 512 queries
  *   per pass, k <= 64, d >= 64; pairs of CTAs share each MMA), 4 = tcgen05 scan with single
  *   CTAs. Automatic: the tcgen05 scan for 9 or more queries where it applies, else warp-MMA.
- * UNSUPPORTED if the variant cannot serve the index's metric or dimension. */
+ * UNSUPPORTED if the variant cannot serve the index's metric or dimension. The environment
+ * variable RALM_FORCE_VARIANT=<1..4> applies the same pin to every index at creation. */
 ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant);
 
 /* Override the scan kernel's launch shape on this index (benchmarking aid; 0 keeps the

@@ -6,6 +6,7 @@
 
 #include <algorithm>
 #include <atomic>
+#include <cstdlib>
 #include <mutex>
 #include <new>
 #include <utility>
@@ -580,6 +581,12 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
             ralm_index_destroy(idx);
             return RALM_ERR_CUDA;
         }
+    }
+    // benchmarking aid: RALM_FORCE_VARIANT=<n> pins the scan variant of every new index, as
+    // ralm_index_set_variant(n) would (ignored when that variant cannot serve the index)
+    if (const char *forced = std::getenv("RALM_FORCE_VARIANT")) {
+        const int v = std::atoi(forced);
+        if (v >= 1 && v <= 4) ralm_index_set_variant(idx, v);
     }
     *out = idx;
     return RALM_OK;

@@ -13,9 +13,15 @@
 //               accumulator is drained while the next is being filled.
 //   warps 2..5  selection: each warp owns one quarter of the TMEM lanes (32 corpus rows),
 //               reads the scores with tcgen05.ld, compares each with its query's threshold
-//               (the CTA's current k-th best) and appends what passes to that query's
-//               candidate list in global memory. Lists are compacted (sorted, cut to k,
-//               threshold raised) by the same warps between units, before they can overflow.
+//               (the CTA's current k-th best, or a better bound handed in by the caller) and
+//               appends what passes to that query's candidate list in global memory. Lists are
+//               compacted (sorted in registers, cut to k, threshold raised) by the same warps
+//               between units, before they can overflow.
+//
+// A launch covers the row tiles [tile0, tile0 + ntiles) and may start from given thresholds:
+// the host scans a small sample of the corpus first, merges it, and starts the main launch
+// from the sample's k-th scores, which makes appends rare (the selection would otherwise, at
+// hundreds of queries, cost more than the MMAs).
 //
 // The kernel is bound by the bytes it stages per MMA, so by default it runs as clusters of two
 // CTAs (cta_group::2): a row tile is then 256 rows, each CTA stages its own 128 rows but only
