@@ -245,6 +245,19 @@ def test_tcgen05_scan_adversarial_row_order():
         check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 64, exact=True)
 
 
+def test_long_rows_take_the_tcgen05_scan_even_for_small_batches():
+    """d = 4096: two 16-row stages of the small-batch scan do not fit in shared memory; inner
+    product indexes then use the large-batch scan (64 columns per stage) for any batch size."""
+    ralm = _ralm()
+    x = workloads.integer_valued((900, 4096), seed=91, lo=-3, hi=3, device=DEV)
+    q = workloads.integer_valued((3, 4096), seed=92, lo=-3, hi=3, device=DEV)
+    ids, scores = _run(x, q, oracle.IP, 4)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 4, exact=True)
+    idx = ralm.Index(x, oracle.L2, 3, 4)                   # L2 has no such route yet
+    with pytest.raises(ralm.RalmError):
+        ralm.search(idx, q, 4)
+
+
 def test_large_k_falls_back_from_the_tcgen05_scan():
     x, _ = workloads.mixture_corpus(30_000, 128, 16, seed=71, device=DEV)
     q, _ = workloads.noisy_copy_queries(x, 20, seed=72)
