@@ -206,20 +206,6 @@ bool encode_rows_map(CUtensorMap *map, const void *base, long long rows, int d, 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// The same rows seen as [rows][d / 16][16]: a box of box_rows x 4 slices x 16 elements lands in
-// shared memory as four blocks of 32-byte rows (32-byte swizzle). Needs d % 16 == 0.
-bool encode_rows_map_sliced(CUtensorMap *map, const void *base, long long rows, int d, int box_rows) {
-    EncodeTiledFn enc = tensor_map_encoder();
-    if (!enc) return false;
-    const cuuint64_t dims[3] = {16, static_cast<cuuint64_t>(rows), static_cast<cuuint64_t>(d / 16)};
-    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2, 32};
-    const cuuint32_t box[3] = {16, static_cast<cuuint32_t>(box_rows), 4};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 bool tc_can_serve(const ralm_index *idx, int k) {
     return idx->metric == RALM_IP && idx->tc_cand != nullptr && k <= kTcMaxK && idx->d >= kTcChunkK;
 }
@@ -261,11 +247,7 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
     p.k = k;
     p.off_stage = align_up(kTcOffEnd, 1024);
     CUtensorMap map_x, map_q;
-    static const bool sw32_env = std::getenv("RALM_TC_SW32") != nullptr;
-    p.sw32 = (sw32_env && idx->d % 16 == 0) ? 1 : 0;
-    if (!(p.sw32 ? encode_rows_map_sliced(&map_x, idx->corpus, idx->N, idx->d, kTcTileM)
-                 : encode_rows_map(&map_x, idx->corpus, idx->N, idx->d, kTcTileM)))
-        return RALM_ERR_CUDA;
+    if (!encode_rows_map(&map_x, idx->corpus, idx->N, idx->d, kTcTileM)) return RALM_ERR_CUDA;
     for (;;) {
         const int group_rows = pair ? 2 * kTcTileM : kTcTileM;
         p.tile0 = row_begin / group_rows;  // row_begin is a multiple of 256
@@ -277,9 +259,7 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
         p.stages = std::min(kTcMaxStages, (idx->smem_optin - p.off_stage) / p.stage_bytes);
         if (p.stages < 2) return RALM_ERR_UNSUPPORTED;
         const int smem = p.off_stage + p.stages * p.stage_bytes;
-        if (!(p.sw32 ? encode_rows_map_sliced(&map_q, queries, sp, idx->d, nb_cta)
-                     : encode_rows_map(&map_q, queries, sp, idx->d, nb_cta)))
-            return RALM_ERR_CUDA;
+        if (!encode_rows_map(&map_q, queries, sp, idx->d, nb_cta)) return RALM_ERR_CUDA;
         if (!pair) {
             const int grid = static_cast<int>(std::min<long long>(idx->num_sms, p.ntiles));
             if (cudaFuncSetAttribute(scan_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=

@@ -72,9 +72,6 @@ struct TcParams {
     int stage_bytes;    // kTcABytes + (staged query rows) * 128, a multiple of 1024
     int off_stage;      // shared-memory offset of the stage ring (1024-byte aligned)
     int cand_q;         // queries the candidate workspace was sized for (>= s)
-    int sw32;           // operand layout in shared memory: 0 = rows of 128 bytes (64 columns) with
-                        // the 128-byte swizzle; 1 = four K slices of rows of 32 bytes (16 columns)
-                        // with the 32-byte swizzle, so that one MMA's operand is contiguous
 };
 
 struct TcHeader {
@@ -102,14 +99,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
         "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
         "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z,
-                                            uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
         : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() {
@@ -140,16 +129,6 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr) {
     desc |= static_cast<uint64_t>(1024 >> 4) << 32; // stride byte offset: next group of 8 rows
     desc |= static_cast<uint64_t>(1) << 46;         // descriptor version of this architecture
     desc |= static_cast<uint64_t>(2) << 61;         // 128-byte swizzle
-    return desc;
-}
-// The same for a K slice stored as rows of 32 bytes with the 32-byte swizzle: groups of 8 rows
-// are 256 bytes apart.
-__device__ __forceinline__ uint64_t tc_smem_desc32(uint32_t addr) {
-    uint64_t desc = (addr & 0x3FFFFu) >> 4;
-    desc |= static_cast<uint64_t>(1) << 16;
-    desc |= static_cast<uint64_t>(256 >> 4) << 32;
-    desc |= static_cast<uint64_t>(1) << 46;
-    desc |= static_cast<uint64_t>(6) << 61;         // 32-byte swizzle
     return desc;
 }
 // Instruction descriptor: fp16 A and B (both K-major), fp32 accumulator, M = m, N = n.
@@ -320,14 +299,6 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(cluster_bar)
         : "memory");
 }
-__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap *map, int x, int y, int z,
-                                                 uint32_t cluster_bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(cluster_bar)
-        : "memory");
-}
 // Arrive on the barrier at this offset in both CTAs of the pair once the MMAs issued so far are done.
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
     asm volatile(
@@ -446,22 +417,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     if (PAIR) {
                         const uint32_t lead_bar = map_to_cta(bar, 0);
                         if (leader) mbar_arrive_expect_tx(bar, stage_tx);
-                        if (p.sw32) {
-                            tma_load_3d_pair(dst, &map_x, 0, row_y, c * 4, lead_bar);
-                            tma_load_3d_pair(dst + kTcABytes, &map_q, 0, query_y, c * 4, lead_bar);
-                        } else {
-                            tma_load_2d_pair(dst, &map_x, c * kTcChunkK, row_y, lead_bar);
-                            tma_load_2d_pair(dst + kTcABytes, &map_q, c * kTcChunkK, query_y, lead_bar);
-                        }
+                        tma_load_2d_pair(dst, &map_x, c * kTcChunkK, row_y, lead_bar);
+                        tma_load_2d_pair(dst + kTcABytes, &map_q, c * kTcChunkK, query_y, lead_bar);
                     } else {
                         mbar_arrive_expect_tx(bar, stage_tx);
-                        if (p.sw32) {
-                            tma_load_3d(dst, &map_x, 0, row_y, c * 4, bar);
-                            tma_load_3d(dst + kTcABytes, &map_q, 0, query_y, c * 4, bar);
-                        } else {
-                            tma_load_2d(dst, &map_x, c * kTcChunkK, row_y, bar);
-                            tma_load_2d(dst + kTcABytes, &map_q, c * kTcChunkK, query_y, bar);
-                        }
+                        tma_load_2d(dst, &map_x, c * kTcChunkK, row_y, bar);
+                        tma_load_2d(dst + kTcABytes, &map_q, c * kTcChunkK, query_y, bar);
                     }
                     ++issued;
                     if (++st == S) {
@@ -509,14 +470,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     const uint32_t b_addr = a_addr + kTcABytes;
 #pragma unroll
                     for (int kk = 0; kk < kTcChunkK / 16; ++kk) {
-                        // K slice kk of the stage: 32 bytes further along the 128-byte rows, or
-                        // the kk-th block of 32-byte rows
-                        const uint64_t a_desc = p.sw32 ? tc_smem_desc32(a_addr + kk * (kTcTileM * 32))
-                                                       : tc_smem_desc(a_addr + kk * 32);
-                        const uint64_t b_desc = p.sw32 ? tc_smem_desc32(b_addr + kk * (nb_cta * 32))
-                                                       : tc_smem_desc(b_addr + kk * 32);
-                        if (PAIR) tc_mma_f16_pair(d_tmem, a_desc, b_desc, idesc, (c | kk) != 0 ? 1u : 0u);
-                        else tc_mma_f16(d_tmem, a_desc, b_desc, idesc, (c | kk) != 0 ? 1u : 0u);
+                        if (PAIR)
+                            tc_mma_f16_pair(d_tmem, tc_smem_desc(a_addr + kk * 32), tc_smem_desc(b_addr + kk * 32),
+                                            idesc, (c | kk) != 0 ? 1u : 0u);
+                        else
+                            tc_mma_f16(d_tmem, tc_smem_desc(a_addr + kk * 32), tc_smem_desc(b_addr + kk * 32),
+                                       idesc, (c | kk) != 0 ? 1u : 0u);
                     }
                     // stage reusable (in both CTAs of a pair) once these MMAs are done
                     if (PAIR) tc_commit_pair(smem_u32(&hdr->empty[st]));
