@@ -368,9 +368,10 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f16 inputs, f32 accumulate", "data": "synthetic",
+            "dtype": "f32", "data": "synthetic",
             "config": {"workload": "%s %dx%d %s s=%d k=%d; cache lookup R=%d C=%d q=%d; verify stride %d"
                                    % (cfg.name, N, d, cfg.metric, s, k, R, cache.shape[1], stride, vstride),
+                       "arithmetic": "fp16 corpus and queries, exact fp16 x fp16 products, fp32 accumulation",
                        "variant": args.variant, "tune": args.tune, "replicas": world,
                        "l2": "inputs larger than L2 (%.1f GB corpus streamed every step)"
                              % (corpus_bytes / 1e9) if corpus_bytes > 2.5e8 else
