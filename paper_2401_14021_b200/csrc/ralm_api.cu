@@ -365,7 +365,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     const int per_pass = mma ? kScanMaxQueries : kFmaQueriesPerPass;
     // k > 1 on a large corpus: scan a sample first and start the rest from the sample's merged
     // k-th scores (see the large-batch path above); the sample's list is block num_sms of `partial`
-    long long sample = std::max<long long>(idx->N / 64, 4LL * idx->num_sms * kTcTileM);
+    // (1/128 of the rows here: measured best for this scan; the large-batch scan prefers 1/64)
+    long long sample = std::max<long long>(idx->N / 128, 4LL * idx->num_sms * kTcTileM);
     sample = (sample + 255) / 256 * 256;
     // (two more launches: only worth it when the scan itself takes a millisecond or more)
     const bool two_phase = k > 1 && idx->tc_thr && idx->tc_two_phase && sample * 32 <= idx->N;

@@ -258,6 +258,18 @@ def test_long_rows_take_the_tcgen05_scan_even_for_small_batches():
         ralm.search(idx, q, 4)
 
 
+def test_largest_batch_and_k_limits_of_the_tcgen05_scan():
+    """RALM_MAX_QUERIES queries in one call (eight passes of 512), and k at the large-batch
+    scan's limit (64) and one beyond it (65, served by the small-batch scan)."""
+    x = workloads.integer_valued((3000, 64), seed=93, lo=-3, hi=3, device=DEV)
+    q = workloads.integer_valued((4096, 64), seed=94, lo=-3, hi=3, device=DEV)
+    ids, scores = _run(x, q, oracle.IP, 3)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 3, exact=True)
+    for k in (64, 65):
+        ids, scores = _run(x, q[:20].contiguous(), oracle.IP, k)
+        check_search(ids, scores, x.cpu().numpy(), q[:20].cpu().numpy(), oracle.IP, k, exact=True)
+
+
 def test_large_k_falls_back_from_the_tcgen05_scan():
     x, _ = workloads.mixture_corpus(30_000, 128, 16, seed=71, device=DEV)
     q, _ = workloads.noisy_copy_queries(x, 20, seed=72)
