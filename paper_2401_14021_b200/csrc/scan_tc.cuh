@@ -463,9 +463,11 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 if (!ok || *abort_flag) break;
                 tc_fence_after();
                 for (int c = 0; c < p.nchunks; ++c) {
+                    // (the mbarrier wait orders the TMA writes before the MMAs that read them; no
+                    // tcgen05 fence here: it is only needed where tcgen05 work of other threads,
+                    // the selection warps' loads, has to be ordered, as above)
                     ok = mbar_wait_bounded(smem_u32(&hdr->full[st]), lap & 1);
                     if (!ok || *abort_flag) break;
-                    tc_fence_after();
                     const uint32_t a_addr = stage_base + static_cast<uint32_t>(st) * p.stage_bytes;
                     const uint32_t b_addr = a_addr + kTcABytes;
 #pragma unroll
