@@ -350,7 +350,8 @@ def main():
                                 if cfg.metric == "ip" and args.variant in (0, 2) and not args.tune
                                 and s <= 8 else None),
                     "traffic_note": "2M-row ncu capture scaled by rows; null if the kernel changed since"}
-        uses_tc = cfg.metric == "ip" and k <= 64 and d >= 64 and (args.variant == 3 or (args.variant == 0 and s >= 9))
+        uses_tc = k <= 64 and d >= 64 and (cfg.metric == "ip" or N >= 700_000) and \
+            (args.variant in (3, 4) or (args.variant == 0 and s >= 9))
         if uses_tc:
             roofline["kernel"] = "scan_tc_kernel"
         if uses_tc and s > 255:

@@ -189,9 +189,11 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
 /* Pin the scan variant used by ralm_search on this index (benchmarking aid).
  *   0 = automatic, 1 = FMA scan (fp32 FMAs, d <= 1024, 4 queries per pass), 2 = warp-MMA scan
  *   (8 queries per pass; for L2 the tensor-core value only filters and the ranked distance is
- *   the direct sum of squared differences), 3 = tcgen05 scan (inner product, up to 512 queries
- *   per pass, k <= 64, d >= 64; pairs of CTAs share each MMA), 4 = tcgen05 scan with single
- *   CTAs. Automatic: the tcgen05 scan for 9 or more queries where it applies, else warp-MMA.
+ *   the direct sum of squared differences), 3 = tcgen05 scan (up to 512 queries per pass, k <= 64,
+ *   d >= 64; pairs of CTAs share each MMA; for L2 the tensor-core value again only filters,
+ *   and the corpus must be large enough to scan a sample first, about 600 K rows), 4 = tcgen05
+ *   scan with single CTAs. Automatic: the tcgen05 scan for 9 or more queries where it applies,
+ *   else warp-MMA.
  * UNSUPPORTED if the variant cannot serve the index's metric or dimension. The environment
  * variable RALM_FORCE_VARIANT=<1..4> applies the same pin to every index at creation. */
 ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant);

@@ -207,7 +207,8 @@ bool encode_rows_map(CUtensorMap *map, const void *base, long long rows, int d, 
 }
 
 bool tc_can_serve(const ralm_index *idx, int k) {
-    return idx->metric == RALM_IP && idx->tc_cand != nullptr && k <= kTcMaxK && idx->d >= kTcChunkK;
+    return (idx->metric == RALM_IP || idx->norms != nullptr) && idx->tc_cand != nullptr && k <= kTcMaxK &&
+           idx->d >= kTcChunkK;
 }
 
 bool alloc_tc_workspace(ralm_index *idx, int queries) {
@@ -232,7 +233,7 @@ bool alloc_tc_workspace(ralm_index *idx, int queries) {
 // MMA (half the query bytes staged per CTA); falls back to single CTAs when no cluster fits.
 ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int s_total, int q0, int k,
                              bool pair, long long row_begin, long long row_end, const float *thr_init,
-                             int *grid_out, cudaStream_t st) {
+                             int mode, int *grid_out, cudaStream_t st) {
     TcParams p;
     p.partial = idx->partial;
     p.cand = idx->tc_cand;
@@ -240,6 +241,12 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
     p.status = idx->status;
     p.N = row_end;
     p.thr_init = thr_init;
+    p.mode = mode;
+    p.d = idx->d;
+    p.slack = static_cast<float>(idx->d) * (1.0f / 2097152.0f);  // as in the small-batch L2 scan
+    p.norms = idx->norms;
+    p.corpus = idx->corpus;
+    p.queries = queries;
     p.nchunks = (idx->d + kTcChunkK - 1) / kTcChunkK;
     p.s = sp;
     p.s_total = s_total;
@@ -313,18 +320,23 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     // whose stages hold 64 columns at a time)
     ScanPlan probe;
     const bool small_scan_fits = plan_scan(idx, true, kScanMaxQueries, k, &probe);
-    const bool tc = tc_can_serve(idx, k) &&
+    // L2 on this path always runs sample first (the sample is what keeps its exact rescoring
+    // rare), so it needs a corpus large enough for one
+    const long long tc_rows = 2 * kTcTileM;
+    long long tc_sample = std::max<long long>(idx->N / 64, 4LL * idx->num_sms * kTcTileM);
+    tc_sample = (tc_sample + tc_rows - 1) / tc_rows * tc_rows;
+    const bool tc_two_phase = tc_sample * 8 <= idx->N && idx->tc_two_phase;
+    const bool l2 = idx->metric == RALM_L2;
+    const bool tc = tc_can_serve(idx, k) && (!l2 || tc_two_phase) &&
                     (idx->variant == 3 || idx->variant == 4 ||
-                     (idx->variant == 0 && (s >= kTcAutoMinQueries || !small_scan_fits)));
+                     (idx->variant == 0 && (s >= kTcAutoMinQueries || (!small_scan_fits && !l2))));
     if (tc) {
         // Large corpora are scanned in two phases: a small sample first, whose merged top-k gives
         // every query a score that k rows are known to reach; the rest then starts from those
         // thresholds, so that hardly any score passes and the selection stays off the critical
         // path. The sample's list rejoins the final merge (block index num_sms of `partial`).
-        const long long group_rows = 2 * kTcTileM;
-        long long sample = std::max<long long>(idx->N / 64, 4LL * idx->num_sms * kTcTileM);
-        sample = (sample + group_rows - 1) / group_rows * group_rows;
-        const bool two_phase = sample * 8 <= idx->N && idx->tc_two_phase;
+        const long long sample = tc_sample;
+        const bool two_phase = tc_two_phase;
         int grid = 0;
         const int per_pass = std::min(kTcMaxQueries, idx->tc_cand_q);
         for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
@@ -335,7 +347,10 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             ralm_status_t rs = RALM_OK;
             if (two_phase) {
                 int grid1 = 0;
-                rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, sample, nullptr, &grid1, st);
+                // L2: the sample is ranked by lower bounds of the tensor-core value and only yields
+                // thresholds; its rows are scanned again, exactly, by the main launch
+                rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, sample, nullptr, l2 ? 1 : 0,
+                                    &grid1, st);
                 if (rs == RALM_OK) {
                     merge_kernel<<<sp, kMergeThreads, 0, st>>>(
                         idx->partial + static_cast<size_t>(q0) * k, grid1, s, k, 0, nullptr, nullptr,
@@ -343,18 +358,18 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
                     if (cudaGetLastError() != cudaSuccess) rs = RALM_ERR_CUDA;
                 }
                 if (rs == RALM_OK)
-                    rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, sample, idx->N, idx->tc_thr,
-                                        &grid, st);
+                    rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, l2 ? 0 : sample, idx->N,
+                                        idx->tc_thr, l2 ? 2 : 0, &grid, st);
                 idx->launches += 2;
             } else {
-                rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, idx->N, nullptr, &grid, st);
+                rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, idx->N, nullptr, 0, &grid, st);
             }
             timing_end(idx, st, ev);
             if (rs != RALM_OK) return rs;
             idx->launches++;
         }
-        merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, 0, ids, scores, nullptr, nullptr,
-                                                  two_phase ? idx->num_sms : -1);
+        merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, l2 ? 1 : 0, ids, scores, nullptr, nullptr,
+                                                  (two_phase && !l2) ? idx->num_sms : -1);
         if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
         idx->launches++;
         return RALM_OK;
@@ -564,7 +579,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     if (metric == RALM_L2 && N > 0) alloc(&idx->norms, sizeof(float) * N);
     ScanPlan probe;
     const bool small_scan_fits = plan_scan(idx, true, kScanMaxQueries, 1, &probe);
-    if (metric == RALM_IP && (max_s >= kTcAutoMinQueries || !small_scan_fits) && d >= kTcChunkK &&
+    if ((max_s >= kTcAutoMinQueries || (!small_scan_fits && metric == RALM_IP)) && d >= kTcChunkK &&
         first_error == cudaSuccess &&
         !alloc_tc_workspace(idx, std::min(kTcMaxQueries, align_up(max_s, 16))))
         first_error = cudaErrorMemoryAllocation;
@@ -740,7 +755,8 @@ ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant) {
     if (!idx || variant < 0 || variant > 4) return RALM_ERR_INVALID_ARG;
     if (variant == 1 && idx->d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
     if (variant == 3 || variant == 4) {
-        if (idx->metric != RALM_IP || idx->d < kTcChunkK || !tensor_map_encoder()) return RALM_ERR_UNSUPPORTED;
+        if ((idx->metric != RALM_IP && !idx->norms) || idx->d < kTcChunkK || !tensor_map_encoder())
+            return RALM_ERR_UNSUPPORTED;
         if (!alloc_tc_workspace(idx, std::min(kTcMaxQueries, align_up(idx->max_s, 16)))) return RALM_ERR_OOM;
     }
     idx->variant = variant;

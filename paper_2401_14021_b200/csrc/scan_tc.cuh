@@ -1,4 +1,5 @@
-// Corpus scan for large query batches (inner product, up to 512 queries per pass) on the
+// Corpus scan for large query batches (up to 512 queries per pass; inner product, and L2 through
+// the same inner-product tiles, see TcParams::mode) on the
 // fifth-generation tensor cores: scores = corpus tile [128 rows] x queries^T [up to 256] with
 // tcgen05.mma, fp16 operands, fp32 accumulators in tensor memory (TMEM), fused with the
 // per-CTA top-k selection so that the N x s score matrix never exists in memory.
@@ -72,6 +73,19 @@ struct TcParams {
     int stage_bytes;    // kTcABytes + (staged query rows) * 128, a multiple of 1024
     int off_stage;      // shared-memory offset of the stage ring (1024-byte aligned)
     int cand_q;         // queries the candidate workspace was sized for (>= s)
+    // L2 (squared distance) on the same inner-product tiles. mode 0: inner product. The tensor-
+    // core value v = 2 x.q - |x|^2 - |q|^2 = -distance^2 cancels, so it is never ranked:
+    // mode 1 (sample launch): keys are the LOWER BOUNDS v - slack (|x|^2 + |q|^2); their merged
+    //         k-th value is a rank value that k rows are known to reach;
+    // mode 2 (main launch, over all rows): a pair passes the filter when v + slack (|x|^2 + |q|^2)
+    //         reaches the threshold, and is then scored again in the direct sum-of-squared-
+    //         differences form from global memory; only that value is ranked and returned.
+    int mode;
+    int d;
+    float slack;
+    const float *norms;      // |x|^2 of every corpus row (fp32)
+    const __half *corpus;    // the rows and queries themselves, for the direct form
+    const __half *queries;   // [s][d] of this pass
 };
 
 struct TcHeader {
@@ -90,7 +104,8 @@ static_assert(sizeof(TcHeader) <= kTcHeaderBytes, "header too large");
 constexpr int kTcOffThr = kTcHeaderBytes;                      // float [512]
 constexpr int kTcOffCnt = kTcOffThr + kTcMaxQueries * 4;       // int [512]
 constexpr int kTcOffSorted = kTcOffCnt + kTcMaxQueries * 4;    // int [512]
-constexpr int kTcOffEnd = kTcOffSorted + kTcMaxQueries * 4;
+constexpr int kTcOffQn = kTcOffSorted + kTcMaxQueries * 4;      // float [512]: |q|^2 (L2)
+constexpr int kTcOffEnd = kTcOffQn + kTcMaxQueries * 4;
 
 // ---- tcgen05 / TMA wrappers -------------------------------------------------------------
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
@@ -272,6 +287,99 @@ __device__ __noinline__ void tc_append_chunk(uint32_t taddr, const float *thr_ch
     }
 }
 
+// Squared distance between one corpus row and one query, both read from global memory (the row
+// has just passed through L2, the queries live there), by the whole warp in the direct
+// sum-of-squared-differences form. Every lane returns the full sum.
+__device__ __forceinline__ float tc_direct_l2(const __half *row, const __half *query, int d, int lane) {
+    float2 sum = make_float2(0.f, 0.f);
+    for (int piece = lane; piece * 8 < d; piece += 32) {
+        const uint4 xr = __ldg(reinterpret_cast<const uint4 *>(row) + piece);
+        const uint4 qr = __ldg(reinterpret_cast<const uint4 *>(query) + piece);
+        const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
+        const uint32_t qw[4] = {qr.x, qr.y, qr.z, qr.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float2 x = __half22float2(*reinterpret_cast<const __half2 *>(&xw[e]));
+            const float2 q = __half22float2(*reinterpret_cast<const __half2 *>(&qw[e]));
+            const float dx = x.x - q.x, dy = x.y - q.y;
+            sum.x = fmaf(dx, dx, sum.x);
+            sum.y = fmaf(dy, dy, sum.y);
+        }
+    }
+    float v = sum.x + sum.y;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// The rare part of the selection for L2 (see tc_append_chunk for the appending itself).
+// bound_sign = -1: sample launch, the value kept is the lower bound; +1: main launch, pairs that
+// pass the filter are scored again in the direct form and kept only if that value passes.
+__device__ __noinline__ void tc_append_chunk_l2(uint32_t taddr, const float *thr_chunk, const float *qn_chunk,
+                                                int *cnt_chunk, uint64_t *cand_chunk, uint32_t row, bool row_ok,
+                                                float nx, float slack, float bound_sign, const __half *corpus,
+                                                const __half *queries_chunk, int d, volatile int *dirty,
+                                                int lane) {
+    uint32_t v[32];
+    tmem_ld32(taddr, v);
+    uint32_t hit = 0;
+#pragma unroll
+    for (int b = 0; b < 32; ++b) {
+        const float s2 = nx + qn_chunk[b];
+        const float val = fmaf(2.0f, __uint_as_float(v[b]), 0.0f - s2);
+        const float bound = fmaf(bound_sign * slack, s2, val);
+        hit |= (bound >= thr_chunk[b] ? 1u : 0u) << b;
+        v[b] = __float_as_uint(bound);      // what the sample launch ranks
+    }
+    if (!row_ok) hit = 0;
+    uint32_t any_col = __reduce_or_sync(0xffffffffu, hit);
+    if (bound_sign > 0.0f) {
+#pragma unroll
+        for (int b = 0; b < 32; ++b) {
+            if (any_col & (1u << b)) {
+                unsigned m = __ballot_sync(0xffffffffu, (hit >> b) & 1u);
+                while (m) {
+                    const int src = __ffs(m) - 1;
+                    m &= m - 1;
+                    const uint32_t row_src = __shfl_sync(0xffffffffu, row, src);
+                    const float dist = tc_direct_l2(corpus + static_cast<size_t>(row_src) * d,
+                                                    queries_chunk + static_cast<size_t>(b) * d, d, lane);
+                    if (lane == src) {
+                        const float exact = 0.0f - dist;
+                        v[b] = __float_as_uint(exact);
+                        if (!(exact >= thr_chunk[b])) hit &= ~(1u << b);
+                    }
+                }
+            }
+        }
+        any_col = __reduce_or_sync(0xffffffffu, hit);
+    }
+    uint32_t mine = 0;
+#pragma unroll
+    for (int b = 0; b < 32; ++b) {
+        if (any_col & (1u << b)) {
+            const uint32_t m = __ballot_sync(0xffffffffu, (hit >> b) & 1u);
+            if (lane == b) mine = m;
+        }
+    }
+    int base = 0;
+    if (mine) {
+        base = atomicAdd(&cnt_chunk[lane], __popc(mine));
+        if (base + __popc(mine) >= kTcSoft) *dirty = 1;
+    }
+    const uint32_t below = (1u << lane) - 1u;
+#pragma unroll
+    for (int b = 0; b < 32; ++b) {
+        if (any_col & (1u << b)) {
+            const int base_b = __shfl_sync(0xffffffffu, base, b);
+            const uint32_t rows_b = __shfl_sync(0xffffffffu, mine, b);
+            if ((hit >> b) & 1u)
+                cand_chunk[static_cast<size_t>(b) * kTcCap + base_b + __popc(rows_b & below)] =
+                    make_key(__uint_as_float(v[b]), row);
+        }
+    }
+}
+
 // ---- CTA-pair helpers (PAIR = true: two CTAs of a cluster work as one MMA unit) -----------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
@@ -361,6 +469,20 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         thr[q] = (q < p.s) ? (p.thr_init ? p.thr_init[p.q_base + q] : -INFINITY) : INFINITY;
         cnt[q] = 0;
         sorted[q] = 0;
+    }
+    float *qn = reinterpret_cast<float *>(tc_smem + kTcOffQn);
+    if (p.mode != 0) {
+        for (int q = threadIdx.x; q < kTcMaxQueries; q += kTcThreads) {
+            float acc = 0.f;
+            if (q < p.s) {
+                const __half *qv = p.queries + static_cast<size_t>(q) * p.d;
+                for (int i = 0; i < p.d; ++i) {
+                    const float a = __half2float(qv[i]);
+                    acc = fmaf(a, a, acc);
+                }
+            }
+            qn[q] = acc;
+        }
     }
     if (warp == 1) {
         if (PAIR) {
@@ -533,7 +655,33 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const bool row_ok = row < p.N;
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                        static_cast<uint32_t>(acc * kTcMaxN);
-                for (int j = 0; j * 32 < nq; ++j) {
+                const float nx = (p.mode != 0 && row_ok) ? __ldg(p.norms + row) : 0.f;
+                const float bound_sign = p.mode == 1 ? -1.0f : 1.0f;
+                for (int j = 0; p.mode != 0 && j * 32 < nq; ++j) {
+                    // L2: the same loop on the bound of -distance^2 (see TcParams::mode)
+                    uint32_t v[32];
+                    tmem_ld32(t_row + j * 32, v);
+                    const float4 *t4 = reinterpret_cast<const float4 *>(thr + qb + j * 32);
+                    const float4 *n4 = reinterpret_cast<const float4 *>(qn + qb + j * 32);
+                    const float sl = bound_sign * p.slack;
+                    bool p0 = false, p1 = false, p2 = false, p3 = false;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 th = t4[i];
+                        const float4 nq4 = n4[i];
+                        const float s0 = nx + nq4.x, s1 = nx + nq4.y, s2 = nx + nq4.z, s3 = nx + nq4.w;
+                        p0 |= fmaf(sl, s0, fmaf(2.0f, __uint_as_float(v[4 * i + 0]), 0.0f - s0)) >= th.x;
+                        p1 |= fmaf(sl, s1, fmaf(2.0f, __uint_as_float(v[4 * i + 1]), 0.0f - s1)) >= th.y;
+                        p2 |= fmaf(sl, s2, fmaf(2.0f, __uint_as_float(v[4 * i + 2]), 0.0f - s2)) >= th.z;
+                        p3 |= fmaf(sl, s3, fmaf(2.0f, __uint_as_float(v[4 * i + 3]), 0.0f - s3)) >= th.w;
+                    }
+                    if (__any_sync(0xffffffffu, row_ok && (p0 | p1 | p2 | p3)))
+                        tc_append_chunk_l2(t_row + j * 32, thr + qb + j * 32, qn + qb + j * 32, cnt + qb + j * 32,
+                                           my_cand + static_cast<size_t>(qb + j * 32) * kTcCap,
+                                           static_cast<uint32_t>(row), row_ok, nx, p.slack, bound_sign, p.corpus,
+                                           p.queries + static_cast<size_t>(qb + j * 32) * p.d, p.d, dirty, lane);
+                }
+                for (int j = 0; p.mode == 0 && j * 32 < nq; ++j) {
                     uint32_t v[32];
                     tmem_ld32(t_row + j * 32, v);
                     const float4 *t4 = reinterpret_cast<const float4 *>(thr + qb + j * 32);

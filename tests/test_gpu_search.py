@@ -172,8 +172,10 @@ def test_argument_errors():
     with pytest.raises(ralm.RalmError):
         idx.set_variant(7)
     l2 = ralm.Index(x, oracle.L2, 2, 5)
+    l2.set_variant(3)                     # (small corpora still take the small-batch scan)
+    narrow = ralm.Index(workloads.unit_gaussian_corpus(100, 32, seed=6, device=DEV), oracle.IP, 2, 5)
     with pytest.raises(ralm.RalmError):
-        l2.set_variant(3)                 # the tcgen05 scan cannot serve L2
+        narrow.set_variant(3)             # the tcgen05 scan needs d >= 64
 
 
 # ------------------------------------------------------------------ large batches (tcgen05 scan)
@@ -218,6 +220,28 @@ def test_tcgen05_scan_two_phases_integer_inputs():
         for variant in (3, 4):
             ids, scores = _run(x, q, oracle.IP, k, variant)
             check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+    # L2 on the same scan: the sample launch ranks lower bounds of the tensor-core value, the main
+    # launch filters with it and scores what passes in the direct form
+    q = workloads.integer_valued((40, d), seed=79, lo=-2, hi=2, device=DEV)
+    for variant in (3, 4):
+        ids, scores = _run(x, q, oracle.L2, 5, variant)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, 5, exact=True)
+
+
+def test_tcgen05_scan_l2_parity_and_duplicates():
+    """Unnormalised rows with log-normal norms (the KNN-LM datastore's shape), 64 queries, L2."""
+    N, d, s, k = 700_000, 128, 64, 20
+    x, _ = workloads.mixture_corpus(N, d, 256, seed=95, device=DEV, normalise=False, lognormal_sigma=0.3)
+    q, src = workloads.noisy_copy_queries(x, s, seed=96)
+    q[:4] = x[src[:4]]                                   # exact copies: distance exactly 0, ranked first
+    ids, scores = _run(x, q, oracle.L2, k)               # 64 queries: the large-batch scan by itself
+    strict, band = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, k)
+    assert ids[:, 0].tolist() == src.tolist()
+    assert (scores[:4, 0] == 0).all()
+    ids8, scores8 = _run(x, q, oracle.L2, k, 2)          # eight queries per pass on the same batch
+    assert torch.equal(ids[:, 0], ids8[:, 0])
+    torch.testing.assert_close(scores, scores8, rtol=1e-4, atol=1e-4)
+    print("L2 large batch: strict=%d band=%d" % (strict, band))
 
 
 @pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
