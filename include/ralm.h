@@ -69,8 +69,11 @@ typedef enum {
  *   max_s   largest number of queries a later ralm_search will pass (1..RALM_MAX_QUERIES).
  *   max_k   largest k a later call will pass (1..RALM_MAX_K).
  *   out     receives the handle (host memory owned by the library).
- * Allocates the per-index device workspace (partial top-k lists, staging buffers, status
- * word) on the current device. Synchronous.
+ * Allocates the per-index device workspace on the current device: partial top-k lists, staging
+ * buffers, a status word; for L2 the squared norm of every row (4 N bytes, computed here in one
+ * pass over the corpus); for max_k > 256 spilled candidate lists (about 19 MB at k = 1024); for
+ * max_s >= 9 the candidate lists of the large-batch scan (about 300 KB per query, 155 MB at 512
+ * queries). Synchronous.
  * Errors: INVALID_ARG (null pointer, misaligned corpus, bad sizes), OOM, CUDA,
  * UNSUPPORTED (device is not compute capability 10.x). */
 ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_metric_t metric,

@@ -153,5 +153,16 @@ def test_c4_full_size_l2_k1024():
     strict, band, n_sub = _sampled_parity(x, q, ids, scores, oracle.L2, 1024, 14, 16_384, seed=3400)
     print("C4: strict=%d band=%d over a %d-row sub-corpus" % (strict, band, n_sub))
     idx.close()
+    # 64 concurrent queries, k = 20: L2 on the large-batch scan (lower-bound sample, filter, rescoring)
+    q64, src64 = workloads.noisy_copy_queries(x, 64, workloads.seed_for(4, "queries") + 5)
+    idx = ralm.Index(x, oracle.L2, max_s=64, max_k=20)
+    ids, scores = ralm.search(idx, q64, 20)
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    assert ids[:, 0].tolist() == src64.tolist()
+    strict, band, n_sub = _sampled_parity(x, q64, ids, scores, oracle.L2, 20, 6, 16_384, seed=3450,
+                                          query_sel=range(0, 64, 4))
+    print("C4, 64 queries: strict=%d band=%d over a %d-row sub-corpus, 16 of 64 queries" % (strict, band, n_sub))
+    idx.close()
     del x
     torch.cuda.empty_cache()
