@@ -14,17 +14,23 @@
 //     the direct sum-of-squared-differences form, which has no cancellation).
 //   warp-MMA flavour: m16n8k16 tensor-core tiles with the 16 corpus rows as M and the (up
 //     to) 8 queries as N, fp32 accumulators. The k index is permuted (the same way for rows
-//     and queries) so that each lane reads 16 contiguous bytes per row. For L2 the tensor
-//     cores also give the rows' squared norms (diagonals of rows x rows products) and
-//     |x|^2 - 2 x.q + |q|^2 serves as a conservative filter; every pair that passes is scored
-//     again in the direct form, and only that value is ranked and returned.
+//     and queries) so that each lane reads 16 contiguous bytes per row. For L2 the rows'
+//     squared norms come from the index (or, without one, from the tensor cores: diagonals
+//     of rows x rows products) and |x|^2 - 2 x.q + |q|^2 serves as a conservative filter;
+//     every pair that passes is scored again from the staged tile in the direct form, and
+//     only that value is ranked and returned.
 //
 // Selection: k == 1 keeps a running best key per thread. k > 1 uses a per-query threshold
-// (the current k-th best of this CTA) and a shared-memory candidate buffer. A push that lands
-// near the end of a buffer raises a flag; every consumer warp polls the flag while it waits
-// for a tile and all of them meet to compact (sort, keep k, raise the threshold) the buffers,
-// spread over the warps, before any buffer can overflow: after the flag is up each warp
-// pushes at most the rest of the tile it is on.
+// (the current k-th best of this CTA, or a better bound handed in by the caller) and a
+// candidate buffer, in shared memory or, when large, in global memory with one shared sort
+// scratch. A push that lands beyond the buffer's soft limit raises a flag; every consumer warp
+// polls the flag while it waits for a tile and all of them meet to compact (sort, keep k, raise
+// the threshold) the buffers, spread over the warps, before any buffer can overflow: after the
+// flag is up each warp pushes at most the rest of the tile it is on.
+//
+// A launch covers the rows [row_begin, N) and may start from given thresholds: on large corpora
+// the host scans a sample first, merges it, and starts the main launch from the sample's k-th
+// values, so that few rows pass.
 #pragma once
 
 #include "common.cuh"
