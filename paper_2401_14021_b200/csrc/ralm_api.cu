@@ -89,7 +89,9 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
     }
     pl->stage_bytes = align_up(pl->tile_rows * idx->d * 2, 128);
     pl->off_q = kScanHeaderBytes;
-    int off = pl->off_q + (mma ? align_up(kScanMaxQueries * (idx->d * 2 + kQueryPadBytes), 128) : 0);
+    // (the warp-MMA flavour stages 8 query rows, or 16 when a pass carries more than 8)
+    const int q_rows = s_pass > kScanMaxQueries ? kScanMaxPassQueries : kScanMaxQueries;
+    int off = pl->off_q + (mma ? align_up(q_rows * (idx->d * 2 + kQueryPadBytes), 128) : 0);
     pl->off_cand = off;
     pl->cap = 0;
     pl->soft_limit = 0;
@@ -311,7 +313,8 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
     }
 }
 
-constexpr int kTcAutoMinQueries = 9;  // batches the 8-query scan cannot serve in one pass
+constexpr int kTcAutoMinQueries = 9;     // batches the 8-query scan cannot serve in one pass
+constexpr int kTcAutoMinQueriesIp = 17;  // inner product: the small-batch scan takes 16 in one pass
 
 ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k, int64_t *ids,
                             float *scores, cudaStream_t st) {
@@ -329,7 +332,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     const bool l2 = idx->metric == RALM_L2;
     const bool tc = tc_can_serve(idx, k) && (!l2 || tc_two_phase) &&
                     (idx->variant == 3 || idx->variant == 4 ||
-                     (idx->variant == 0 && (s >= kTcAutoMinQueries || (!small_scan_fits && !l2))));
+                     (idx->variant == 0 &&
+                      (s >= (l2 ? kTcAutoMinQueries : kTcAutoMinQueriesIp) || (!small_scan_fits && !l2))));
     if (tc) {
         // Large corpora are scanned in two phases: a small sample first, whose merged top-k gives
         // every query a score that k rows are known to reach; the rest then starts from those
@@ -377,7 +381,10 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     const int variant = resolve_variant(idx);
     const bool mma = variant == 2;
     if (!mma && idx->d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
-    const int per_pass = mma ? kScanMaxQueries : kFmaQueriesPerPass;
+    // inner product on the warp-MMA flavour: two groups of 8 queries share every staged tile
+    // when the batch has more than 8 (the tile is read from shared memory twice, from HBM once)
+    const bool wide = mma && idx->metric == RALM_IP && s > kScanMaxQueries;
+    const int per_pass = mma ? (wide ? kScanMaxPassQueries : kScanMaxQueries) : kFmaQueriesPerPass;
     // k > 1 on a large corpus: scan a sample first and start the rest from the sample's merged
     // k-th scores (see the large-batch path above); the sample's list is block num_sms of `partial`
     // (1/128 of the rows here: measured best for this scan; the large-batch scan prefers 1/64)
@@ -430,6 +437,9 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             if (mma && idx->metric == RALM_L2)
                 return (k == 1) ? launch_scan<true, true, 8, 1, true>(p, g, pl.smem_bytes, st)
                                 : launch_scan<true, true, 8, 1, false>(p, g, pl.smem_bytes, st);
+            if (mma && sp > kScanMaxQueries)
+                return (k == 1) ? launch_scan<true, false, 16, 1, true>(p, g, pl.smem_bytes, st)
+                                : launch_scan<true, false, 16, 1, false>(p, g, pl.smem_bytes, st);
             if (mma)
                 return (k == 1) ? launch_scan<true, false, 8, 1, true>(p, g, pl.smem_bytes, st)
                                 : launch_scan<true, false, 8, 1, false>(p, g, pl.smem_bytes, st);
@@ -572,9 +582,10 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     };
     alloc(&idx->partial, partial_bytes);
     alloc(&idx->tc_thr, sizeof(float) * max_s);
-    if (max_k > 1 && std::max(512, 2 * next_pow2(max_k)) * 8 > kSmemCandBytes / kScanMaxQueries) {
+    const int pass_queries = std::min(max_s, metric == RALM_IP ? kScanMaxPassQueries : kScanMaxQueries);
+    if (max_k > 1 && std::max(512, 2 * next_pow2(max_k)) * 8 * pass_queries > kSmemCandBytes) {
         idx->spill_cap = std::max(512, 2 * next_pow2(max_k));
-        alloc(&idx->spill, sizeof(uint64_t) * idx->num_sms * kScanMaxQueries * static_cast<size_t>(idx->spill_cap));
+        alloc(&idx->spill, sizeof(uint64_t) * idx->num_sms * kScanMaxPassQueries * static_cast<size_t>(idx->spill_cap));
     }
     if (metric == RALM_L2 && N > 0) alloc(&idx->norms, sizeof(float) * N);
     ScanPlan probe;

@@ -39,7 +39,8 @@ namespace ralm {
 
 constexpr int kMaxStages = 24;
 constexpr int kMaxConsumerWarps = 8;
-constexpr int kScanMaxQueries = 8;
+constexpr int kScanMaxQueries = 8;       // queries of one MMA group (the N of m16n8k16)
+constexpr int kScanMaxPassQueries = 16;  // queries per pass: two groups in the inner-product warp-MMA flavour
 constexpr int kScanThreads = 32 * (kMaxConsumerWarps + 1);
 constexpr int kQueryPadBytes = 64;
 
@@ -76,9 +77,9 @@ struct ScanParams {
 struct ScanHeader {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
-    unsigned long long best[kScanMaxQueries];
-    float thr[kScanMaxQueries];
-    int cnt[kScanMaxQueries];
+    unsigned long long best[kScanMaxPassQueries];
+    float thr[kScanMaxPassQueries];
+    int cnt[kScanMaxPassQueries];
     int abort;
     int flag;  // some query's candidate buffer is nearly full: everyone meet and compact
     int done;  // consumer warps that have finished their tiles
@@ -118,10 +119,10 @@ __device__ inline void compact_query(ScanHeader *hdr, uint64_t *cand, uint64_t *
 // called by all W * 32 consumer threads, with no push in flight.
 __device__ inline void compact_all(ScanHeader *hdr, uint64_t *cand, uint64_t *scratch, int cap, int s,
                                    int k, int min_count, int w, int lane, int W) {
-    int list[kScanMaxQueries];
+    int list[kScanMaxPassQueries];
     int nq = 0;
 #pragma unroll
-    for (int q = 0; q < kScanMaxQueries; ++q)
+    for (int q = 0; q < kScanMaxPassQueries; ++q)
         if (q < s && hdr->cnt[q] > min_count) list[nq++] = q;
     // nobody may start rewriting cnt[] before everybody has taken the same snapshot of it
     named_barrier(1, W * 32);
@@ -136,7 +137,7 @@ __device__ inline void compact_all(ScanHeader *hdr, uint64_t *cand, uint64_t *sc
     for (int i = group; i < nq; i += ngroups) {
         int q = 0;
 #pragma unroll
-        for (int j = 0; j < kScanMaxQueries; ++j)
+        for (int j = 0; j < kScanMaxPassQueries; ++j)
             if (j == i) q = list[j];
         compact_query(hdr, cand, scratch, cap, q, k, tid, G * 32, bar_id);
     }
@@ -237,7 +238,7 @@ scan_kernel(const ScanParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     ScanHeader *hdr = reinterpret_cast<ScanHeader *>(smem);
     uint64_t *scratch = p.spill ? reinterpret_cast<uint64_t *>(smem + p.off_cand) : nullptr;
-    uint64_t *cand = p.spill ? p.spill + static_cast<size_t>(blockIdx.x) * kScanMaxQueries * p.cap
+    uint64_t *cand = p.spill ? p.spill + static_cast<size_t>(blockIdx.x) * kScanMaxPassQueries * p.cap
                              : reinterpret_cast<uint64_t *>(smem + p.off_cand);
     const int W = p.nwarps;
     const int S = W * p.depth;
@@ -256,7 +257,7 @@ scan_kernel(const ScanParams p) {
         hdr->flag = 0;
         hdr->done = 0;
     }
-    if (threadIdx.x < kScanMaxQueries) {
+    if (threadIdx.x < kScanMaxPassQueries) {
         hdr->thr[threadIdx.x] = (p.thr_init && threadIdx.x < p.s) ? p.thr_init[p.q_base + threadIdx.x] : -INFINITY;
         hdr->cnt[threadIdx.x] = 0;
         hdr->best[threadIdx.x] = 0ull;
@@ -266,7 +267,7 @@ scan_kernel(const ScanParams p) {
         // kQueryPadBytes so that the eight query rows do not all start on the same bank
         const uint4 *qg = reinterpret_cast<const uint4 *>(p.queries);
         const int per_row = d / 8;
-        for (int i = threadIdx.x; i < kScanMaxQueries * per_row; i += blockDim.x) {
+        for (int i = threadIdx.x; i < (MMA ? SQ : kScanMaxQueries) * per_row; i += blockDim.x) {
             const int row = i / per_row, col = i - row * per_row;
             *reinterpret_cast<uint4 *>(smem + p.off_q + row * (d * 2 + kQueryPadBytes) + col * 16) =
                 (row < p.s) ? qg[i] : make_uint4(0, 0, 0, 0);
@@ -336,7 +337,11 @@ scan_kernel(const ScanParams p) {
         const int cthreads = W * 32;
         const int g = lane >> 2, t = lane & 3;
 
-        uint64_t best0 = 0, best1 = 0;
+        // inner-product warp-MMA flavour: SQ / 8 groups of 8 queries share every tile
+        constexpr int NG = (MMA && !L2) ? SQ / 8 : 1;
+        uint64_t bestA[NG], bestB[NG];
+#pragma unroll
+        for (int grp = 0; grp < NG; ++grp) bestA[grp] = bestB[grp] = 0;
         // FMA flavour: this lane's slice of every query as fp32 pairs (negated for L2 so
         // that the difference is one packed add)
         constexpr int DPR = MMA ? 1 : DP;
@@ -438,8 +443,11 @@ scan_kernel(const ScanParams p) {
                 // ---- 16 rows x 8 queries on tensor cores; two accumulator sets halve the
                 // dependent chain. For L2 two more products per step, rows x rows, put the
                 // rows' squared norms on the diagonals of nlo (rows 0..7) and nhi (rows 8..15).
-                float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                float acc_b[4] = {0.f, 0.f, 0.f, 0.f};
+                float acc[NG][4], acc_b[NG][4];
+#pragma unroll
+                for (int grp = 0; grp < NG; ++grp)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[grp][i] = acc_b[grp][i] = 0.f;
                 float nlo[4] = {0.f, 0.f, 0.f, 0.f}, nlo_b[4] = {0.f, 0.f, 0.f, 0.f};
                 float nhi[4] = {0.f, 0.f, 0.f, 0.f}, nhi_b[4] = {0.f, 0.f, 0.f, 0.f};
                 const int nchunks = (d + 31) >> 5;
@@ -451,14 +459,18 @@ scan_kernel(const ScanParams p) {
                     // logical k (2t, 2t+1, 2t+8, 2t+9 of two MMAs) <- physical halves
                     // off..off+7, the same permutation for every row and query
                     const int off = c * 32 + t * 8;
-                    uint4 b = make_uint4(0, 0, 0, 0), lo = b, hi = b;
+                    uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
                     if (off < d) {  // ragged last chunk: absent pieces stay zero
-                        b = lds128(q_addr + off * 2);
                         lo = lds128(a_lo_addr + off * 2);
                         hi = lds128(a_hi_addr + off * 2);
                     }
-                    mma_m16n8k16(acc, lo.x, hi.x, lo.y, hi.y, b.x, b.y);
-                    mma_m16n8k16(acc_b, lo.z, hi.z, lo.w, hi.w, b.z, b.w);
+#pragma unroll
+                    for (int grp = 0; grp < NG; ++grp) {
+                        uint4 b = make_uint4(0, 0, 0, 0);
+                        if (off < d) b = lds128(q_addr + grp * kScanMaxQueries * q_pitch + off * 2);
+                        mma_m16n8k16(acc[grp], lo.x, hi.x, lo.y, hi.y, b.x, b.y);
+                        mma_m16n8k16(acc_b[grp], lo.z, hi.z, lo.w, hi.w, b.z, b.w);
+                    }
                     if (L2 && !NRM) {
                         mma_m16n8k16(nlo, lo.x, hi.x, lo.y, hi.y, lo.x, lo.y);
                         mma_m16n8k16(nhi, lo.x, hi.x, lo.y, hi.y, hi.x, hi.y);
@@ -467,7 +479,9 @@ scan_kernel(const ScanParams p) {
                     }
                 }
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[i] += acc_b[i];
+                for (int grp = 0; grp < NG; ++grp)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[grp][i] += acc_b[grp][i];
                 if (!L2) {  // the L2 flavour still needs the rows: it hands the stage back below
                     __syncwarp();
                     if (lane == 0) mbar_arrive(empty_bar);
@@ -502,10 +516,10 @@ scan_kernel(const ScanParams p) {
                     }
                     const float sl = p.l2_slack;
                     bool pass[4];
-                    pass[0] = r_lo < p.N && q0 < p.s && (2.f * acc[0] - n_lo - qn0) + sl * (n_lo + qn0) >= th0;
-                    pass[1] = r_lo < p.N && q1 < p.s && (2.f * acc[1] - n_lo - qn1) + sl * (n_lo + qn1) >= th1;
-                    pass[2] = r_hi < p.N && q0 < p.s && (2.f * acc[2] - n_hi - qn0) + sl * (n_hi + qn0) >= th0;
-                    pass[3] = r_hi < p.N && q1 < p.s && (2.f * acc[3] - n_hi - qn1) + sl * (n_hi + qn1) >= th1;
+                    pass[0] = r_lo < p.N && q0 < p.s && (2.f * acc[0][0] - n_lo - qn0) + sl * (n_lo + qn0) >= th0;
+                    pass[1] = r_lo < p.N && q1 < p.s && (2.f * acc[0][1] - n_lo - qn1) + sl * (n_lo + qn1) >= th1;
+                    pass[2] = r_hi < p.N && q0 < p.s && (2.f * acc[0][2] - n_hi - qn0) + sl * (n_hi + qn0) >= th0;
+                    pass[3] = r_hi < p.N && q1 < p.s && (2.f * acc[0][3] - n_hi - qn1) + sl * (n_hi + qn1) >= th1;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         unsigned m = __ballot_sync(0xffffffffu, pass[i]);
@@ -530,36 +544,40 @@ scan_kernel(const ScanParams p) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive(empty_bar);
                 } else {
-                if (TOP1) {
-                    if (r_lo < p.N) {
-                        const uint64_t k0 = make_key(acc[0], static_cast<uint32_t>(r_lo));
-                        const uint64_t k1 = make_key(acc[1], static_cast<uint32_t>(r_lo));
-                        best0 = k0 > best0 ? k0 : best0;
-                        best1 = k1 > best1 ? k1 : best1;
-                    }
-                    if (r_hi < p.N) {
-                        const uint64_t k0 = make_key(acc[2], static_cast<uint32_t>(r_hi));
-                        const uint64_t k1 = make_key(acc[3], static_cast<uint32_t>(r_hi));
-                        best0 = k0 > best0 ? k0 : best0;
-                        best1 = k1 > best1 ? k1 : best1;
-                    }
-                } else {
-                    const float th0 = hdr->thr[q0], th1 = hdr->thr[q1];
-                    if (r_lo < p.N) {
-                        if (q0 < p.s && acc[0] >= th0)
-                            push_candidate(hdr, cand, p.cap, p.soft_limit, q0,
-                                           make_key(acc[0], static_cast<uint32_t>(r_lo)));
-                        if (q1 < p.s && acc[1] >= th1)
-                            push_candidate(hdr, cand, p.cap, p.soft_limit, q1,
-                                           make_key(acc[1], static_cast<uint32_t>(r_lo)));
-                    }
-                    if (r_hi < p.N) {
-                        if (q0 < p.s && acc[2] >= th0)
-                            push_candidate(hdr, cand, p.cap, p.soft_limit, q0,
-                                           make_key(acc[2], static_cast<uint32_t>(r_hi)));
-                        if (q1 < p.s && acc[3] >= th1)
-                            push_candidate(hdr, cand, p.cap, p.soft_limit, q1,
-                                           make_key(acc[3], static_cast<uint32_t>(r_hi)));
+#pragma unroll
+                for (int grp = 0; grp < NG; ++grp) {
+                    const int gq0 = grp * kScanMaxQueries + q0, gq1 = gq0 + 1;
+                    if (TOP1) {
+                        if (r_lo < p.N) {
+                            const uint64_t k0 = make_key(acc[grp][0], static_cast<uint32_t>(r_lo));
+                            const uint64_t k1 = make_key(acc[grp][1], static_cast<uint32_t>(r_lo));
+                            bestA[grp] = k0 > bestA[grp] ? k0 : bestA[grp];
+                            bestB[grp] = k1 > bestB[grp] ? k1 : bestB[grp];
+                        }
+                        if (r_hi < p.N) {
+                            const uint64_t k0 = make_key(acc[grp][2], static_cast<uint32_t>(r_hi));
+                            const uint64_t k1 = make_key(acc[grp][3], static_cast<uint32_t>(r_hi));
+                            bestA[grp] = k0 > bestA[grp] ? k0 : bestA[grp];
+                            bestB[grp] = k1 > bestB[grp] ? k1 : bestB[grp];
+                        }
+                    } else {
+                        const float th0 = hdr->thr[gq0], th1 = hdr->thr[gq1];
+                        if (r_lo < p.N) {
+                            if (gq0 < p.s && acc[grp][0] >= th0)
+                                push_candidate(hdr, cand, p.cap, p.soft_limit, gq0,
+                                               make_key(acc[grp][0], static_cast<uint32_t>(r_lo)));
+                            if (gq1 < p.s && acc[grp][1] >= th1)
+                                push_candidate(hdr, cand, p.cap, p.soft_limit, gq1,
+                                               make_key(acc[grp][1], static_cast<uint32_t>(r_lo)));
+                        }
+                        if (r_hi < p.N) {
+                            if (gq0 < p.s && acc[grp][2] >= th0)
+                                push_candidate(hdr, cand, p.cap, p.soft_limit, gq0,
+                                               make_key(acc[grp][2], static_cast<uint32_t>(r_hi)));
+                            if (gq1 < p.s && acc[grp][3] >= th1)
+                                push_candidate(hdr, cand, p.cap, p.soft_limit, gq1,
+                                               make_key(acc[grp][3], static_cast<uint32_t>(r_hi)));
+                        }
                     }
                 }
                 }
@@ -616,7 +634,7 @@ scan_kernel(const ScanParams p) {
                     if ((lane & 1) == 0 && row < p.N && jq < p.s) {
                         if (TOP1) {
                             const uint64_t key = make_key(val, static_cast<uint32_t>(row));
-                            best0 = key > best0 ? key : best0;
+                            bestA[0] = key > bestA[0] ? key : bestA[0];
                         } else if (val >= hdr->thr[jq]) {
                             push_candidate(hdr, cand, p.cap, p.soft_limit, jq,
                                            make_key(val, static_cast<uint32_t>(row)));
@@ -630,11 +648,15 @@ scan_kernel(const ScanParams p) {
         if (TOP1) {
             if (MMA) {
                 // (the L2 flavour has put its keys into hdr->best as it went)
-                if (best0) atomicMax(&hdr->best[2 * t], static_cast<unsigned long long>(best0));
-                if (best1) atomicMax(&hdr->best[2 * t + 1], static_cast<unsigned long long>(best1));
+#pragma unroll
+                for (int grp = 0; grp < NG; ++grp) {
+                    const int gq = grp * kScanMaxQueries + 2 * t;
+                    if (bestA[grp]) atomicMax(&hdr->best[gq], static_cast<unsigned long long>(bestA[grp]));
+                    if (bestB[grp]) atomicMax(&hdr->best[gq + 1], static_cast<unsigned long long>(bestB[grp]));
+                }
             } else {
                 const int jq = (lane >> 1) % SQR;
-                if (best0) atomicMax(&hdr->best[jq], static_cast<unsigned long long>(best0));
+                if (bestA[0]) atomicMax(&hdr->best[jq], static_cast<unsigned long long>(bestA[0]));
             }
             named_barrier(1, cthreads);
             if (ctid < p.s)

@@ -50,6 +50,18 @@ def test_integer_inputs_are_bit_exact(metric, N, d, s, k):
         check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), metric, k, exact=True)
 
 
+@pytest.mark.parametrize("N,d,s,k", [(5000, 768, 9, 1), (5000, 768, 12, 20), (4000, 64, 16, 5), (3001, 1024, 13, 300),
+                                     (70_000, 128, 16, 1), (900, 72, 35, 4)])
+def test_sixteen_queries_per_pass_integer_inputs(N, d, s, k):
+    """Inner product with 9..16 queries runs as ONE pass of the small-batch scan (two groups of
+    8 queries share every staged tile); more queries under variant 2 run in passes of 16."""
+    x = workloads.integer_valued((N, d), seed=600 + N, lo=-3, hi=3, device=DEV)
+    q = workloads.integer_valued((s, d), seed=700 + N, lo=-3, hi=3, device=DEV)
+    for variant in (0, 2):
+        ids, scores = _run(x, q, oracle.IP, k, variant)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+
+
 # ------------------------------------------------------------------ shape sweep, real values
 @pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
 @pytest.mark.parametrize("N", [1, 31, 32, 33, 1000, 100_003])
