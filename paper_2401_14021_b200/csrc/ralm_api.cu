@@ -90,7 +90,7 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
     pl->stage_bytes = align_up(pl->tile_rows * idx->d * 2, 128);
     pl->off_q = kScanHeaderBytes;
     // (the warp-MMA flavour stages 8 query rows, or 16 when a pass carries more than 8)
-    const int q_rows = s_pass > kScanMaxQueries ? kScanMaxPassQueries : kScanMaxQueries;
+    const int q_rows = s_pass > 16 ? 32 : (s_pass > kScanMaxQueries ? 16 : kScanMaxQueries);
     int off = pl->off_q + (mma ? align_up(q_rows * (idx->d * 2 + kQueryPadBytes), 128) : 0);
     pl->off_cand = off;
     pl->cap = 0;
@@ -314,7 +314,7 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
 }
 
 constexpr int kTcAutoMinQueries = 9;     // batches the 8-query scan cannot serve in one pass
-constexpr int kTcAutoMinQueriesIp = 17;  // inner product: the small-batch scan takes 16 in one pass
+constexpr int kTcAutoMinQueriesIp = 33;  // inner product: the small-batch scan takes 32 in one pass
 
 ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k, int64_t *ids,
                             float *scores, cudaStream_t st) {
@@ -437,6 +437,9 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             if (mma && idx->metric == RALM_L2)
                 return (k == 1) ? launch_scan<true, true, 8, 1, true>(p, g, pl.smem_bytes, st)
                                 : launch_scan<true, true, 8, 1, false>(p, g, pl.smem_bytes, st);
+            if (mma && sp > 16)
+                return (k == 1) ? launch_scan<true, false, 32, 1, true>(p, g, pl.smem_bytes, st)
+                                : launch_scan<true, false, 32, 1, false>(p, g, pl.smem_bytes, st);
             if (mma && sp > kScanMaxQueries)
                 return (k == 1) ? launch_scan<true, false, 16, 1, true>(p, g, pl.smem_bytes, st)
                                 : launch_scan<true, false, 16, 1, false>(p, g, pl.smem_bytes, st);

@@ -1,4 +1,5 @@
-// Corpus scan for small query batches (at most 8 queries per pass): scores every corpus
+// Corpus scan for small query batches (8 queries per pass; 16 or 32 for larger inner-product
+// batches, as groups of 8 that share every staged tile): scores every corpus
 // row against every query and keeps, per CTA and query, the best k rows.
 //
 // One persistent CTA per SM. Warp 0 is the producer: one thread streams tiles of whole rows
@@ -40,7 +41,7 @@ namespace ralm {
 constexpr int kMaxStages = 24;
 constexpr int kMaxConsumerWarps = 8;
 constexpr int kScanMaxQueries = 8;       // queries of one MMA group (the N of m16n8k16)
-constexpr int kScanMaxPassQueries = 16;  // queries per pass: two groups in the inner-product warp-MMA flavour
+constexpr int kScanMaxPassQueries = 32;  // queries per pass: up to four groups in the inner-product warp-MMA flavour
 constexpr int kScanThreads = 32 * (kMaxConsumerWarps + 1);
 constexpr int kQueryPadBytes = 64;
 

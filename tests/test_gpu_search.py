@@ -51,10 +51,11 @@ def test_integer_inputs_are_bit_exact(metric, N, d, s, k):
 
 
 @pytest.mark.parametrize("N,d,s,k", [(5000, 768, 9, 1), (5000, 768, 12, 20), (4000, 64, 16, 5), (3001, 1024, 13, 300),
-                                     (70_000, 128, 16, 1), (900, 72, 35, 4)])
-def test_sixteen_queries_per_pass_integer_inputs(N, d, s, k):
-    """Inner product with 9..16 queries runs as ONE pass of the small-batch scan (two groups of
-    8 queries share every staged tile); more queries under variant 2 run in passes of 16."""
+                                     (70_000, 128, 16, 1), (900, 72, 35, 4), (6000, 768, 17, 20), (6000, 256, 32, 1),
+                                     (2000, 64, 70, 3)])
+def test_several_query_groups_per_pass_integer_inputs(N, d, s, k):
+    """Inner product with 9..32 queries runs as ONE pass of the small-batch scan (two or four
+    groups of 8 queries share every staged tile); more queries under variant 2 run in passes of 32."""
     x = workloads.integer_valued((N, d), seed=600 + N, lo=-3, hi=3, device=DEV)
     q = workloads.integer_valued((s, d), seed=700 + N, lo=-3, hi=3, device=DEV)
     for variant in (0, 2):
