@@ -192,11 +192,11 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
 
 /* Pin the scan variant used by ralm_search on this index (benchmarking aid).
  *   0 = automatic, 1 = FMA scan (fp32 FMAs, d <= 1024, 4 queries per pass), 2 = warp-MMA scan
- *   (8 queries per pass, 16 or 32 for larger inner-product batches; for L2 the tensor-core
+ *   (8 queries per pass, 16 for larger batches, 32 for inner product; for L2 the tensor-core
  *   value only filters and the ranked distance is the direct sum of squared differences), 3 = tcgen05 scan (up to 512 queries per pass, k <= 64,
  *   d >= 64; pairs of CTAs share each MMA; for L2 the tensor-core value again only filters,
  *   and the corpus must be large enough to scan a sample first, about 600 K rows), 4 = tcgen05
- *   scan with single CTAs. Automatic: warp-MMA up to 32 queries (inner product) or 8 (L2), the
+ *   scan with single CTAs. Automatic: warp-MMA up to 32 queries (inner product) or 16 (L2), the
  *   tcgen05 scan beyond that where it applies.
  * UNSUPPORTED if the variant cannot serve the index's metric or dimension. The environment
  * variable RALM_FORCE_VARIANT=<1..4> applies the same pin to every index at creation. */

@@ -314,7 +314,8 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
 }
 
 constexpr int kTcAutoMinQueries = 9;     // batches the 8-query scan cannot serve in one pass
-constexpr int kTcAutoMinQueriesIp = 33;  // inner product: the small-batch scan takes 32 in one pass
+constexpr int kTcAutoMinQueriesIp = 33;  // inner product: the small-batch scan takes up to 32 in one pass
+constexpr int kTcAutoMinQueriesL2 = 17;  // L2: up to 16
 
 ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k, int64_t *ids,
                             float *scores, cudaStream_t st) {
@@ -333,7 +334,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     const bool tc = tc_can_serve(idx, k) && (!l2 || tc_two_phase) &&
                     (idx->variant == 3 || idx->variant == 4 ||
                      (idx->variant == 0 &&
-                      (s >= (l2 ? kTcAutoMinQueries : kTcAutoMinQueriesIp) || (!small_scan_fits && !l2))));
+                      (s >= (l2 ? kTcAutoMinQueriesL2 : kTcAutoMinQueriesIp) || (!small_scan_fits && !l2))));
     if (tc) {
         // Large corpora are scanned in two phases: a small sample first, whose merged top-k gives
         // every query a score that k rows are known to reach; the rest then starts from those
@@ -381,10 +382,12 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     const int variant = resolve_variant(idx);
     const bool mma = variant == 2;
     if (!mma && idx->d > kFmaMaxD) return RALM_ERR_UNSUPPORTED;
-    // inner product on the warp-MMA flavour: two groups of 8 queries share every staged tile
-    // when the batch has more than 8 (the tile is read from shared memory twice, from HBM once)
-    const bool wide = mma && idx->metric == RALM_IP && s > kScanMaxQueries;
-    const int per_pass = mma ? (wide ? kScanMaxPassQueries : kScanMaxQueries) : kFmaQueriesPerPass;
+    // warp-MMA flavour: up to four groups of 8 queries share every staged tile when the batch
+    // has more than 8 (the tile is read from HBM once)
+    const bool wide = mma && s > kScanMaxQueries && (idx->metric == RALM_IP || idx->norms != nullptr);
+    // (L2 stops at two groups: with four, its filter and rescoring cost more than a second pass)
+    const int wide_pass = idx->metric == RALM_L2 ? 16 : kScanMaxPassQueries;
+    const int per_pass = mma ? (wide ? wide_pass : kScanMaxQueries) : kFmaQueriesPerPass;
     // k > 1 on a large corpus: scan a sample first and start the rest from the sample's merged
     // k-th scores (see the large-batch path above); the sample's list is block num_sms of `partial`
     // (1/128 of the rows here: measured best for this scan; the large-batch scan prefers 1/64)
@@ -431,6 +434,9 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             // the same grid whatever the tile height of the pass: the merge reads one list per CTA
             const int g = static_cast<int>(std::min<long long>(idx->num_sms, (end - begin + 15) / 16));
             *grid_out = g;
+            if (mma && idx->metric == RALM_L2 && idx->norms && sp > kScanMaxQueries)
+                return (k == 1) ? launch_scan<true, true, 16, 1, true, true>(p, g, pl.smem_bytes, st)
+                                : launch_scan<true, true, 16, 1, false, true>(p, g, pl.smem_bytes, st);
             if (mma && idx->metric == RALM_L2 && idx->norms)
                 return (k == 1) ? launch_scan<true, true, 8, 1, true, true>(p, g, pl.smem_bytes, st)
                                 : launch_scan<true, true, 8, 1, false, true>(p, g, pl.smem_bytes, st);
@@ -585,7 +591,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     };
     alloc(&idx->partial, partial_bytes);
     alloc(&idx->tc_thr, sizeof(float) * max_s);
-    const int pass_queries = std::min(max_s, metric == RALM_IP ? kScanMaxPassQueries : kScanMaxQueries);
+    const int pass_queries = std::min(max_s, kScanMaxPassQueries);
     if (max_k > 1 && std::max(512, 2 * next_pow2(max_k)) * 8 * pass_queries > kSmemCandBytes) {
         idx->spill_cap = std::max(512, 2 * next_pow2(max_k));
         alloc(&idx->spill, sizeof(uint64_t) * idx->num_sms * kScanMaxPassQueries * static_cast<size_t>(idx->spill_cap));

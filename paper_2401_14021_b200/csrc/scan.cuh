@@ -338,8 +338,8 @@ scan_kernel(const ScanParams p) {
         const int cthreads = W * 32;
         const int g = lane >> 2, t = lane & 3;
 
-        // inner-product warp-MMA flavour: SQ / 8 groups of 8 queries share every tile
-        constexpr int NG = (MMA && !L2) ? SQ / 8 : 1;
+        // warp-MMA flavour: SQ / 8 groups of 8 queries share every tile
+        constexpr int NG = MMA ? SQ / 8 : 1;
         uint64_t bestA[NG], bestB[NG];
 #pragma unroll
         for (int grp = 0; grp < NG; ++grp) bestA[grp] = bestB[grp] = 0;
@@ -375,14 +375,19 @@ scan_kernel(const ScanParams p) {
         // norms of this lane's two queries (2t, 2t+1), summed in fp32
         const uint32_t q_pitch = static_cast<uint32_t>(d * 2 + kQueryPadBytes);
         const uint32_t q_base_addr = smem_u32(smem + p.off_q);
-        float qn0 = 0.f, qn1 = 0.f;
-        if (MMA && L2) {
-            const __half *qa = reinterpret_cast<const __half *>(smem + p.off_q + (2 * t) * q_pitch);
-            const __half *qb = reinterpret_cast<const __half *>(smem + p.off_q + (2 * t + 1) * q_pitch);
-            for (int i = 0; i < d; ++i) {
-                const float a = __half2float(qa[i]), b = __half2float(qb[i]);
-                qn0 = fmaf(a, a, qn0);
-                qn1 = fmaf(b, b, qn1);
+        float qn0[NG], qn1[NG];
+#pragma unroll
+        for (int grp = 0; grp < NG; ++grp) {
+            qn0[grp] = qn1[grp] = 0.f;
+            if (MMA && L2) {
+                const int row_a = grp * kScanMaxQueries + 2 * t;
+                const __half *qa = reinterpret_cast<const __half *>(smem + p.off_q + row_a * q_pitch);
+                const __half *qb = reinterpret_cast<const __half *>(smem + p.off_q + (row_a + 1) * q_pitch);
+                for (int i = 0; i < d; ++i) {
+                    const float a = __half2float(qa[i]), b = __half2float(qb[i]);
+                    qn0[grp] = fmaf(a, a, qn0[grp]);
+                    qn1[grp] = fmaf(b, b, qn1[grp]);
+                }
             }
         }
 
@@ -490,7 +495,7 @@ scan_kernel(const ScanParams p) {
                 // acc[0]: (row g, query 2t)     acc[1]: (row g, query 2t+1)
                 // acc[2]: (row g+8, query 2t)   acc[3]: (row g+8, query 2t+1)
                 const long long r_lo = row0 + g, r_hi = row0 + g + 8;
-                const int q0 = 2 * t, q1 = 2 * t + 1;
+                const int q0 = 2 * t;  // this lane's first query within a group; the second is q0 + 1
                 if (L2) {
                     // |x|^2 - 2 x.q + |q|^2 from the tensor cores is only a FILTER (it cancels):
                     // a pair passes when it could still beat the threshold given the slack that
@@ -505,39 +510,44 @@ scan_kernel(const ScanParams p) {
                         n_lo = __shfl_sync(0xffffffffu, d_lo, diag_lane);
                         n_hi = __shfl_sync(0xffffffffu, d_hi, diag_lane);
                     }
-                    float th0, th1;
-                    if (TOP1) {
-                        const unsigned long long b0 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[q0]);
-                        const unsigned long long b1 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[q1]);
-                        th0 = b0 ? key_value(b0) : -INFINITY;
-                        th1 = b1 ? key_value(b1) : -INFINITY;
-                    } else {
-                        th0 = *reinterpret_cast<volatile float *>(&hdr->thr[q0]);
-                        th1 = *reinterpret_cast<volatile float *>(&hdr->thr[q1]);
-                    }
                     const float sl = p.l2_slack;
-                    bool pass[4];
-                    pass[0] = r_lo < p.N && q0 < p.s && (2.f * acc[0][0] - n_lo - qn0) + sl * (n_lo + qn0) >= th0;
-                    pass[1] = r_lo < p.N && q1 < p.s && (2.f * acc[0][1] - n_lo - qn1) + sl * (n_lo + qn1) >= th1;
-                    pass[2] = r_hi < p.N && q0 < p.s && (2.f * acc[0][2] - n_hi - qn0) + sl * (n_hi + qn0) >= th0;
-                    pass[3] = r_hi < p.N && q1 < p.s && (2.f * acc[0][3] - n_hi - qn1) + sl * (n_hi + qn1) >= th1;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        unsigned m = __ballot_sync(0xffffffffu, pass[i]);
-                        while (m) {
-                            const int src = __ffs(m) - 1;
-                            m &= m - 1;
-                            const int row_local = (src >> 2) + ((i & 2) ? 8 : 0);
-                            const int q = 2 * (src & 3) + (i & 1);
-                            const float dist = warp_direct_l2(stage_addr + row_local * d * 2,
-                                                              q_base_addr + q * q_pitch, d, lane);
-                            if (lane == 0) {
-                                const float val = 0.0f - dist;
-                                const uint64_t key = make_key(val, static_cast<uint32_t>(row0 + row_local));
-                                if (TOP1) {
-                                    atomicMax(&hdr->best[q], static_cast<unsigned long long>(key));
-                                } else if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q])) {
-                                    push_candidate(hdr, cand, p.cap, p.soft_limit, q, key);
+                    for (int grp = 0; grp < NG; ++grp) {
+                        const int gq0 = grp * kScanMaxQueries + q0, gq1 = gq0 + 1;
+                        float th0, th1;
+                        if (TOP1) {
+                            const unsigned long long b0 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[gq0]);
+                            const unsigned long long b1 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[gq1]);
+                            th0 = b0 ? key_value(b0) : -INFINITY;
+                            th1 = b1 ? key_value(b1) : -INFINITY;
+                        } else {
+                            th0 = *reinterpret_cast<volatile float *>(&hdr->thr[gq0]);
+                            th1 = *reinterpret_cast<volatile float *>(&hdr->thr[gq1]);
+                        }
+                        const float a0 = qn0[grp], a1 = qn1[grp];
+                        bool pass[4];
+                        pass[0] = r_lo < p.N && gq0 < p.s && (2.f * acc[grp][0] - n_lo - a0) + sl * (n_lo + a0) >= th0;
+                        pass[1] = r_lo < p.N && gq1 < p.s && (2.f * acc[grp][1] - n_lo - a1) + sl * (n_lo + a1) >= th1;
+                        pass[2] = r_hi < p.N && gq0 < p.s && (2.f * acc[grp][2] - n_hi - a0) + sl * (n_hi + a0) >= th0;
+                        pass[3] = r_hi < p.N && gq1 < p.s && (2.f * acc[grp][3] - n_hi - a1) + sl * (n_hi + a1) >= th1;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            unsigned m = __ballot_sync(0xffffffffu, pass[i]);
+                            while (m) {
+                                const int src = __ffs(m) - 1;
+                                m &= m - 1;
+                                const int row_local = (src >> 2) + ((i & 2) ? 8 : 0);
+                                const int q = grp * kScanMaxQueries + 2 * (src & 3) + (i & 1);
+                                const float dist = warp_direct_l2(stage_addr + row_local * d * 2,
+                                                                  q_base_addr + q * q_pitch, d, lane);
+                                if (lane == 0) {
+                                    const float val = 0.0f - dist;
+                                    const uint64_t key = make_key(val, static_cast<uint32_t>(row0 + row_local));
+                                    if (TOP1) {
+                                        atomicMax(&hdr->best[q], static_cast<unsigned long long>(key));
+                                    } else if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q])) {
+                                        push_candidate(hdr, cand, p.cap, p.soft_limit, q, key);
+                                    }
                                 }
                             }
                         }

@@ -54,13 +54,14 @@ def test_integer_inputs_are_bit_exact(metric, N, d, s, k):
                                      (70_000, 128, 16, 1), (900, 72, 35, 4), (6000, 768, 17, 20), (6000, 256, 32, 1),
                                      (2000, 64, 70, 3)])
 def test_several_query_groups_per_pass_integer_inputs(N, d, s, k):
-    """Inner product with 9..32 queries runs as ONE pass of the small-batch scan (two or four
-    groups of 8 queries share every staged tile); more queries under variant 2 run in passes of 32."""
+    """9..32 queries run as ONE pass of the small-batch scan (two or four groups of 8 queries
+    share every staged tile); more queries under variant 2 run in passes of 32."""
     x = workloads.integer_valued((N, d), seed=600 + N, lo=-3, hi=3, device=DEV)
     q = workloads.integer_valued((s, d), seed=700 + N, lo=-3, hi=3, device=DEV)
-    for variant in (0, 2):
-        ids, scores = _run(x, q, oracle.IP, k, variant)
-        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+    for metric in (oracle.IP, oracle.L2):
+        for variant in (0, 2):
+            ids, scores = _run(x, q, metric, k, variant)
+            check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), metric, k, exact=True)
 
 
 # ------------------------------------------------------------------ shape sweep, real values
