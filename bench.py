@@ -397,7 +397,7 @@ def main():
 
 # (dram__bytes_read.sum + dram__bytes_write.sum) / corpus bytes of one scan launch, from the
 # committed ncu capture of a 2 M-row case; traffic grows in proportion to the rows.
-TRAFFIC_RATIO = {"scan_kernel<mma,ip>": 1.0016}  # dram bytes / corpus bytes, profiles/scan_mma_ip_s8_k1_2Mx768.md
+TRAFFIC_RATIO = {"scan_kernel<mma,ip>": 1.0015}  # dram bytes / corpus bytes, profiles/scan_mma_ip_s8_k1_2Mx768.md
 
 if __name__ == "__main__":
     main()
