@@ -115,6 +115,24 @@ def test_c3_serving_step_cache_and_verify(c3_corpus):
     idx.close()
 
 
+@pytest.mark.parametrize("s,k", [(16, 1), (16, 20), (32, 20), (64, 20)])
+def test_c3_full_size_mid_batches(c3_corpus, s, k):
+    """Between the two headline cases: 16 and 32 queries run as one pass of the small-batch scan
+    (two and four query groups per staged tile), 64 on the tcgen05 scan."""
+    ralm = _ralm()
+    x, _ = c3_corpus
+    q, src = workloads.noisy_copy_queries(x, s, workloads.seed_for(3, "queries") + s)
+    idx = ralm.Index(x, oracle.IP, max_s=s, max_k=k)
+    ids, scores = ralm.search(idx, q, k)
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    assert ids[:, 0].tolist() == src.tolist()
+    strict, band, n_sub = _sampled_parity(x, q, ids, scores, oracle.IP, k, 8, 16_384, seed=3600 + s + k,
+                                          query_sel=range(0, s, max(1, s // 16)))
+    print("C3 s=%d k=%d: strict=%d band=%d over a %d-row sub-corpus" % (s, k, strict, band, n_sub))
+    idx.close()
+
+
 def test_c5_full_size_512_queries(c3_corpus):
     """The high-concurrency configuration: 512 queries, k = 20, on the tcgen05 scan."""
     ralm = _ralm()
@@ -163,6 +181,16 @@ def test_c4_full_size_l2_k1024():
     strict, band, n_sub = _sampled_parity(x, q64, ids, scores, oracle.L2, 20, 6, 16_384, seed=3450,
                                           query_sel=range(0, 64, 4))
     print("C4, 64 queries: strict=%d band=%d over a %d-row sub-corpus, 16 of 64 queries" % (strict, band, n_sub))
+    idx.close()
+    # 16 concurrent queries, k = 20: one pass of the small-batch scan with two query groups
+    q16, src16 = workloads.noisy_copy_queries(x, 16, workloads.seed_for(4, "queries") + 9)
+    idx = ralm.Index(x, oracle.L2, max_s=16, max_k=20)
+    ids, scores = ralm.search(idx, q16, 20)
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    assert ids[:, 0].tolist() == src16.tolist()
+    strict, band, n_sub = _sampled_parity(x, q16, ids, scores, oracle.L2, 20, 6, 16_384, seed=3460)
+    print("C4, 16 queries: strict=%d band=%d over a %d-row sub-corpus" % (strict, band, n_sub))
     idx.close()
     del x
     torch.cuda.empty_cache()
