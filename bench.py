@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--s", type=int, default=None)
     ap.add_argument("--k", type=int, default=None)
     ap.add_argument("--variant", type=int, default=0)
+    ap.add_argument("--q8", action="store_true",
+                    help="stream the index's one-byte copy of the corpus (exact results; inner product, s <= 8)")
     ap.add_argument("--rows", type=int, default=None, help="override the corpus size (profiling)")
     ap.add_argument("--tune", default=None, help="consumer_warps,ring_depth,tile_rows (0 = default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -251,6 +253,8 @@ def main():
     idx = ralm.Index(corpus, metric_id, max_s=max(s, 1), max_k=max(k, 1))
     if args.variant:
         idx.set_variant(args.variant)
+    if args.q8:
+        idx.enable_q8()
     if args.tune:
         idx.set_tuning(*[int(v) for v in args.tune.split(",")])
     stream = torch.cuda.current_stream()
@@ -350,6 +354,17 @@ def main():
                                 if cfg.metric == "ip" and args.variant in (0, 2) and not args.tune
                                 and s <= 8 else None),
                     "traffic_note": "2M-row ncu capture scaled by rows; null if the kernel changed since"}
+        if args.q8 and cfg.metric == "ip" and args.variant == 0 and s <= 8 and k <= 256:
+            # the 8-bit scan streams the one-byte copy and one fp32 bound per row; the sample
+            # (1/128 of the rows, when the corpus is large enough for one) is scanned in fp16
+            sample = max(N // 128, 4 * 148 * 128) if max(N // 128, 4 * 148 * 128) * 32 <= N else 0
+            q8_bytes = sample * d * 2 + (N - sample) * (d + 4)
+            achieved = q8_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None
+            roofline.update({"achieved": achieved, "frac": achieved / peaks["hbm_gbs"] if achieved else None,
+                             "frac_of_nominal_8000": achieved / 8000.0 if achieved else None,
+                             "kernel": "scan_q8_kernel", "bytes_per_launch": q8_bytes, "traffic": None,
+                             "fp16_equivalent_gbs": corpus_bytes / (scan_avg_ms * 1e-3) / 1e9
+                             if scan_launches else None})
         uses_tc = k <= 64 and d >= 64 and (cfg.metric == "ip" or N >= 700_000) and \
             (args.variant in (3, 4) or (args.variant == 0 and s >= 9))
         if uses_tc:
@@ -373,7 +388,7 @@ def main():
             "config": {"workload": "%s %dx%d %s s=%d k=%d; cache lookup R=%d C=%d q=%d; verify stride %d"
                                    % (cfg.name, N, d, cfg.metric, s, k, R, cache.shape[1], stride, vstride),
                        "arithmetic": "fp16 corpus and queries, exact fp16 x fp16 products, fp32 accumulation",
-                       "variant": args.variant, "tune": args.tune, "replicas": world,
+                       "variant": args.variant, "tune": args.tune, "replicas": world, "q8": bool(args.q8),
                        "l2": "inputs larger than L2 (%.1f GB corpus streamed every step)"
                              % (corpus_bytes / 1e9) if corpus_bytes > 2.5e8 else
                              "corpus near L2 size: L2-warm figure, not an HBM number"},

@@ -14,6 +14,7 @@
 
 #include "aux_kernels.cuh"
 #include "scan.cuh"
+#include "scan_q8.cuh"
 #include "scan_tc.cuh"
 
 using namespace ralm;
@@ -34,6 +35,8 @@ struct ralm_index {
     uint64_t *spill;       // large k: candidate lists of the small-batch scan, [num_sms][8][spill_cap]
     int spill_cap;
     float *norms;          // L2: squared norm of every corpus row (fp32 [N]), or null
+    uint8_t *x8;           // inner product, optional: one-byte (E5M2) copy of the corpus, [N][d]
+    float *x8_bound;       // per row: bound on |q.x - q.x8| per unit of |q| (see scan_q8.cuh)
     float *tc_thr;         // thresholds from the sample phase of a two-phase scan, [max_s]
     bool tc_two_phase;     // sample phase enabled (tuning aid)
     int tc_clusters;       // CTA pairs the device runs at once (-1 = not asked yet)
@@ -114,6 +117,34 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
     // every consumer warp owns `depth` stages; fewer warps when the stages are large
     pl->nwarps = std::min(pl->nwarps, fit);
     pl->depth = std::min(fit / pl->nwarps, idx->tune_depth > 0 ? idx->tune_depth : 3);
+    pl->smem_bytes = pl->off_stage + pl->nwarps * pl->depth * pl->stage_bytes;
+    return true;
+}
+
+// Shared-memory layout of one CTA of the 8-bit scan: 16-row tiles of d bytes, 8 staged queries,
+// candidate lists in shared memory (k <= kQ8MaxK keeps them within kSmemCandBytes).
+constexpr int kQ8MaxK = 256;
+bool plan_scan_q8(const ralm_index *idx, int k, ScanPlan *pl) {
+    pl->tile_rows = 16;
+    pl->stage_bytes = align_up(pl->tile_rows * idx->d, 128);
+    pl->off_q = kScanHeaderBytes;
+    int off = pl->off_q + align_up(kScanMaxQueries * (idx->d * 2 + kQueryPadBytes), 128);
+    pl->off_cand = off;
+    pl->cap = 0;
+    pl->soft_limit = 0;
+    pl->spill = false;
+    if (k > 1) {
+        pl->cap = std::max(512, 2 * next_pow2(k));
+        pl->soft_limit = std::min(pl->cap - (kMaxConsumerWarps + 1) * pl->tile_rows, std::max(4 * k, 64));
+        off += kScanMaxQueries * pl->cap * 8;
+    }
+    pl->off_stage = align_up(off, 128);
+    const int fit = std::min(kMaxStages, (idx->smem_optin - pl->off_stage) / pl->stage_bytes);
+    if (fit < 2) return false;
+    // two stages per consumer warp before an eighth warp: a warp that is scoring a row again
+    // from global memory must not hold up the producer
+    pl->depth = fit >= 3 * kMaxConsumerWarps ? 3 : (fit >= 4 ? 2 : 1);
+    pl->nwarps = std::min(kMaxConsumerWarps, fit / pl->depth);
     pl->smem_bytes = pl->off_stage + pl->nwarps * pl->depth * pl->stage_bytes;
     return true;
 }
@@ -394,7 +425,13 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     long long sample = std::max<long long>(idx->N / 128, 4LL * idx->num_sms * kTcTileM);
     sample = (sample + 255) / 256 * 256;
     // (two more launches: only worth it when the scan itself takes a millisecond or more)
-    const bool two_phase = k > 1 && idx->tc_thr && idx->tc_two_phase && sample * 32 <= idx->N;
+    // An index with an 8-bit copy (ralm_index_enable_q8) streams that copy for batches of up to 8
+    // queries and scores again, exactly, what its filter lets through; the sample is scanned in
+    // fp16 also for k == 1, since the filter needs thresholds to be of any use.
+    ScanPlan pl8;
+    const bool use_q8 = idx->x8 && idx->metric == RALM_IP && idx->variant == 0 && s <= kScanMaxQueries &&
+                        k <= kQ8MaxK && plan_scan_q8(idx, k, &pl8);
+    const bool two_phase = (k > 1 || use_q8) && idx->tc_thr && idx->tc_two_phase && sample * 32 <= idx->N;
     int grid = 0;
     for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
         const int sp = std::min(per_pass, s - q0);
@@ -404,6 +441,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
         p.corpus = idx->corpus;
         p.queries = queries + static_cast<size_t>(q0) * idx->d;
         p.norms = idx->norms;
+        p.x8 = nullptr;
         p.spill = pl.spill ? idx->spill : nullptr;
         p.partial = idx->partial;
         p.status = idx->status;
@@ -455,10 +493,51 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             return idx->metric == RALM_L2 ? launch_fma<true>(p, g, pl.smem_bytes, st)
                                           : launch_fma<false>(p, g, pl.smem_bytes, st);
         };
+        auto scan_rows_q8 = [&](long long begin, long long end, const float *thr_init, int *grid_out) -> cudaError_t {
+            ScanParams p8 = p;
+            p8.x8 = idx->x8;
+            p8.norms = idx->x8_bound;
+            p8.spill = nullptr;
+            p8.cap = pl8.cap;
+            p8.soft_limit = pl8.soft_limit;
+            p8.tile_rows = pl8.tile_rows;
+            p8.nwarps = pl8.nwarps;
+            p8.depth = pl8.depth;
+            p8.stage_bytes = pl8.stage_bytes;
+            p8.off_q = pl8.off_q;
+            p8.off_cand = pl8.off_cand;
+            p8.off_stage = pl8.off_stage;
+            p8.row_begin = begin;
+            p8.N = end;
+            p8.thr_init = thr_init;
+            p8.ntiles = (end - begin + pl8.tile_rows - 1) / pl8.tile_rows;
+            const int g = static_cast<int>(std::min<long long>(idx->num_sms, (end - begin + 15) / 16));
+            *grid_out = g;
+            auto kern = (k == 1) ? scan_q8_kernel<true> : scan_q8_kernel<false>;
+            cudaError_t ke = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl8.smem_bytes);
+            if (ke != cudaSuccess) return ke;
+            kern<<<g, 32 * (pl8.nwarps + 1), pl8.smem_bytes, st>>>(p8);
+            return cudaGetLastError();
+        };
         cudaError_t e;
         TimedEvents ev{nullptr, nullptr};
         if (!timing_begin(idx, st, &ev)) return RALM_ERR_CUDA;
-        if (two_phase) {
+        if (use_q8) {
+            if (two_phase) {
+                int grid1 = 0;
+                e = scan_rows(0, sample, nullptr, &grid1);
+                if (e == cudaSuccess) {
+                    merge_kernel<<<sp, kMergeThreads, 0, st>>>(
+                        idx->partial + static_cast<size_t>(q0) * k, grid1, s, k, 0, nullptr, nullptr,
+                        idx->partial + (static_cast<size_t>(idx->num_sms) * s + q0) * k, idx->tc_thr + q0);
+                    e = cudaGetLastError();
+                }
+                if (e == cudaSuccess) e = scan_rows_q8(sample, idx->N, idx->tc_thr, &grid);
+                idx->launches += 2;
+            } else {
+                e = scan_rows_q8(0, idx->N, nullptr, &grid);
+            }
+        } else if (two_phase) {
             int grid1 = 0;
             e = scan_rows(0, sample, nullptr, &grid1);
             if (e == cudaSuccess) {
@@ -583,6 +662,8 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->tc_thr = nullptr;
     idx->tc_two_phase = true;
     idx->norms = nullptr;
+    idx->x8 = nullptr;
+    idx->x8_bound = nullptr;
     idx->spill = nullptr;
     idx->spill_cap = 0;
     cudaError_t first_error = cudaSuccess;
@@ -643,6 +724,8 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
     cudaFree(idx->tc_cand);
     cudaFree(idx->tc_thr);
     cudaFree(idx->norms);
+    cudaFree(idx->x8);
+    cudaFree(idx->x8_bound);
     cudaFree(idx->spill);
     cudaFree(idx->status);
     cudaFree(idx->h_queries);
@@ -783,6 +866,32 @@ ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant) {
     return RALM_OK;
 }
 
+ralm_status_t ralm_index_enable_q8(ralm_index_t *idx) {
+    if (!idx) return RALM_ERR_INVALID_ARG;
+    if (idx->metric != RALM_IP || idx->d % 16 != 0) return RALM_ERR_UNSUPPORTED;
+    if (idx->x8 || idx->N == 0) return RALM_OK;
+    ScanPlan probe;
+    if (!plan_scan_q8(idx, 1, &probe)) return RALM_ERR_UNSUPPORTED;
+    uint8_t *x8 = nullptr;
+    float *bound = nullptr;
+    if (device_alloc(&x8, static_cast<size_t>(idx->N) * idx->d) != cudaSuccess ||
+        device_alloc(&bound, sizeof(float) * idx->N) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(x8);
+        return RALM_ERR_OOM;
+    }
+    const int blocks = static_cast<int>(std::min<long long>((idx->N + 7) / 8, 32LL * idx->num_sms));
+    quantize_rows_kernel<<<blocks, 256>>>(idx->corpus, idx->N, idx->d, x8, bound);
+    if (cudaGetLastError() != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+        cudaFree(x8);
+        cudaFree(bound);
+        return RALM_ERR_CUDA;
+    }
+    idx->x8 = x8;
+    idx->x8_bound = bound;
+    return RALM_OK;
+}
+
 ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_metric_t metric,
                                  const void *queries, int32_t s, int32_t k, int64_t *ids,
                                  float *scores, int32_t *device_status, void *stream) {
@@ -826,6 +935,8 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.spill = nullptr;
     view.spill_cap = 0;
     view.norms = nullptr;  // no index, no stored norms: the scan derives them on the tensor cores
+    view.x8 = nullptr;
+    view.x8_bound = nullptr;
     view.status = status;
     view.h_queries = nullptr;
     view.h_ids = nullptr;

@@ -49,6 +49,8 @@ struct ScanParams {
     const __half *corpus;
     const __half *queries;  // [s][d] of this pass
     const float *norms;     // warp-MMA L2 with NRM: squared norm of every corpus row, fp32 [N]
+                            // (8-bit scan: the per-row bound of its filter)
+    const uint8_t *x8;      // 8-bit scan: the one-byte copy of the corpus, [N][d]
     uint64_t *partial;      // [gridDim.x][s_total][k] sorted keys, 0 = empty
     uint64_t *spill;        // large k: candidate lists in global memory, [gridDim.x][8][cap]; the
                             // shared-memory candidate area then holds one sort scratch of cap keys

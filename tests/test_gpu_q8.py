@@ -1,0 +1,92 @@
+"""GPU parity of the 8-bit (E5M2) corpus scan: ralm_search on an index with ralm_index_enable_q8
+against the fp64 oracle, through the C ABI. The 8-bit copy only filters; every (row, query) pair
+it lets through is scored again from the fp16 row, so the results must be those of the plain
+definition: the oracle is the same exact top-k as for every other path (Section 5.1: the exact
+dense retriever), with no tolerance of its own."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+from parity import check_search
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _search(x, q, k, q8):
+    import paper_2401_14021_b200 as ralm
+    idx = ralm.Index(x, oracle.IP, max_s=max(1, q.shape[0]), max_k=k)
+    if q8:
+        idx.enable_q8()
+        idx.enable_q8()                      # a second call is a no-op
+    ids, scores = ralm.search(idx, q, k)
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    launches = idx.launch_count()
+    idx.close()
+    return ids, scores, launches
+
+
+# Integers up to 20 in magnitude: 9, 11, 13, 15, 17, 18, 19 have no E5M2 value, so the stored
+# bound is non-zero and the filter really decides; every score is still an exact fp32 integer
+# and ties abound, so ids (tie-break included) and scores must equal the oracle's bit for bit.
+@pytest.mark.parametrize("N,d,s,k", [(1, 16, 1, 1), (15, 16, 3, 4), (17, 64, 8, 1), (33, 48, 2, 40),
+                                     (1000, 80, 8, 7), (5000, 768, 4, 5), (3001, 1024, 5, 256),
+                                     (40_000, 208, 8, 20), (9000, 128, 7, 1), (100_003, 768, 8, 1),
+                                     (2_500_000, 64, 8, 1), (2_500_000, 64, 8, 20), (2_450_001, 32, 3, 100)])
+def test_q8_integer_inputs_are_bit_exact(N, d, s, k):
+    x = workloads.integer_valued((N, d), seed=1100 + N % 1000 + d, lo=-20, hi=20, device=DEV)
+    q = workloads.integer_valued((s, d), seed=1200 + N % 1000 + d, lo=-20, hi=20, device=DEV)
+    ids, scores, _ = _search(x, q, k, q8=True)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+
+
+@pytest.mark.parametrize("N,d,s,k", [(120_001, 768, 8, 20), (2_450_000, 128, 8, 1), (2_450_000, 128, 5, 20)])
+def test_q8_mixture_rows_match_the_oracle_and_the_fp16_scan(N, d, s, k):
+    """Real-valued mixture rows (near-ties inside a cluster): the band rule against the oracle,
+    the planted source at rank 0, and the same ranking as the fp16 scan."""
+    x, _ = workloads.mixture_corpus(N, d, 64, seed=1300 + d, device=DEV)
+    q, src = workloads.noisy_copy_queries(x, s, seed=1301 + d)
+    ids, scores, _ = _search(x, q, k, q8=True)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k)
+    assert ids[:, 0].tolist() == src.tolist()
+    ids16, scores16, _ = _search(x, q, k, q8=False)
+    assert torch.equal(ids[:, 0], ids16[:, 0])
+    torch.testing.assert_close(scores, scores16, rtol=1e-5, atol=1e-6)
+
+
+def test_q8_large_values_saturate_without_losing_rows():
+    """fp16 values beyond the largest finite E5M2 value (57344) are stored saturated; the bound
+    covers the difference, so the row that holds them is still found."""
+    N, d = 4000, 64
+    x = workloads.integer_valued((N, d), seed=1400, lo=-4, hi=4, device=DEV)
+    x[1234, 5] = 65504.0
+    x[77, 9] = -65504.0
+    q = torch.zeros((2, d), dtype=torch.float16, device=DEV)
+    q[0, 5] = 1.0
+    q[1, 9] = -1.0
+    ids, scores, _ = _search(x, q, 3, q8=True)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 3, exact=True)
+    assert ids[0, 0].item() == 1234 and ids[1, 0].item() == 77
+
+
+def test_q8_is_refused_where_it_does_not_apply_and_falls_back_where_it_cannot_serve():
+    import paper_2401_14021_b200 as ralm
+    x = workloads.integer_valued((500, 24), seed=1500, lo=-3, hi=3, device=DEV)
+    idx = ralm.Index(x, oracle.IP, max_s=4, max_k=4)      # d % 16 != 0
+    with pytest.raises(ralm.RalmError):
+        idx.enable_q8()
+    idx.close()
+    x = workloads.integer_valued((500, 32), seed=1501, lo=-3, hi=3, device=DEV)
+    idx = ralm.Index(x, oracle.L2, max_s=4, max_k=4)      # the filter is an inner-product bound
+    with pytest.raises(ralm.RalmError):
+        idx.enable_q8()
+    idx.close()
+    # k beyond the 8-bit scan's limit and batches of more than 8 queries take the fp16 scans
+    q = workloads.integer_valued((12, 32), seed=1502, lo=-3, hi=3, device=DEV)
+    for s, k in ((4, 300), (12, 5)):
+        ids, scores, _ = _search(x, q[:s].contiguous(), k, q8=True)
+        check_search(ids, scores, x.cpu().numpy(), q[:s].cpu().numpy(), oracle.IP, k, exact=True)
