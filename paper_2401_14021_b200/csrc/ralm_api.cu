@@ -126,9 +126,9 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
 constexpr int kQ8MaxK = 256;
 bool plan_scan_q8(const ralm_index *idx, int k, ScanPlan *pl) {
     pl->tile_rows = 16;
-    pl->stage_bytes = align_up(pl->tile_rows * idx->d, 128);
+    pl->stage_bytes = align_up(pl->tile_rows * idx->d + kQ8TileBytesExtra, 128);
     pl->off_q = kScanHeaderBytes;
-    int off = pl->off_q + align_up(kScanMaxQueries * (idx->d * 2 + kQueryPadBytes), 128);
+    int off = pl->off_q + align_up(kScanMaxQueries * q8_query_pitch(idx->d), 128);
     pl->off_cand = off;
     pl->cap = 0;
     pl->soft_limit = 0;
@@ -145,6 +145,10 @@ bool plan_scan_q8(const ralm_index *idx, int k, ScanPlan *pl) {
     // from global memory must not hold up the producer
     pl->depth = fit >= 3 * kMaxConsumerWarps ? 3 : (fit >= 4 ? 2 : 1);
     pl->nwarps = std::min(kMaxConsumerWarps, fit / pl->depth);
+    if (idx->tune_warps > 0 && idx->tune_depth > 0 && idx->tune_warps * idx->tune_depth <= fit) {
+        pl->nwarps = std::min(idx->tune_warps, kMaxConsumerWarps);
+        pl->depth = idx->tune_depth;
+    }
     pl->smem_bytes = pl->off_stage + pl->nwarps * pl->depth * pl->stage_bytes;
     return true;
 }

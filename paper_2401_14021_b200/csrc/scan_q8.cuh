@@ -14,6 +14,12 @@
 // global memory, and only that value is compared, kept and returned. The result is therefore
 // the same as the fp16 scan's, at half the streamed bytes plus the rows that pass.
 //
+// Shared-memory banks: a lane reads 16 bytes of two rows per step, and the lanes of a quarter
+// warp hold two different rows, which collide when d is a multiple of 128 bytes. So a tile is
+// staged as two copies of 8 rows, the second shifted by 64 bytes, and MMA row m takes its data
+// from staged row q8_phys_row(m), which alternates between the two groups; the staged queries
+// get a pitch of 16 bytes modulo 128 for the same reason.
+//
 // Structure (producer warp, private stage rings per consumer warp, candidate buffers, compaction
 // meetings) is that of scan_kernel; the tile is 16 rows of d bytes. The host starts this kernel
 // from the thresholds of an fp16 scan of a small sample, without which nearly every pair would
@@ -23,6 +29,17 @@
 #include "scan.cuh"
 
 namespace ralm {
+
+// staged row (0..15, rows 8..15 sit 64 bytes further) that feeds MMA row m
+__host__ __device__ __forceinline__ int q8_phys_row(int m) {
+    return ((m & 1) << 3) + ((m & 8) >> 1) + ((m & 7) >> 1);
+}
+__host__ __device__ __forceinline__ int q8_row_offset(int phys_row, int d) {
+    return phys_row * d + ((phys_row & 8) << 3);
+}
+// bytes between staged queries: 2 d rounded up to 16 modulo 128
+__host__ __device__ __forceinline__ int q8_query_pitch(int d) { return 2 * d + (144 - (2 * d) % 128) % 128; }
+constexpr int kQ8TileBytesExtra = 64;
 
 // fp16 -> E5M2 byte, round to nearest even, saturating at the largest finite value (inputs are
 // finite). Exposed to the quantisation kernel only.
@@ -115,7 +132,7 @@ scan_q8_kernel(const ScanParams p) {
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int d = p.d;
-    const uint32_t q_pitch = static_cast<uint32_t>(d * 2 + kQueryPadBytes);
+    const uint32_t q_pitch = static_cast<uint32_t>(q8_query_pitch(d));
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < S; ++i) {
@@ -155,57 +172,19 @@ scan_q8_kernel(const ScanParams p) {
     volatile int *compact_flag = &hdr->flag;
     volatile int *done_count = &hdr->done;
 
-    if (warp == 0) {
-        // ---------------------------------------------------------------- producer
-        if (lane == 0) {
-            long long issued = 0;
-            bool ok = true;
-            int cw = 0, slot = 0;
-            uint32_t use = 0;
-            long long row0 = p.row_begin + static_cast<long long>(blockIdx.x) * T;
-            const long long row_step = static_cast<long long>(gridDim.x) * T;
-            const uint32_t stage_base = smem_u32(smem + p.off_stage);
-            for (long long it = 0; it < my_tiles; ++it) {
-                const int st = cw + slot * W;
-                if (use > 0) {
-                    ok = mbar_wait_bounded(smem_u32(&hdr->empty[st]), (use - 1) & 1);
-                    if (!ok) break;
-                }
-                if (*abort_flag) break;
-                const long long rows = (p.N - row0 < T) ? (p.N - row0) : T;
-                const uint32_t bytes = static_cast<uint32_t>(rows) * static_cast<uint32_t>(d);
-                const uint32_t bar = smem_u32(&hdr->full[st]);
-                mbar_arrive_expect_tx(bar, bytes);
-                bulk_load(stage_base + static_cast<uint32_t>(st) * p.stage_bytes, p.x8 + row0 * d, bytes, bar);
-                issued = it + 1;
-                row0 += row_step;
-                if (++cw == W) {
-                    cw = 0;
-                    if (++slot == p.depth) {
-                        slot = 0;
-                        ++use;
-                    }
-                }
-            }
-            if (!ok) {
-                atomicMax(p.status, kStatusTimeout);
-                *abort_flag = 1;
-            }
-            if (*abort_flag) {
-                // winding down early: let every copy already issued land before exit
-                for (long long it = (issued > S ? issued - S : 0); it < issued; ++it) {
-                    const long long local = it / W;
-                    mbar_wait_bounded(smem_u32(&hdr->full[(it % W) + (local % p.depth) * W]), (local / p.depth) & 1);
-                }
-            }
-        }
-    } else if (warp - 1 < W) {
+    // Every consumer warp streams its own tiles: its lane 0 refills a stage as soon as the warp has
+    // read it (a single producer thread could not issue tiles of this size fast enough). Warp 0
+    // only takes part in the set-up above.
+    if (warp >= 1 && warp - 1 < W) {
         // ---------------------------------------------------------------- consumers
         const int w = warp - 1;
         const int ctid = threadIdx.x - 32;
         const int cthreads = W * 32;
         const int g = lane >> 2, t = lane & 3;
         const uint32_t q_base_addr = smem_u32(smem + p.off_q);
+
+        long long row0 = p.row_begin + (static_cast<long long>(blockIdx.x) + static_cast<long long>(w) * gridDim.x) * T;
+        const long long row_step = static_cast<long long>(gridDim.x) * W * T;
 
         // |q| of this lane's two queries (2t, 2t + 1), rounded up
         float qn0 = 0.f, qn1 = 0.f;
@@ -224,17 +203,48 @@ scan_q8_kernel(const ScanParams p) {
 
         int slot = 0;
         uint32_t parity = 0;
-        long long row0 = p.row_begin + (static_cast<long long>(blockIdx.x) + static_cast<long long>(w) * gridDim.x) * T;
-        const long long row_step = static_cast<long long>(gridDim.x) * W * T;
+        // this warp's tiles: the CTA's tiles w, w + W, ...; the j-th goes to slot j % depth of the
+        // warp's private ring (stage w + slot * W)
+        const long long n_mine = (my_tiles > w) ? (my_tiles - w + W - 1) / W : 0;
+        const uint32_t stage_base = smem_u32(smem + p.off_stage);
+        auto issue_tile = [&](long long first_row, int slot_) {   // lane 0 only
+            const long long rows = (p.N - first_row < T) ? (p.N - first_row) : T;
+            const uint32_t bytes = static_cast<uint32_t>(rows) * static_cast<uint32_t>(d);
+            const int st_ = w + slot_ * W;
+            const uint32_t bar = smem_u32(&hdr->full[st_]);
+            mbar_arrive_expect_tx(bar, bytes);
+            // rows 0..7 and rows 8..15 as two copies, the second 64 bytes further
+            const uint32_t first = rows < 8 ? bytes : static_cast<uint32_t>(8 * d);
+            const uint32_t dst = stage_base + static_cast<uint32_t>(st_) * p.stage_bytes;
+            bulk_load(dst, p.x8 + first_row * d, first, bar);
+            if (bytes > first)
+                bulk_load(dst + first + kQ8TileBytesExtra, p.x8 + (first_row + 8) * d, bytes - first, bar);
+        };
+        long long issued = 0, landed = 0;   // of this warp's tiles (lane 0 issues; all lanes count alike)
+        for (; issued < p.depth && issued < n_mine; ++issued)
+            if (lane == 0) issue_tile(row0 + issued * row_step, static_cast<int>(issued));
+
+        // The rows' bounds are fetched one tile ahead: the tile itself is usually resident by the
+        // time its turn comes, and a load issued only then would stall the warp for a DRAM latency.
+        const int ph_lo = q8_phys_row(g), ph_hi = q8_phys_row(g + 8);
+        float e_lo_next = 0.f, e_hi_next = 0.f;
+        if (w < my_tiles) {
+            if (row0 + ph_lo < p.N) e_lo_next = __ldg(p.norms + row0 + ph_lo);
+            if (row0 + ph_hi < p.N) e_hi_next = __ldg(p.norms + row0 + ph_hi);
+        }
         for (long long it = w; it < my_tiles; it += W, row0 += row_step) {
+            const float e_lo = e_lo_next, e_hi = e_hi_next;
+            e_lo_next = e_hi_next = 0.f;
+            if (it + W < my_tiles) {
+                const long long nrow = row0 + row_step;
+                if (nrow + ph_lo < p.N) e_lo_next = __ldg(p.norms + nrow + ph_lo);
+                if (nrow + ph_hi < p.N) e_hi_next = __ldg(p.norms + nrow + ph_hi);
+            }
             if (*abort_flag) continue;
             const int st = w + slot * W;
+            const int cur_slot = slot;
             const uint32_t full_bar = smem_u32(&hdr->full[st]);
             const uint32_t my_parity = parity;
-            // the rows' bounds, in flight during the wait
-            float e_lo = 0.f, e_hi = 0.f;
-            if (row0 + g < p.N) e_lo = __ldg(p.norms + row0 + g);
-            if (row0 + g + 8 < p.N) e_hi = __ldg(p.norms + row0 + g + 8);
             if (++slot == p.depth) {
                 slot = 0;
                 parity ^= 1;
@@ -266,26 +276,39 @@ scan_q8_kernel(const ScanParams p) {
                 }
             }
             if (!have_tile) continue;
+            ++landed;
             const uint32_t stage_addr = smem_u32(smem + p.off_stage + static_cast<size_t>(st) * p.stage_bytes);
-            const uint32_t empty_bar = smem_u32(&hdr->empty[st]);
 
             // ---- 16 rows x 8 queries on tensor cores. Per step a lane takes 16 bytes of rows g
             // and g + 8 (16 elements) and the same 16 elements of query g; each 32-bit word of a
             // row unpacks into the fp16 pairs (e0, e2) and (e1, e3), which is how the query is stored.
-            float acc[4] = {0.f, 0.f, 0.f, 0.f}, acc_b[4] = {0.f, 0.f, 0.f, 0.f};
+            // four accumulator sets: each MMA depends only on the one four before it
+            float accs[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) accs[i][j] = 0.f;
             const int nchunks = (d + 63) >> 6;
             const uint32_t q_addr = q_base_addr + g * q_pitch;
-            const uint32_t a_lo_addr = stage_addr + g * d;
-            const uint32_t a_hi_addr = stage_addr + (g + 8) * d;
-#pragma unroll 2
+            const uint32_t a_lo_addr = stage_addr + q8_row_offset(ph_lo, d);
+            const uint32_t a_hi_addr = stage_addr + q8_row_offset(ph_hi, d);
+            // (the loads of step c + 1 are issued before the MMAs of step c)
+            uint4 lo = make_uint4(0, 0, 0, 0), hi = lo, b0 = lo, b1 = lo;
+            if (t * 16 < d) {
+                lo = lds128(a_lo_addr + t * 16);
+                hi = lds128(a_hi_addr + t * 16);
+                b0 = lds128(q_addr + t * 32);
+                b1 = lds128(q_addr + t * 32 + 16);
+            }
+#pragma unroll 4
             for (int c = 0; c < nchunks; ++c) {
-                const int off = c * 64 + t * 16;
-                uint4 lo = make_uint4(0, 0, 0, 0), hi = lo, b0 = lo, b1 = lo;
+                const int off = (c + 1) * 64 + t * 16;
+                uint4 nlo = make_uint4(0, 0, 0, 0), nhi = nlo, nb0 = nlo, nb1 = nlo;
                 if (off < d) {  // ragged last chunk: absent pieces stay zero (the MMAs are warp-wide)
-                    lo = lds128(a_lo_addr + off);
-                    hi = lds128(a_hi_addr + off);
-                    b0 = lds128(q_addr + off * 2);
-                    b1 = lds128(q_addr + off * 2 + 16);
+                    nlo = lds128(a_lo_addr + off);
+                    nhi = lds128(a_hi_addr + off);
+                    nb0 = lds128(q_addr + off * 2);
+                    nb1 = lds128(q_addr + off * 2 + 16);
                 }
                 const uint32_t lw[4] = {lo.x, lo.y, lo.z, lo.w};
                 const uint32_t hw[4] = {hi.x, hi.y, hi.z, hi.w};
@@ -294,18 +317,28 @@ scan_q8_kernel(const ScanParams p) {
                 for (int i = 0; i < 4; ++i) {
                     const uint32_t l02 = __byte_perm(lw[i], 0u, 0x2404), l13 = lw[i] & 0xff00ff00u;
                     const uint32_t h02 = __byte_perm(hw[i], 0u, 0x2404), h13 = hw[i] & 0xff00ff00u;
-                    if (i & 1) mma_m16n8k16(acc_b, l02, h02, l13, h13, bw[2 * i], bw[2 * i + 1]);
-                    else mma_m16n8k16(acc, l02, h02, l13, h13, bw[2 * i], bw[2 * i + 1]);
+                    mma_m16n8k16(accs[i], l02, h02, l13, h13, bw[2 * i], bw[2 * i + 1]);
                 }
+                lo = nlo;
+                hi = nhi;
+                b0 = nb0;
+                b1 = nb1;
             }
+            float acc[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc[i] += acc_b[i];
+            for (int i = 0; i < 4; ++i) acc[i] = (accs[0][i] + accs[1][i]) + (accs[2][i] + accs[3][i]);
+            // every lane has read the stage, since the MMAs above have consumed what it loaded (the
+            // rest works from registers and global memory):
+            // refill it with this warp's tile `depth` further on
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty_bar);  // the rest works from registers and global memory
+            if (issued < n_mine && !*abort_flag) {
+                if (lane == 0) issue_tile(row0 + static_cast<long long>(p.depth) * row_step, cur_slot);
+                ++issued;
+            }
 
-            // acc[0]: (row g, query 2t)     acc[1]: (row g, query 2t+1)
-            // acc[2]: (row g+8, query 2t)   acc[3]: (row g+8, query 2t+1)
-            const long long r_lo = row0 + g, r_hi = row0 + g + 8;
+            // acc[0]: (MMA row g, query 2t)     acc[1]: (MMA row g, query 2t+1)
+            // acc[2]: (MMA row g+8, query 2t)   acc[3]: (MMA row g+8, query 2t+1)
+            const long long r_lo = row0 + ph_lo, r_hi = row0 + ph_hi;
             const int q0 = 2 * t, q1 = q0 + 1;
             float th0 = *reinterpret_cast<volatile float *>(&hdr->thr[q0]);
             float th1 = *reinterpret_cast<volatile float *>(&hdr->thr[q1]);
@@ -326,7 +359,7 @@ scan_q8_kernel(const ScanParams p) {
                 while (m) {
                     const int src = __ffs(m) - 1;
                     m &= m - 1;
-                    const int row_local = (src >> 2) + ((i & 2) ? 8 : 0);
+                    const int row_local = q8_phys_row((src >> 2) + ((i & 2) ? 8 : 0));
                     const int q = 2 * (src & 3) + (i & 1);
                     const long long row = row0 + row_local;
                     const float val = warp_exact_ip(p.corpus + row * d, q_base_addr + q * q_pitch, d, lane);
@@ -342,6 +375,12 @@ scan_q8_kernel(const ScanParams p) {
                 }
             }
         }
+
+        // winding down early: let every copy this warp has issued land before the CTA exits
+        if (lane == 0)
+            for (long long j = landed; j < issued; ++j)
+                mbar_wait_bounded(smem_u32(&hdr->full[w + static_cast<int>(j % p.depth) * W]),
+                                  static_cast<uint32_t>((j / p.depth) & 1));
 
         // ------------------------------------------------------------ CTA result
         if (TOP1) {
