@@ -115,6 +115,31 @@ def test_c3_serving_step_cache_and_verify(c3_corpus):
     idx.close()
 
 
+@pytest.mark.parametrize("k", [1, 20])
+def test_c3_full_size_s8_with_8bit_filter_copy(c3_corpus, k):
+    """The headline configuration through the 8-bit scan (ralm_index_enable_q8: the one-byte copy
+    filters, every pair it lets through is scored again from the fp16 row): the same sampled
+    check against the oracle, and the same lists as the fp16 scan of the same index shape."""
+    ralm = _ralm()
+    x, _ = c3_corpus
+    q, src = workloads.noisy_copy_queries(x, 8, workloads.seed_for(3, "queries"))
+    idx = ralm.Index(x, oracle.IP, max_s=8, max_k=k)
+    ids16, scores16 = ralm.search(idx, q, k)
+    idx.enable_q8()
+    ids, scores = ralm.search(idx, q, k)
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    assert ids[:, 0].tolist() == src.tolist()
+    strict, band, n_sub = _sampled_parity(x, q, ids, scores, oracle.IP, k, 30, 16_384, seed=3700 + k)
+    print("C3 8-bit scan k=%d: strict=%d band=%d over a %d-row sub-corpus" % (k, strict, band, n_sub))
+    assert torch.equal(ids[:, 0], ids16[:, 0])
+    torch.testing.assert_close(scores, scores16, rtol=1e-5, atol=1e-6)
+    for s in (1, 5):
+        ids_s, _ = ralm.search(idx, q[:s].contiguous(), k)
+        assert torch.equal(ids_s, ids[:s])
+    idx.close()
+
+
 @pytest.mark.parametrize("s,k", [(16, 1), (16, 20), (32, 20), (64, 20)])
 def test_c3_full_size_mid_batches(c3_corpus, s, k):
     """Between the two headline cases: 16 and 32 queries run as one pass of the small-batch scan
