@@ -354,10 +354,12 @@ def main():
                                 if cfg.metric == "ip" and args.variant in (0, 2) and not args.tune
                                 and s <= 8 else None),
                     "traffic_note": "2M-row ncu capture scaled by rows; null if the kernel changed since"}
-        if args.q8 and cfg.metric == "ip" and args.variant == 0 and s <= 8 and k <= 256:
+        uses_q8 = args.q8 and cfg.metric == "ip" and args.variant == 0 and \
+            ((s <= 8 and k <= 256) or (s <= 16 and k <= 64)) and max(N // 128, 4 * 148 * 128) * 32 <= N
+        if uses_q8:
             # the 8-bit scan streams the one-byte copy and one fp32 bound per row; the sample
             # (1/128 of the rows, when the corpus is large enough for one) is scanned in fp16
-            sample = max(N // 128, 4 * 148 * 128) if max(N // 128, 4 * 148 * 128) * 32 <= N else 0
+            sample = max(N // 128, 4 * 148 * 128)
             q8_bytes = sample * d * 2 + (N - sample) * (d + 4)
             achieved = q8_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None
             roofline.update({"achieved": achieved, "frac": achieved / peaks["hbm_gbs"] if achieved else None,
@@ -366,7 +368,8 @@ def main():
                              "fp16_equivalent_gbs": corpus_bytes / (scan_avg_ms * 1e-3) / 1e9
                              if scan_launches else None})
         uses_tc = k <= 64 and d >= 64 and (cfg.metric == "ip" or N >= 700_000) and \
-            (args.variant in (3, 4) or (args.variant == 0 and s >= 9))
+            (args.variant in (3, 4) or (args.variant == 0 and not uses_q8 and
+                                        s >= (33 if cfg.metric == "ip" else 17)))
         if uses_tc:
             roofline["kernel"] = "scan_tc_kernel"
         if uses_tc and s > 255:

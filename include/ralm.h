@@ -204,17 +204,19 @@ ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant);
 
 /* Optional for inner-product indexes: build a one-byte-per-element copy of the corpus (E5M2,
  * N * d bytes, plus one fp32 bound per row) that ralm_search then streams instead of the fp16 rows
- * for batches of up to 8 queries with k <= 256 under the automatic variant. The copy only
+ * for batches of up to 8 queries with k <= 256, and of 9..16 queries with k <= 64, under the
+ * automatic variant (other shapes take the fp16 scans). The copy only
  * FILTERS: by the Cauchy-Schwarz inequality the score of the rounded row is within
  * |q| * |x - x8| of the true one, a (row, query) pair whose upper bound cannot reach the score
  * that k rows are already known to reach is dropped, and every other pair is scored again from
  * the fp16 row, which is the value that is ranked and returned. Results are those of the fp16
  * scan (what the paper's exact dense retriever returns, Section 5.1); the bytes streamed per
- * batch drop to about half. Worth it on corpora large enough for the sample phase (about
- * 2.4 M rows); smaller ones are served correctly but without thresholds to start from.
+ * batch drop to about half. The copy is used on corpora large enough for the sample phase that
+ * gives the filter its thresholds (about 2.4 M rows); smaller ones keep the fp16 scan unless
+ * `force` is non-zero (a testing aid: correct, but slow without thresholds to start from).
  * One pass over the corpus on the default stream, synchronous; allocates device memory.
- * Errors: UNSUPPORTED for L2 indexes or d % 16 != 0; OOM. Calling it again is a no-op. */
-ralm_status_t ralm_index_enable_q8(ralm_index_t *idx);
+ * Errors: UNSUPPORTED for L2 indexes or d % 16 != 0; OOM. Calling it again only updates `force`. */
+ralm_status_t ralm_index_enable_q8(ralm_index_t *idx, int32_t force);
 
 /* Override the scan kernel's launch shape on this index (benchmarking aid; 0 keeps the
  * library's choice): consumer warps per CTA (1..8), shared-memory stages per consumer warp,

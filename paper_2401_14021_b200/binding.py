@@ -61,7 +61,7 @@ def load_library() -> ctypes.CDLL:
     lib.ralm_device_status.restype = i32
     lib.ralm_device_status.argtypes = [p, p]
     lib.ralm_index_enable_q8.restype = i32
-    lib.ralm_index_enable_q8.argtypes = [p]
+    lib.ralm_index_enable_q8.argtypes = [p, i32]
     lib.ralm_index_set_variant.restype = i32
     lib.ralm_index_set_variant.argtypes = [p, i32]
     lib.ralm_index_set_tuning.restype = i32
@@ -137,8 +137,8 @@ class Index:
     def handle(self):
         return self._handle
 
-    def enable_q8(self):
-        _check(self._lib.ralm_index_enable_q8(self._handle), "ralm_index_enable_q8")
+    def enable_q8(self, force: bool = False):
+        _check(self._lib.ralm_index_enable_q8(self._handle, int(force)), "ralm_index_enable_q8")
 
     def set_variant(self, variant: int):
         _check(self._lib.ralm_index_set_variant(self._handle, variant), "ralm_index_set_variant")

@@ -37,6 +37,7 @@ struct ralm_index {
     float *norms;          // L2: squared norm of every corpus row (fp32 [N]), or null
     uint8_t *x8;           // inner product, optional: one-byte (E5M2) copy of the corpus, [N][d]
     float *x8_bound;       // per row: bound on |q.x - q.x8| per unit of |q| (see scan_q8.cuh)
+    bool x8_force;         // use the copy also on corpora too small for a sample phase (testing aid)
     float *tc_thr;         // thresholds from the sample phase of a two-phase scan, [max_s]
     bool tc_two_phase;     // sample phase enabled (tuning aid)
     int tc_clusters;       // CTA pairs the device runs at once (-1 = not asked yet)
@@ -121,22 +122,27 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
     return true;
 }
 
-// Shared-memory layout of one CTA of the 8-bit scan: 16-row tiles of d bytes, 8 staged queries,
-// candidate lists in shared memory (k <= kQ8MaxK keeps them within kSmemCandBytes).
+// Shared-memory layout of one CTA of the 8-bit scan: 16-row tiles of d bytes, 8 or 16 staged
+// queries, candidate lists in shared memory: k <= kQ8MaxK for up to 8 queries, k <= kQ8MaxKWide
+// (lists of 256 slots) for 9..16, which keeps them within kSmemCandBytes.
 constexpr int kQ8MaxK = 256;
-bool plan_scan_q8(const ralm_index *idx, int k, ScanPlan *pl) {
+constexpr int kQ8MaxKWide = 64;
+constexpr int kQ8MaxQueries = 2 * kScanMaxQueries;
+bool plan_scan_q8(const ralm_index *idx, int s_pass, int k, ScanPlan *pl) {
+    const int q_rows = s_pass > kScanMaxQueries ? kQ8MaxQueries : kScanMaxQueries;
+    if (s_pass > kQ8MaxQueries || k > (q_rows > kScanMaxQueries ? kQ8MaxKWide : kQ8MaxK)) return false;
     pl->tile_rows = 16;
     pl->stage_bytes = align_up(pl->tile_rows * idx->d + kQ8TileBytesExtra, 128);
     pl->off_q = kScanHeaderBytes;
-    int off = pl->off_q + align_up(kScanMaxQueries * q8_query_pitch(idx->d), 128);
+    int off = pl->off_q + align_up(q_rows * q8_query_pitch(idx->d), 128);
     pl->off_cand = off;
     pl->cap = 0;
     pl->soft_limit = 0;
     pl->spill = false;
     if (k > 1) {
-        pl->cap = std::max(512, 2 * next_pow2(k));
+        pl->cap = q_rows > kScanMaxQueries ? 256 : std::max(512, 2 * next_pow2(k));
         pl->soft_limit = std::min(pl->cap - (kMaxConsumerWarps + 1) * pl->tile_rows, std::max(4 * k, 64));
-        off += kScanMaxQueries * pl->cap * 8;
+        off += q_rows * pl->cap * 8;
     }
     pl->off_stage = align_up(off, 128);
     const int fit = std::min(kMaxStages, (idx->smem_optin - pl->off_stage) / pl->stage_bytes);
@@ -422,19 +428,22 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     const bool wide = mma && s > kScanMaxQueries && (idx->metric == RALM_IP || idx->norms != nullptr);
     // (L2 stops at two groups: with four, its filter and rescoring cost more than a second pass)
     const int wide_pass = idx->metric == RALM_L2 ? 16 : kScanMaxPassQueries;
-    const int per_pass = mma ? (wide ? wide_pass : kScanMaxQueries) : kFmaQueriesPerPass;
+    // An index with an 8-bit copy (ralm_index_enable_q8) streams that copy for batches of up to 16
+    // queries and scores again, exactly, what its filter lets through; the sample is scanned in
+    // fp16 also for k == 1, since the filter needs thresholds to be of any use.
+    ScanPlan pl8;
+    // (only where a sample phase is possible: without thresholds nearly every pair passes the filter)
+    const long long q8_sample = (std::max<long long>(idx->N / 128, 4LL * idx->num_sms * kTcTileM) + 255) / 256 * 256;
+    const bool use_q8 = idx->x8 && idx->metric == RALM_IP && idx->variant == 0 && s <= kQ8MaxQueries &&
+                        (idx->x8_force || (idx->tc_thr && idx->tc_two_phase && q8_sample * 32 <= idx->N)) &&
+                        plan_scan_q8(idx, s, k, &pl8);
+    const int per_pass = use_q8 ? kQ8MaxQueries : mma ? (wide ? wide_pass : kScanMaxQueries) : kFmaQueriesPerPass;
     // k > 1 on a large corpus: scan a sample first and start the rest from the sample's merged
     // k-th scores (see the large-batch path above); the sample's list is block num_sms of `partial`
     // (1/128 of the rows here: measured best for this scan; the large-batch scan prefers 1/64)
     long long sample = std::max<long long>(idx->N / 128, 4LL * idx->num_sms * kTcTileM);
     sample = (sample + 255) / 256 * 256;
     // (two more launches: only worth it when the scan itself takes a millisecond or more)
-    // An index with an 8-bit copy (ralm_index_enable_q8) streams that copy for batches of up to 8
-    // queries and scores again, exactly, what its filter lets through; the sample is scanned in
-    // fp16 also for k == 1, since the filter needs thresholds to be of any use.
-    ScanPlan pl8;
-    const bool use_q8 = idx->x8 && idx->metric == RALM_IP && idx->variant == 0 && s <= kScanMaxQueries &&
-                        k <= kQ8MaxK && plan_scan_q8(idx, k, &pl8);
     const bool two_phase = (k > 1 || use_q8) && idx->tc_thr && idx->tc_two_phase && sample * 32 <= idx->N;
     int grid = 0;
     for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
@@ -517,7 +526,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             p8.ntiles = (end - begin + pl8.tile_rows - 1) / pl8.tile_rows;
             const int g = static_cast<int>(std::min<long long>(idx->num_sms, (end - begin + 15) / 16));
             *grid_out = g;
-            auto kern = (k == 1) ? scan_q8_kernel<true> : scan_q8_kernel<false>;
+            auto kern = (k == 1) ? scan_q8_kernel<true, 1> : scan_q8_kernel<false, 1>;
+            if (sp > kScanMaxQueries) kern = (k == 1) ? scan_q8_kernel<true, 2> : scan_q8_kernel<false, 2>;
             cudaError_t ke = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl8.smem_bytes);
             if (ke != cudaSuccess) return ke;
             kern<<<g, 32 * (pl8.nwarps + 1), pl8.smem_bytes, st>>>(p8);
@@ -668,6 +678,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->norms = nullptr;
     idx->x8 = nullptr;
     idx->x8_bound = nullptr;
+    idx->x8_force = false;
     idx->spill = nullptr;
     idx->spill_cap = 0;
     cudaError_t first_error = cudaSuccess;
@@ -870,12 +881,13 @@ ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant) {
     return RALM_OK;
 }
 
-ralm_status_t ralm_index_enable_q8(ralm_index_t *idx) {
+ralm_status_t ralm_index_enable_q8(ralm_index_t *idx, int32_t force) {
     if (!idx) return RALM_ERR_INVALID_ARG;
     if (idx->metric != RALM_IP || idx->d % 16 != 0) return RALM_ERR_UNSUPPORTED;
+    idx->x8_force = force != 0;
     if (idx->x8 || idx->N == 0) return RALM_OK;
     ScanPlan probe;
-    if (!plan_scan_q8(idx, 1, &probe)) return RALM_ERR_UNSUPPORTED;
+    if (!plan_scan_q8(idx, 1, 1, &probe)) return RALM_ERR_UNSUPPORTED;
     uint8_t *x8 = nullptr;
     float *bound = nullptr;
     if (device_alloc(&x8, static_cast<size_t>(idx->N) * idx->d) != cudaSuccess ||
@@ -941,6 +953,7 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.norms = nullptr;  // no index, no stored norms: the scan derives them on the tensor cores
     view.x8 = nullptr;
     view.x8_bound = nullptr;
+    view.x8_force = false;
     view.status = status;
     view.h_queries = nullptr;
     view.h_ids = nullptr;

@@ -119,8 +119,9 @@ __device__ __forceinline__ float warp_exact_ip(const __half *row, uint32_t q_add
 }
 
 // p.x8: the 8-bit copy; p.norms: the per-row bound e_j; p.corpus: the fp16 rows (rescoring).
-// Up to 8 queries per pass; p.tile_rows == 16; d % 16 == 0.
-template <bool TOP1>
+// NG groups of 8 queries per pass share every staged tile (NG = 1 or 2); p.tile_rows == 16;
+// d % 16 == 0.
+template <bool TOP1, int NG>
 __global__ void __launch_bounds__(kScanThreads, 1)
 scan_q8_kernel(const ScanParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -150,11 +151,11 @@ scan_q8_kernel(const ScanParams p) {
         hdr->best[threadIdx.x] = 0ull;
     }
     {
-        // queries as fp16 [8][d] in shared memory, rows >= s zeroed, every group of four elements
+        // queries as fp16 [8 NG][d] in shared memory, rows >= s zeroed, every group of four elements
         // stored as (e0, e2, e1, e3): the order in which a 32-bit word of the 8-bit rows unpacks
         const uint2 *qg = reinterpret_cast<const uint2 *>(p.queries);
         const int per_row = d / 4;
-        for (int i = threadIdx.x; i < kScanMaxQueries * per_row; i += blockDim.x) {
+        for (int i = threadIdx.x; i < NG * kScanMaxQueries * per_row; i += blockDim.x) {
             const int row = i / per_row, col = i - row * per_row;
             uint2 v = make_uint2(0u, 0u);
             if (row < p.s) {
@@ -187,18 +188,21 @@ scan_q8_kernel(const ScanParams p) {
         const long long row_step = static_cast<long long>(gridDim.x) * W * T;
 
         // |q| of this lane's two queries (2t, 2t + 1), rounded up
-        float qn0 = 0.f, qn1 = 0.f;
-        {
-            const __half *qa = reinterpret_cast<const __half *>(smem + p.off_q + (2 * t) * q_pitch);
-            const __half *qb = reinterpret_cast<const __half *>(smem + p.off_q + (2 * t + 1) * q_pitch);
+        float qn0[NG], qn1[NG];
+#pragma unroll
+        for (int grp = 0; grp < NG; ++grp) {
+            const int row_a = grp * kScanMaxQueries + 2 * t;
+            const __half *qa = reinterpret_cast<const __half *>(smem + p.off_q + row_a * q_pitch);
+            const __half *qb = reinterpret_cast<const __half *>(smem + p.off_q + (row_a + 1) * q_pitch);
+            float a2 = 0.f, b2 = 0.f;
             for (int i = 0; i < d; ++i) {
                 const float a = __half2float(qa[i]), b = __half2float(qb[i]);
-                qn0 = fmaf(a, a, qn0);
-                qn1 = fmaf(b, b, qn1);
+                a2 = fmaf(a, a, a2);
+                b2 = fmaf(b, b, b2);
             }
             const float up = 1.0f + 1.0f / 1024.0f;
-            qn0 = __fmul_ru(__fsqrt_ru(qn0), up);
-            qn1 = __fmul_ru(__fsqrt_ru(qn1), up);
+            qn0[grp] = __fmul_ru(__fsqrt_ru(a2), up);
+            qn1[grp] = __fmul_ru(__fsqrt_ru(b2), up);
         }
 
         int slot = 0;
@@ -282,51 +286,79 @@ scan_q8_kernel(const ScanParams p) {
             // ---- 16 rows x 8 queries on tensor cores. Per step a lane takes 16 bytes of rows g
             // and g + 8 (16 elements) and the same 16 elements of query g; each 32-bit word of a
             // row unpacks into the fp16 pairs (e0, e2) and (e1, e3), which is how the query is stored.
-            // four accumulator sets: each MMA depends only on the one four before it
-            float accs[4][4];
+            // several accumulator sets per group shorten the chain of dependent MMAs
+            constexpr int NA = NG == 1 ? 4 : 2;
+            float accs[NG][NA][4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int grp = 0; grp < NG; ++grp)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) accs[i][j] = 0.f;
+                for (int i = 0; i < NA; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) accs[grp][i][j] = 0.f;
             const int nchunks = (d + 63) >> 6;
             const uint32_t q_addr = q_base_addr + g * q_pitch;
+            const uint32_t grp_pitch = kScanMaxQueries * q_pitch;
             const uint32_t a_lo_addr = stage_addr + q8_row_offset(ph_lo, d);
             const uint32_t a_hi_addr = stage_addr + q8_row_offset(ph_hi, d);
             // (the loads of step c + 1 are issued before the MMAs of step c)
-            uint4 lo = make_uint4(0, 0, 0, 0), hi = lo, b0 = lo, b1 = lo;
+            uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
+            uint4 b0[NG], b1[NG];
+#pragma unroll
+            for (int grp = 0; grp < NG; ++grp) b0[grp] = b1[grp] = lo;
             if (t * 16 < d) {
                 lo = lds128(a_lo_addr + t * 16);
                 hi = lds128(a_hi_addr + t * 16);
-                b0 = lds128(q_addr + t * 32);
-                b1 = lds128(q_addr + t * 32 + 16);
+#pragma unroll
+                for (int grp = 0; grp < NG; ++grp) {
+                    b0[grp] = lds128(q_addr + grp * grp_pitch + t * 32);
+                    b1[grp] = lds128(q_addr + grp * grp_pitch + t * 32 + 16);
+                }
             }
 #pragma unroll 4
             for (int c = 0; c < nchunks; ++c) {
                 const int off = (c + 1) * 64 + t * 16;
-                uint4 nlo = make_uint4(0, 0, 0, 0), nhi = nlo, nb0 = nlo, nb1 = nlo;
+                uint4 nlo = make_uint4(0, 0, 0, 0), nhi = nlo;
+                uint4 nb0[NG], nb1[NG];
+#pragma unroll
+                for (int grp = 0; grp < NG; ++grp) nb0[grp] = nb1[grp] = nlo;
                 if (off < d) {  // ragged last chunk: absent pieces stay zero (the MMAs are warp-wide)
                     nlo = lds128(a_lo_addr + off);
                     nhi = lds128(a_hi_addr + off);
-                    nb0 = lds128(q_addr + off * 2);
-                    nb1 = lds128(q_addr + off * 2 + 16);
+#pragma unroll
+                    for (int grp = 0; grp < NG; ++grp) {
+                        nb0[grp] = lds128(q_addr + grp * grp_pitch + off * 2);
+                        nb1[grp] = lds128(q_addr + grp * grp_pitch + off * 2 + 16);
+                    }
                 }
                 const uint32_t lw[4] = {lo.x, lo.y, lo.z, lo.w};
                 const uint32_t hw[4] = {hi.x, hi.y, hi.z, hi.w};
-                const uint32_t bw[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const uint32_t l02 = __byte_perm(lw[i], 0u, 0x2404), l13 = lw[i] & 0xff00ff00u;
                     const uint32_t h02 = __byte_perm(hw[i], 0u, 0x2404), h13 = hw[i] & 0xff00ff00u;
-                    mma_m16n8k16(accs[i], l02, h02, l13, h13, bw[2 * i], bw[2 * i + 1]);
+#pragma unroll
+                    for (int grp = 0; grp < NG; ++grp) {
+                        const uint32_t bw[8] = {b0[grp].x, b0[grp].y, b0[grp].z, b0[grp].w,
+                                                b1[grp].x, b1[grp].y, b1[grp].z, b1[grp].w};
+                        mma_m16n8k16(accs[grp][i % NA], l02, h02, l13, h13, bw[2 * i], bw[2 * i + 1]);
+                    }
                 }
                 lo = nlo;
                 hi = nhi;
-                b0 = nb0;
-                b1 = nb1;
-            }
-            float acc[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc[i] = (accs[0][i] + accs[1][i]) + (accs[2][i] + accs[3][i]);
+                for (int grp = 0; grp < NG; ++grp) {
+                    b0[grp] = nb0[grp];
+                    b1[grp] = nb1[grp];
+                }
+            }
+            float acc[NG][4];
+#pragma unroll
+            for (int grp = 0; grp < NG; ++grp)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    acc[grp][i] = accs[grp][0][i] + accs[grp][1][i];
+                    if (NA == 4) acc[grp][i] += accs[grp][2 % NA][i] + accs[grp][3 % NA][i];
+                }
             // every lane has read the stage, since the MMAs above have consumed what it loaded (the
             // rest works from registers and global memory):
             // refill it with this warp's tile `depth` further on
@@ -339,37 +371,40 @@ scan_q8_kernel(const ScanParams p) {
             // acc[0]: (MMA row g, query 2t)     acc[1]: (MMA row g, query 2t+1)
             // acc[2]: (MMA row g+8, query 2t)   acc[3]: (MMA row g+8, query 2t+1)
             const long long r_lo = row0 + ph_lo, r_hi = row0 + ph_hi;
-            const int q0 = 2 * t, q1 = q0 + 1;
-            float th0 = *reinterpret_cast<volatile float *>(&hdr->thr[q0]);
-            float th1 = *reinterpret_cast<volatile float *>(&hdr->thr[q1]);
-            if (TOP1) {
-                const unsigned long long k0 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[q0]);
-                const unsigned long long k1 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[q1]);
-                if (k0) th0 = fmaxf(th0, key_value(k0));
-                if (k1) th1 = fmaxf(th1, key_value(k1));
-            }
-            bool pass[4];
-            pass[0] = r_lo < p.N && q0 < p.s && __fmaf_ru(qn0, e_lo, acc[0]) >= th0;
-            pass[1] = r_lo < p.N && q1 < p.s && __fmaf_ru(qn1, e_lo, acc[1]) >= th1;
-            pass[2] = r_hi < p.N && q0 < p.s && __fmaf_ru(qn0, e_hi, acc[2]) >= th0;
-            pass[3] = r_hi < p.N && q1 < p.s && __fmaf_ru(qn1, e_hi, acc[3]) >= th1;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                unsigned m = __ballot_sync(0xffffffffu, pass[i]);
-                while (m) {
-                    const int src = __ffs(m) - 1;
-                    m &= m - 1;
-                    const int row_local = q8_phys_row((src >> 2) + ((i & 2) ? 8 : 0));
-                    const int q = 2 * (src & 3) + (i & 1);
-                    const long long row = row0 + row_local;
-                    const float val = warp_exact_ip(p.corpus + row * d, q_base_addr + q * q_pitch, d, lane);
-                    if (lane == 0) {
-                        const uint64_t key = make_key(val, static_cast<uint32_t>(row));
-                        if (TOP1) {
-                            if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q]))
-                                atomicMax(&hdr->best[q], static_cast<unsigned long long>(key));
-                        } else if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q])) {
-                            push_candidate(hdr, cand, p.cap, p.soft_limit, q, key);
+            for (int grp = 0; grp < NG; ++grp) {
+                const int q0 = grp * kScanMaxQueries + 2 * t, q1 = q0 + 1;
+                float th0 = *reinterpret_cast<volatile float *>(&hdr->thr[q0]);
+                float th1 = *reinterpret_cast<volatile float *>(&hdr->thr[q1]);
+                if (TOP1) {
+                    const unsigned long long k0 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[q0]);
+                    const unsigned long long k1 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[q1]);
+                    if (k0) th0 = fmaxf(th0, key_value(k0));
+                    if (k1) th1 = fmaxf(th1, key_value(k1));
+                }
+                bool pass[4];
+                pass[0] = r_lo < p.N && q0 < p.s && __fmaf_ru(qn0[grp], e_lo, acc[grp][0]) >= th0;
+                pass[1] = r_lo < p.N && q1 < p.s && __fmaf_ru(qn1[grp], e_lo, acc[grp][1]) >= th1;
+                pass[2] = r_hi < p.N && q0 < p.s && __fmaf_ru(qn0[grp], e_hi, acc[grp][2]) >= th0;
+                pass[3] = r_hi < p.N && q1 < p.s && __fmaf_ru(qn1[grp], e_hi, acc[grp][3]) >= th1;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    unsigned m = __ballot_sync(0xffffffffu, pass[i]);
+                    while (m) {
+                        const int src = __ffs(m) - 1;
+                        m &= m - 1;
+                        const int row_local = q8_phys_row((src >> 2) + ((i & 2) ? 8 : 0));
+                        const int q = grp * kScanMaxQueries + 2 * (src & 3) + (i & 1);
+                        const long long row = row0 + row_local;
+                        const float val = warp_exact_ip(p.corpus + row * d, q_base_addr + q * q_pitch, d, lane);
+                        if (lane == 0) {
+                            const uint64_t key = make_key(val, static_cast<uint32_t>(row));
+                            if (TOP1) {
+                                if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q]))
+                                    atomicMax(&hdr->best[q], static_cast<unsigned long long>(key));
+                            } else if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q])) {
+                                push_candidate(hdr, cand, p.cap, p.soft_limit, q, key);
+                            }
                         }
                     }
                 }

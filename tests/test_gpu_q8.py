@@ -20,8 +20,10 @@ def _search(x, q, k, q8):
     import paper_2401_14021_b200 as ralm
     idx = ralm.Index(x, oracle.IP, max_s=max(1, q.shape[0]), max_k=k)
     if q8:
-        idx.enable_q8()
-        idx.enable_q8()                      # a second call is a no-op
+        # (forced: most of these corpora are too small for the sample phase, without which the
+        # library would keep the fp16 scan)
+        idx.enable_q8(force=True)
+        idx.enable_q8(force=True)            # a second call builds nothing
     ids, scores = ralm.search(idx, q, k)
     torch.cuda.synchronize()
     assert idx.device_status() == 0
@@ -36,7 +38,9 @@ def _search(x, q, k, q8):
 @pytest.mark.parametrize("N,d,s,k", [(1, 16, 1, 1), (15, 16, 3, 4), (17, 64, 8, 1), (33, 48, 2, 40),
                                      (1000, 80, 8, 7), (5000, 768, 4, 5), (3001, 1024, 5, 256),
                                      (40_000, 208, 8, 20), (9000, 128, 7, 1), (100_003, 768, 8, 1),
-                                     (2_500_000, 64, 8, 1), (2_500_000, 64, 8, 20), (2_450_001, 32, 3, 100)])
+                                     (2_500_000, 64, 8, 1), (2_500_000, 64, 8, 20), (2_450_001, 32, 3, 100),
+                                     (700, 48, 9, 1), (5000, 768, 16, 5), (40_000, 208, 12, 64), (33, 64, 16, 40),
+                                     (2_450_000, 32, 16, 1), (2_450_000, 32, 13, 20)])
 def test_q8_integer_inputs_are_bit_exact(N, d, s, k):
     x = workloads.integer_valued((N, d), seed=1100 + N % 1000 + d, lo=-20, hi=20, device=DEV)
     q = workloads.integer_valued((s, d), seed=1200 + N % 1000 + d, lo=-20, hi=20, device=DEV)
@@ -44,7 +48,8 @@ def test_q8_integer_inputs_are_bit_exact(N, d, s, k):
     check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
 
 
-@pytest.mark.parametrize("N,d,s,k", [(120_001, 768, 8, 20), (2_450_000, 128, 8, 1), (2_450_000, 128, 5, 20)])
+@pytest.mark.parametrize("N,d,s,k", [(120_001, 768, 8, 20), (2_450_000, 128, 8, 1), (2_450_000, 128, 5, 20),
+                                     (2_450_000, 128, 16, 20), (60_000, 768, 11, 1)])
 def test_q8_mixture_rows_match_the_oracle_and_the_fp16_scan(N, d, s, k):
     """Real-valued mixture rows (near-ties inside a cluster): the band rule against the oracle,
     the planted source at rank 0, and the same ranking as the fp16 scan."""
@@ -73,6 +78,22 @@ def test_q8_large_values_saturate_without_losing_rows():
     assert ids[0, 0].item() == 1234 and ids[1, 0].item() == 77
 
 
+def test_q8_unforced_small_corpus_keeps_the_fp16_scan_and_large_one_uses_the_copy():
+    import paper_2401_14021_b200 as ralm
+    for N, uses in ((200_000, False), (2_450_000, True)):
+        x = workloads.integer_valued((N, 32), seed=1600, lo=-20, hi=20, device=DEV)
+        q = workloads.integer_valued((8, 32), seed=1601, lo=-20, hi=20, device=DEV)
+        idx = ralm.Index(x, oracle.IP, max_s=8, max_k=1)
+        idx.enable_q8()
+        before = idx.launch_count()
+        ids, scores = ralm.search(idx, q, 1)
+        torch.cuda.synchronize()
+        # the 8-bit path is sample scan + merge + 8-bit scan + merge; the plain top-1 scan is 2 launches
+        assert (idx.launch_count() - before == 4) == uses
+        idx.close()
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 1, exact=True)
+
+
 def test_q8_is_refused_where_it_does_not_apply_and_falls_back_where_it_cannot_serve():
     import paper_2401_14021_b200 as ralm
     x = workloads.integer_valued((500, 24), seed=1500, lo=-3, hi=3, device=DEV)
@@ -85,8 +106,9 @@ def test_q8_is_refused_where_it_does_not_apply_and_falls_back_where_it_cannot_se
     with pytest.raises(ralm.RalmError):
         idx.enable_q8()
     idx.close()
-    # k beyond the 8-bit scan's limit and batches of more than 8 queries take the fp16 scans
-    q = workloads.integer_valued((12, 32), seed=1502, lo=-3, hi=3, device=DEV)
-    for s, k in ((4, 300), (12, 5)):
+    # k beyond the 8-bit scan's limits (256 up to 8 queries, 64 up to 16) and batches of more than
+    # 16 queries take the fp16 scans
+    q = workloads.integer_valued((20, 32), seed=1502, lo=-3, hi=3, device=DEV)
+    for s, k in ((4, 300), (12, 65), (20, 5)):
         ids, scores, _ = _search(x, q[:s].contiguous(), k, q8=True)
         check_search(ids, scores, x.cpu().numpy(), q[:s].cpu().numpy(), oracle.IP, k, exact=True)
