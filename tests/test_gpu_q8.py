@@ -63,6 +63,32 @@ def test_q8_mixture_rows_match_the_oracle_and_the_fp16_scan(N, d, s, k):
     torch.testing.assert_close(scores, scores16, rtol=1e-5, atol=1e-6)
 
 
+@pytest.mark.parametrize("N,d", [(3000, 64), (2_450_000, 32)])
+def test_q8_bound_is_tight_where_the_rounding_error_is_parallel_to_the_query(N, d):
+    """The worst case of the Cauchy-Schwarz bound. One row is all 9s: E5M2 stores 8 (9 is the
+    midpoint of 8 and 10), so with an all-ones query its 8-bit score is 8 d while its true score
+    is 9 d, and the difference equals |q| |x - x8| exactly. Every other row is made of 8s and 10s,
+    which E5M2 holds exactly, with scores up to 9 d - 2: above the planted row's 8-bit score, below
+    its true one. A bound that is the least bit too small drops the planted row."""
+    g = torch.Generator(device=DEV).manual_seed(1700 + d)
+    tens = torch.rand((N, d), generator=g, device=DEV) < 0.3
+    x = torch.where(tens, 10.0, 8.0).to(torch.float16)
+    # cap every decoy at d/2 - 1 tens: score <= 8 d + 2 (d/2 - 1) = 9 d - 2
+    over = tens.sum(dim=1) > d // 2 - 1
+    x[over] = 8.0
+    planted = N - 7                                      # in the part the 8-bit launch covers
+    x[planted] = 9.0
+    x[5, : d // 2 - 1] = 10.0                            # the best decoy, in the sample part
+    x[5, d // 2 - 1:] = 8.0
+    q = torch.ones((3, d), dtype=torch.float16, device=DEV)
+    q[1] = 2.0
+    q[2, ::2] = 0.0                                      # half of the coordinates
+    for k in (1, 5):
+        ids, scores, _ = _search(x, q, k, q8=True)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+        assert ids[0, 0].item() == planted and scores[0, 0].item() == 9.0 * d
+
+
 def test_q8_large_values_saturate_without_losing_rows():
     """fp16 values beyond the largest finite E5M2 value (57344) are stored saturated; the bound
     covers the difference, so the row that holds them is still found."""
