@@ -57,6 +57,12 @@ def parse_args():
     ap.add_argument("--rows", type=int, default=None, help="override the corpus size (profiling)")
     ap.add_argument("--tune", default=None, help="consumer_warps,ring_depth,tile_rows (0 = default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flush-l2", action="store_true",
+                    help="write a buffer larger than L2 before every timed step (for corpora near L2 size); "
+                         "the step time is then the sum of per-step event intervals, flushes excluded")
+    ap.add_argument("--sharded", action="store_true",
+                    help="row-sharded search: every rank holds N / world rows, the answers are all-gathered "
+                         "and merged on every rank (strong scaling); without it ranks are replicas")
     return ap.parse_args()
 
 
@@ -82,6 +88,45 @@ def build_inputs(cfg, s, device, rows=None):
                                             workloads.seed_for(cfg.index, "caches"),
                                             n_centres=max(cfg.n_centres, 1))
     return corpus, queries[:s].contiguous(), src[:s], cache, cache_q
+
+
+def build_inputs_sharded(cfg, s, device, rank, world, dist, rows=None):
+    """This rank's rows of the corpus (the same bytes the whole corpus holds there), and the same
+    queries and speculation caches on every rank as the unsharded run builds. Rows that live on
+    another rank (query sources, cached rows) arrive by one all-reduce of zero-filled buffers."""
+    from paper_2401_14021_b200.sharded import shard_rows
+    N = rows or cfg.N
+    lo, hi = shard_rows(N, world, rank)
+    seed = workloads.seed_for(cfg.index)
+    if cfg.corpus == "unit_gaussian":
+        local, assign = workloads.unit_gaussian_corpus(N, cfg.d, seed, device=device, row_range=(lo, hi)), None
+    else:
+        local, assign = workloads.mixture_corpus(N, cfg.d, cfg.n_centres, seed, device=device,
+                                                 sigma_within=cfg.sigma_within, normalise=cfg.normalise,
+                                                 lognormal_sigma=cfg.lognormal_sigma, row_range=(lo, hi))
+
+    def fetch(ids):
+        out = torch.zeros((ids.numel(), cfg.d), dtype=torch.float16, device=device)
+        mine = (ids >= lo) & (ids < hi)
+        out[mine] = local[ids[mine] - lo]
+        if dist is not None:
+            bits = out.view(torch.int32)      # integer sums of one owner's bits and zeros: exact
+            dist.all_reduce(bits)
+        return out
+
+    R = max(cfg.requests, 1)
+    stride = cfg.stride or s
+    C = cfg.cache_entries or 64
+    nq = max(R * stride, s)
+    queries, src = workloads.noisy_copy_queries(local, nq, workloads.seed_for(cfg.index, "queries"),
+                                                n_rows=N, fetch=fetch)
+    cache_q = queries[:R * stride].reshape(R, stride, cfg.d).contiguous()
+    cache = workloads.speculation_cache_ids(assign, N, src[:R * stride].reshape(R, stride), C,
+                                            workloads.seed_for(cfg.index, "caches"),
+                                            n_centres=max(cfg.n_centres, 1))
+    # the cached vectors live with the requests (on every rank here): rows [R * C][d]
+    cache_rows = fetch(cache.flatten())
+    return local, lo, N, queries[:s].contiguous(), src[:s], cache, cache_q, cache_rows
 
 
 class ClockSampler:
@@ -247,10 +292,26 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    corpus, queries, src, cache, cache_q = build_inputs(cfg, s, device, args.rows)
-    N, d = corpus.shape
+    sharded = None
+    if args.sharded:
+        # row-sharded search: this rank holds rows [row_lo, row_lo + local rows) of the N-row corpus
+        from paper_2401_14021_b200.sharded import ShardedIndex
+        corpus, row_lo, N, queries, src, cache, cache_q, cache_rows = build_inputs_sharded(
+            cfg, s, device, rank, world, dist, args.rows)
+        d = corpus.shape[1]
+        sharded = ShardedIndex(corpus, row_lo, metric_id, max_s=max(s, 1), max_k=max(k, 1))
+        idx = sharded.index
+        # speculation runs over the cached vectors kept with the requests; its answers are positions
+        # in cache_rows, translated back to corpus ids through the cache's own id list
+        cache_index = ralm.Index(cache_rows, metric_id, max_s=8, max_k=1)
+        cache_flat = cache.flatten()
+        cache_local = torch.arange(cache_flat.numel(), dtype=torch.int64, device=device).reshape(cache.shape)
+    else:
+        corpus, queries, src, cache, cache_q = build_inputs(cfg, s, device, args.rows)
+        N, d = corpus.shape
+        idx = ralm.Index(corpus, metric_id, max_s=max(s, 1), max_k=max(k, 1))
+    local_rows = corpus.shape[0]
     R, stride = cache_q.shape[0], cache_q.shape[1]
-    idx = ralm.Index(corpus, metric_id, max_s=max(s, 1), max_k=max(k, 1))
     if args.variant:
         idx.set_variant(args.variant)
     if args.q8:
@@ -270,10 +331,23 @@ def main():
     spec_view = spec_ids[:nv, :vstride, 0] if vstride < stride else spec_ids[:nv].reshape(nv, stride)
     retr_view = ids[:nv * vstride].reshape(nv, vstride, k)
 
-    def step():
-        ralm.cache_search(idx, cache, cache_q, 1, spec_ids, spec_scores, stream)
-        ralm.search(idx, queries, k, ids, scores, stream)
-        ralm.verify(spec_view, retr_view, 1, first_mismatch, stream)
+    if sharded is None:
+        def step():
+            ralm.cache_search(idx, cache, cache_q, 1, spec_ids, spec_scores, stream)
+            ralm.search(idx, queries, k, ids, scores, stream)
+            ralm.verify(spec_view, retr_view, 1, first_mismatch, stream)
+    else:
+        spec_local = torch.empty((R, stride, 1), dtype=torch.int64, device=device)
+
+        def step():
+            ralm.cache_search(cache_index, cache_local, cache_q, 1, spec_local, spec_scores, stream)
+            torch.take(cache_flat, spec_local, out=spec_ids)
+            got_ids, got_scores = sharded.search(queries, k, stream)    # scan, all-gather, merge
+            ids.copy_(got_ids)
+            scores.copy_(got_scores)
+            ralm.verify(spec_view, retr_view, 1, first_mismatch, stream)
+
+    flush = torch.empty((512 << 20,), dtype=torch.uint8, device=device) if args.flush_l2 else None
 
     # ---- device-resident timing
     for _ in range(max(args.warmup, 3)):
@@ -286,16 +360,32 @@ def main():
     time.sleep(0.25)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    barrier()
-    total_ms = e0.elapsed_time(e1)
+    if flush is None:
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        barrier()
+        total_ms = e0.elapsed_time(e1)
+    else:
+        # L2 flushed before every step; the step time is the sum of the per-step intervals
+        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                 for _ in range(args.steps)]
+        for a, b in pairs:
+            flush.zero_()
+            a.record(stream)
+            step()
+            b.record(stream)
+        barrier()
+        total_ms = sum(a.elapsed_time(b) for a, b in pairs)
     clocks = sampler.stop()
-    scan_ms, scan_launches = idx.read_timing()
+    pass_ms = idx.read_timing_list(max(4096, 8 * args.steps))
+    scan_ms, scan_launches = sum(pass_ms), len(pass_ms)
+    dispatch = idx.last_dispatch()
     idx.set_timing(False)
     gpu_launches = idx.launch_count() - launches0 + args.steps   # + one verify launch per step
+    if sharded is not None:
+        gpu_launches += 3 * args.steps                           # cache score + rank on the cached vectors, merge_lists
     assert idx.device_status() == 0, "device status word set during the timed region"
     assert ids[:, 0].tolist() == src.tolist(), "rank-0 ids are not the planted sources"
 
@@ -313,16 +403,34 @@ def main():
     h2d = h_q.numel() * 2 + h_cache.numel() * 8 + h_cache_q.numel() * 2 + h_top1.numel() * 8
     d2h = h_ids.numel() * 8 + h_scores.numel() * 4 + h_spec.numel() * 8 + 4 * nv
 
-    def step_e2e():
-        d_cache.copy_(h_cache, non_blocking=True)
-        d_cache_q.copy_(h_cache_q, non_blocking=True)
-        ralm.cache_search(idx, d_cache, d_cache_q, 1, spec_ids, spec_scores, stream)
-        ralm.search_host(idx, h_q, k, h_ids, h_scores, stream)          # H2D, scan, D2H, sync
-        retr1.copy_(h_top1, non_blocking=True)
-        ralm.verify(spec_view, retr1, 1, first_mismatch, stream)
-        h_spec.copy_(spec_ids, non_blocking=True)
-        h_fm.copy_(first_mismatch, non_blocking=True)
-        stream.synchronize()
+    if sharded is None:
+        def step_e2e():
+            d_cache.copy_(h_cache, non_blocking=True)
+            d_cache_q.copy_(h_cache_q, non_blocking=True)
+            ralm.cache_search(idx, d_cache, d_cache_q, 1, spec_ids, spec_scores, stream)
+            ralm.search_host(idx, h_q, k, h_ids, h_scores, stream)          # H2D, scan, D2H, sync
+            retr1.copy_(h_top1, non_blocking=True)
+            ralm.verify(spec_view, retr1, 1, first_mismatch, stream)
+            h_spec.copy_(spec_ids, non_blocking=True)
+            h_fm.copy_(first_mismatch, non_blocking=True)
+            stream.synchronize()
+    else:
+        d_q = torch.empty_like(queries)
+        h2d = h_q.numel() * 2 + h_cache_q.numel() * 2
+
+        def step_e2e():
+            d_cache_q.copy_(h_cache_q, non_blocking=True)
+            d_q.copy_(h_q, non_blocking=True)
+            ralm.cache_search(cache_index, cache_local, d_cache_q, 1, spec_local, spec_scores, stream)
+            torch.take(cache_flat, spec_local, out=spec_ids)
+            got_ids, got_scores = sharded.search(d_q, k, stream)
+            ids.copy_(got_ids)
+            h_ids.copy_(got_ids, non_blocking=True)
+            h_scores.copy_(got_scores, non_blocking=True)
+            ralm.verify(spec_view, retr_view, 1, first_mismatch, stream)
+            h_spec.copy_(spec_ids, non_blocking=True)
+            h_fm.copy_(first_mismatch, non_blocking=True)
+            stream.synchronize()
 
     for _ in range(3):
         step_e2e()
@@ -336,66 +444,75 @@ def main():
 
     # ---- aggregate over ranks: time = max, work = sum
     from paper_2401_14021_b200 import replicas
-    (total_ms, e2e_ms), job_queries = replicas.aggregate([total_ms, e2e_ms], s * args.steps, device)
+    (total_ms, e2e_ms), job_queries = replicas.aggregate(
+        [total_ms, e2e_ms], s * args.steps if (sharded is None or rank == 0) else 0, device)
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         value = job_queries / (total_ms * 1e-3)
         e2e_value = job_queries / (e2e_ms * 1e-3)
-        corpus_bytes = N * d * 2
+        corpus_bytes = local_rows * d * 2            # what this GPU streams per pass
         passes = scan_launches / max(args.steps, 1)
         scan_avg_ms = scan_ms / max(scan_launches, 1)
-        achieved = corpus_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None
+        ordered = sorted(pass_ms)
+        scan_median_ms = ordered[len(ordered) // 2] if ordered else None
+        kernel = dispatch["kernel_name"]
+        sample = dispatch["sample_rows"]
+        # algorithmic bytes of one pass, from what the library says it ran: one read of the fp16
+        # rows; the tcgen05 scan reads its sample's rows twice (sample launch, then the scan proper);
+        # the 8-bit scan reads the sample in fp16 and the rest as one byte per element + one bound
+        if dispatch["kernel"] == 5:
+            pass_bytes = sample * d * 2 + (local_rows - sample) * (d + 4)
+        elif dispatch["kernel"] in (3, 4):
+            pass_bytes = (local_rows + sample) * d * 2
+        else:
+            pass_bytes = corpus_bytes
+        achieved = pass_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None
+        traffic = None
+        if dispatch["kernel"] == 2 and cfg.metric == "ip" and s <= 8 and not args.tune and \
+                TRAFFIC["sources_sha256_16"] == sources_hash(TRAFFIC["sources"]):
+            traffic = corpus_bytes * TRAFFIC["ratio"]
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"] if achieved else None,
-                    "peak_kind": peak_kind, "frac_of_nominal_8000": achieved / 8000.0 if achieved else None,
-                    "kernel": "scan_kernel", "bytes_per_launch": corpus_bytes,
-                    "traffic": (corpus_bytes * TRAFFIC_RATIO["scan_kernel<mma,ip>"]
-                                if cfg.metric == "ip" and args.variant in (0, 2) and not args.tune
-                                and s <= 8 else None),
-                    "traffic_note": "2M-row ncu capture scaled by rows; null if the kernel changed since"}
-        uses_q8 = args.q8 and cfg.metric == "ip" and args.variant == 0 and \
-            ((s <= 8 and k <= 256) or (s <= 16 and k <= 64)) and max(N // 128, 4 * 148 * 128) * 32 <= N
-        if uses_q8:
-            # the 8-bit scan streams the one-byte copy and one fp32 bound per row; the sample
-            # (1/128 of the rows, when the corpus is large enough for one) is scanned in fp16
-            sample = max(N // 128, 4 * 148 * 128)
-            q8_bytes = sample * d * 2 + (N - sample) * (d + 4)
-            achieved = q8_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None
-            roofline.update({"achieved": achieved, "frac": achieved / peaks["hbm_gbs"] if achieved else None,
-                             "frac_of_nominal_8000": achieved / 8000.0 if achieved else None,
-                             "kernel": "scan_q8_kernel", "bytes_per_launch": q8_bytes, "traffic": None,
-                             "fp16_equivalent_gbs": corpus_bytes / (scan_avg_ms * 1e-3) / 1e9
-                             if scan_launches else None})
-        uses_tc = k <= 64 and d >= 64 and (cfg.metric == "ip" or N >= 700_000) and \
-            (args.variant in (3, 4) or (args.variant == 0 and not uses_q8 and
-                                        s >= (33 if cfg.metric == "ip" else 17)))
-        if uses_tc:
-            roofline["kernel"] = "scan_tc_kernel"
-        if uses_tc and s > 255:
+                    "peak_kind": peak_kind + " (copy bandwidth: read + write; a pure-read stream may exceed it)",
+                    "frac_of_nominal_8000": achieved / 8000.0 if achieved else None,
+                    "kernel": kernel, "bytes_per_launch": pass_bytes, "traffic": traffic,
+                    "traffic_note": TRAFFIC["note"],
+                    "median_frac": (pass_bytes / (scan_median_ms * 1e-3) / 1e9 / peaks["hbm_gbs"])
+                    if scan_median_ms else None}
+        if dispatch["kernel"] == 5:
+            roofline["fp16_equivalent_gbs"] = corpus_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None
+        per_pass_queries = s / max(dispatch["passes"], 1)
+        if dispatch["kernel"] in (3, 4) and per_pass_queries > 255:
             # large batch: s flop per corpus byte is beyond the ridge, the tensor pipe bounds it.
             # fp16 runs at the bf16 rate; the kernel is timed inside a long step: sustained peak
-            flops = 2.0 * s * N * d / passes if passes else 0.0
+            flops = 2.0 * per_pass_queries * (local_rows + sample) * d
             tf = flops / (scan_avg_ms * 1e-3) / 1e12 if scan_launches else None
             peak_tf = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
             roofline = {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
                         "frac": tf / peak_tf if tf else None, "peak_kind": peak_kind + " (bf16 sustained)",
                         "frac_of_burst": tf / peaks["bf16_tflops"] if tf else None,
-                        "kernel": "scan_tc_kernel", "flops_per_launch": flops, "traffic": None,
+                        "kernel": kernel, "flops_per_launch": flops, "traffic": None,
+                        "useful_tflops": 2.0 * per_pass_queries * local_rows * d / (scan_avg_ms * 1e-3) / 1e12
+                        if scan_launches else None,
                         "hbm_gbs": achieved}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "higher_is_better": True, "scaling": "strong" if sharded is not None else "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": "%s %dx%d %s s=%d k=%d; cache lookup R=%d C=%d q=%d; verify stride %d"
                                    % (cfg.name, N, d, cfg.metric, s, k, R, cache.shape[1], stride, vstride),
                        "arithmetic": "fp16 corpus and queries, exact fp16 x fp16 products, fp32 accumulation",
-                       "variant": args.variant, "tune": args.tune, "replicas": world, "q8": bool(args.q8),
+                       "variant": args.variant, "tune": args.tune, "q8": bool(args.q8),
+                       "replicas": 1 if sharded is not None else world,
+                       "row_shards": world if sharded is not None else 1,
+                       "dispatch": dispatch, "l2_flushed_every_step": bool(args.flush_l2),
                        "l2": "inputs larger than L2 (%.1f GB corpus streamed every step)"
                              % (corpus_bytes / 1e9) if corpus_bytes > 2.5e8 else
                              "corpus near L2 size: L2-warm figure, not an HBM number"},
-            "scan_gbs": achieved, "scan_ms": scan_avg_ms, "scan_passes_per_step": passes,
+            "scan_gbs": corpus_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None,
+            "scan_ms": scan_avg_ms, "scan_median_ms": scan_median_ms, "scan_passes_per_step": passes,
             "roofline": roofline,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
@@ -408,14 +525,29 @@ def main():
             out["cpu_baseline"] = None
         print(json.dumps(out))
     idx.close()
+    if sharded is not None:
+        cache_index.close()
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
 
 
-# (dram__bytes_read.sum + dram__bytes_write.sum) / corpus bytes of one scan launch, from the
-# committed ncu capture of a 2 M-row case; traffic grows in proportion to the rows.
-TRAFFIC_RATIO = {"scan_kernel<mma,ip>": 1.0015}  # dram bytes / corpus bytes, profiles/scan_mma_ip_s8_k1_2Mx768.md
+def sources_hash(names):
+    """First 16 hex digits of the SHA-256 of the kernel sources a capture depends on."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in names:
+        with open(os.path.join(ROOT, "paper_2401_14021_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+# DRAM traffic of the headline kernel (warp-MMA scan, inner product, up to 8 queries):
+# (dram__bytes_read.sum + dram__bytes_write.sum) / corpus bytes of one scan launch, from an ncu
+# capture of a 2 M-row case (traffic grows in proportion to the rows). Reported only while the
+# sources the kernel is built from are the ones that were captured.
+TRAFFIC = {"ratio": 1.0015, "sources": ("scan.cuh", "common.cuh"), "sources_sha256_16": "unset",
+           "note": "2M-row ncu capture scaled by rows; null when the kernel's sources changed since"}
 
 if __name__ == "__main__":
     main()

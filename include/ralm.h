@@ -27,8 +27,10 @@
  *     product) or +inf (L2).
  *   - Scores are accumulated in fp32.
  *   - One index may be used from one stream at a time (its workspace is shared by calls).
- *   - Device-side anomalies (an out-of-range cache id, a wait that ran out) set a sticky
- *     status word that ralm_device_status reads.
+ *   - Device-side anomalies (an out-of-range cache id, a wait that ran out, a candidate list
+ *     asked to hold more than its capacity: RALM_ERR_INTERNAL, a defect of the library, the
+ *     results of that search are then not to be trusted) set a sticky status word that
+ *     ralm_device_status reads.
  */
 #ifndef RALM_H_
 #define RALM_H_
@@ -51,7 +53,8 @@ typedef enum {
     RALM_ERR_TIMEOUT = 4,
     RALM_ERR_UNSUPPORTED = 5,
     RALM_ERR_BAD_CACHE_ID = 6,
-    RALM_ERR_STATIC_LIMIT = 7
+    RALM_ERR_STATIC_LIMIT = 7,
+    RALM_ERR_INTERNAL = 8
 } ralm_status_t;
 
 /* Limits checked by the host side. */
@@ -117,14 +120,20 @@ ralm_status_t ralm_search_host(ralm_index_t *idx, const void *queries_host, int3
  * RALM_STATIC_MAX_BLOCKS * RALM_STATIC_MAX_S * RALM_STATIC_MAX_K * 8 bytes = 320 KiB (plus a
  * 256-byte status block), held by every GPU that loads the library until the process exits.
  *
- *   corpus, N, d, metric   as for ralm_index_create (DEVICE fp16 [N][d], borrowed for the call)
+ *   corpus, N, d, metric   as for ralm_index_create (DEVICE fp16 [N][d], borrowed for the call),
+ *                          except that two tiles of 16 rows must fit in shared memory next to
+ *                          the queries: d up to about 2800. (An index serves longer rows on its
+ *                          large-batch scan, whose workspace this call does not have.)
  *   queries                DEVICE fp16 [s][d], 16-byte aligned, 0 <= s <= RALM_STATIC_MAX_S
  *   ids, scores            DEVICE int64 [s][k] / fp32 [s][k] (written), 1 <= k <= RALM_STATIC_MAX_K
- *   device_status          DEVICE int32, may be NULL: zeroed by the call, then set to a
- *                          ralm_status_t value if a device-side wait ran out
+ *   device_status          DEVICE int32, may be NULL: zeroed by the call (also when s == 0), then
+ *                          set to a ralm_status_t value if a device-side wait ran out. With NULL
+ *                          the library keeps that word in its own scratch and nobody reads it:
+ *                          pass a status word if a time-out must be seen.
  * Results are identical to ralm_search's.
  * Errors: RALM_ERR_STATIC_LIMIT when s or k exceeds the limits above (nothing is launched);
- * INVALID_ARG, UNSUPPORTED, CUDA as elsewhere.
+ * UNSUPPORTED for rows longer than the limit above or a device that is not compute capability
+ * 10.x; INVALID_ARG, CUDA as elsewhere.
  *
  * The first call on each device looks up the scratch's device address and the device's
  * properties (with that device current); make that first call before any stream capture.
@@ -186,8 +195,8 @@ ralm_status_t ralm_cache_update(int64_t *cache_ids, int32_t *cursor, int32_t R, 
                                 const int32_t *steps, int32_t next_n, int64_t N, void *stream);
 
 /* Synchronise `stream`, read and clear the index's sticky device status word. Returns
- * RALM_OK, RALM_ERR_TIMEOUT, RALM_ERR_BAD_CACHE_ID, or RALM_ERR_CUDA if the stream itself
- * reports an error. */
+ * RALM_OK, RALM_ERR_TIMEOUT, RALM_ERR_BAD_CACHE_ID, RALM_ERR_INTERNAL, or RALM_ERR_CUDA if the
+ * stream itself reports an error. */
 ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
 
 /* Pin the scan variant used by ralm_search on this index (benchmarking aid).
@@ -235,6 +244,19 @@ ralm_status_t ralm_index_set_timing(ralm_index_t *idx, int32_t enabled);
 /* Wait for the scan launches timed since the last read, return the sum of their durations in
  * milliseconds and how many there were, and forget them. HOST pointers. */
 ralm_status_t ralm_index_read_timing(ralm_index_t *idx, double *total_ms, int64_t *launches);
+
+/* As ralm_index_read_timing, but the durations one by one, in the order of the passes:
+ * ms[0 .. *count) (HOST array of `capacity` doubles; passes beyond it are dropped). */
+ralm_status_t ralm_index_read_timing_list(ralm_index_t *idx, double *ms, int64_t capacity, int64_t *count);
+
+/* What the most recent ralm_search / ralm_search_host on this index ran (measurement aid; HOST
+ * pointers). kernel: 0 = no search yet, 1 = FMA scan, 2 = warp-MMA scan, 3 = tcgen05 scan with CTA
+ * pairs, 4 = tcgen05 scan with single CTAs, 5 = 8-bit scan. passes: passes over the corpus (each
+ * serves one slice of the batch). phases: 2 when every pass scans a sample first, else 1.
+ * sample_rows: rows of that sample (0 without one). For kernels 1, 2 and 5 the sample's rows are
+ * scanned once, by the sample launch; for 3 and 4 the main launch scans them again. */
+ralm_status_t ralm_index_last_dispatch(const ralm_index_t *idx, int32_t *kernel, int32_t *passes,
+                                       int32_t *phases, int64_t *sample_rows);
 
 /* ---- Optimal speculation stride scheduler (OS^3): host arithmetic, no device work ---------
  * Section 4 ("Optimal speculation stride scheduler") and Appendix A.2. `a` is the latency of one

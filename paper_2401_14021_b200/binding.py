@@ -9,7 +9,7 @@ L2 = 1
 
 STATUS_NAMES = {0: "RALM_OK", 1: "RALM_ERR_INVALID_ARG", 2: "RALM_ERR_OOM", 3: "RALM_ERR_CUDA",
                 4: "RALM_ERR_TIMEOUT", 5: "RALM_ERR_UNSUPPORTED", 6: "RALM_ERR_BAD_CACHE_ID",
-                7: "RALM_ERR_STATIC_LIMIT"}
+                7: "RALM_ERR_STATIC_LIMIT", 8: "RALM_ERR_INTERNAL"}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _lib = None
@@ -72,6 +72,11 @@ def load_library() -> ctypes.CDLL:
     lib.ralm_index_set_timing.argtypes = [p, i32]
     lib.ralm_index_read_timing.restype = i32
     lib.ralm_index_read_timing.argtypes = [p, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i64)]
+    lib.ralm_index_read_timing_list.restype = i32
+    lib.ralm_index_read_timing_list.argtypes = [p, ctypes.POINTER(ctypes.c_double), i64, ctypes.POINTER(i64)]
+    lib.ralm_index_last_dispatch.restype = i32
+    lib.ralm_index_last_dispatch.argtypes = [p, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                             ctypes.POINTER(i64)]
     f64 = ctypes.c_double
     lib.ralm_os3_expected_verified.restype = f64
     lib.ralm_os3_expected_verified.argtypes = [f64, i32]
@@ -159,6 +164,26 @@ class Index:
         _check(self._lib.ralm_index_read_timing(self._handle, ctypes.byref(ms), ctypes.byref(n)),
                "ralm_index_read_timing")
         return ms.value, n.value
+
+    def read_timing_list(self, capacity: int = 4096):
+        """Durations in ms of the scan passes timed since the last read, one by one."""
+        buf = (ctypes.c_double * max(capacity, 1))()
+        n = ctypes.c_int64()
+        _check(self._lib.ralm_index_read_timing_list(self._handle, buf, capacity, ctypes.byref(n)),
+               "ralm_index_read_timing_list")
+        return [buf[i] for i in range(n.value)]
+
+    KERNEL_NAMES = {0: None, 1: "scan_kernel<fma>", 2: "scan_kernel<mma>", 3: "scan_tc_kernel<pair>",
+                    4: "scan_tc_kernel<single>", 5: "scan_q8_kernel"}
+
+    def last_dispatch(self):
+        """ralm_index_last_dispatch as a dict: kernel (number), kernel_name, passes, phases, sample_rows."""
+        k, ps, ph = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+        rows = ctypes.c_int64()
+        _check(self._lib.ralm_index_last_dispatch(self._handle, ctypes.byref(k), ctypes.byref(ps), ctypes.byref(ph),
+                                                  ctypes.byref(rows)), "ralm_index_last_dispatch")
+        return {"kernel": k.value, "kernel_name": self.KERNEL_NAMES.get(k.value), "passes": ps.value,
+                "phases": ph.value, "sample_rows": rows.value}
 
     def device_status(self, stream=None) -> int:
         return self._lib.ralm_device_status(self._handle, _stream_ptr(stream))

@@ -22,6 +22,31 @@ __device__ __forceinline__ void write_result(uint64_t key, bool l2, int64_t *id_
 }
 
 // ------------------------------------------------------------------------------------
+// Threshold from the maxima of a sample launch: one CTA per query. vals holds G values for the
+// query (vals[g * stride + query], -inf = the group saw no row), each the best rank value of a
+// different, disjoint group of rows, so the k-th largest of them is reached by k different rows.
+// Writes it to thr_out[query], or -inf when fewer than k groups saw a row. G <= kMergeSortMax.
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kMergeThreads, 1)
+kth_of_maxima_kernel(const float *__restrict__ vals, int G, int stride, int k, float *__restrict__ thr_out) {
+    __shared__ uint64_t buf[kMergeSortMax];
+    const int q = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int P = next_pow2(G > 1 ? G : 2);
+    for (int i = tid; i < P; i += kMergeThreads) {
+        uint64_t key = 0;
+        if (i < G) {
+            const float v = vals[static_cast<size_t>(i) * stride + q];
+            if (v != -INFINITY) key = make_key(v, static_cast<uint32_t>(i));
+        }
+        buf[i] = key;
+    }
+    __syncthreads();
+    bitonic_sort_desc(buf, P, tid, kMergeThreads, -1);
+    if (tid == 0) thr_out[q] = (k <= G && buf[k - 1] != 0ull) ? key_value(buf[k - 1]) : -INFINITY;
+}
+
+// ------------------------------------------------------------------------------------
 // Merge: one CTA per query. `partial` holds B lists of k keys, each sorted descending and
 // padded with 0, laid out [B][s][k]. Writes ids [s][k] (int64) and scores [s][k] (fp32).
 // ------------------------------------------------------------------------------------
@@ -135,7 +160,7 @@ merge_lists_kernel(const int64_t *__restrict__ ids, const float *__restrict__ sc
 // Cache lookup, step 1: score. One warp per (request, cache slot); the warp scores its
 // cached corpus row against up to 8 of the request's queries at a time and stores one key
 // per query in keys[r][u][c] (Cp = C rounded up to a power of two; slots >= C hold 0).
-// grid = (ceil(Cp / slots_per_cta), R), block = 256.
+// grid = (R, ceil(Cp / slots_per_cta)), block = 256 (the request index in x: y stops at 65535).
 // ------------------------------------------------------------------------------------
 constexpr int kCacheThreads = 256;
 constexpr int kCacheSlotsPerCta = 32;
@@ -145,10 +170,10 @@ cache_score_kernel(const __half *__restrict__ corpus, long long N, int d, int l2
                    const int64_t *__restrict__ cache_ids, int C, int Cp,
                    const __half *__restrict__ queries, int q, uint64_t *__restrict__ keys,
                    int *status) {
-    const int r = blockIdx.y;
+    const int r = blockIdx.x;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int pieces = d >> 3;
-    for (int c = blockIdx.x * kCacheSlotsPerCta + warp; c < (blockIdx.x + 1) * kCacheSlotsPerCta && c < Cp;
+    for (int c = blockIdx.y * kCacheSlotsPerCta + warp; c < (blockIdx.y + 1) * kCacheSlotsPerCta && c < Cp;
          c += kCacheThreads / 32) {
         long long id = -1;
         if (c < C) id = cache_ids[static_cast<size_t>(r) * C + c];

@@ -10,6 +10,7 @@ namespace ralm {
 // Device status word values (match ralm_status_t).
 constexpr int kStatusTimeout = 4;
 constexpr int kStatusBadCacheId = 6;
+constexpr int kStatusInternal = 8;  // a candidate list was asked to hold more than its capacity
 
 // ---------------------------------------------------------------------------------
 // Ranking keys. Every candidate is one 64-bit key whose unsigned order IS the ranking:

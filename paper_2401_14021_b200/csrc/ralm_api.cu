@@ -39,6 +39,7 @@ struct ralm_index {
     float *x8_bound;       // per row: bound on |q.x - q.x8| per unit of |q| (see scan_q8.cuh)
     bool x8_force;         // use the copy also on corpora too small for a sample phase (testing aid)
     float *tc_thr;         // thresholds from the sample phase of a two-phase scan, [max_s]
+    float *tc_gmax;        // tcgen05 scan, sample launch: [num_sms * 4][max_s] maxima per selection warp
     bool tc_two_phase;     // sample phase enabled (tuning aid)
     int tc_clusters;       // CTA pairs the device runs at once (-1 = not asked yet)
     uint64_t *tc_cand;     // tcgen05 scan: [num_sms][tc_cand_q][kTcCap] candidate lists, or null
@@ -49,6 +50,9 @@ struct ralm_index {
     int64_t *h_ids;
     float *h_scores;
     int64_t launches;
+    // what the last search ran (ralm_index_last_dispatch)
+    int last_kernel, last_passes, last_phases;
+    int64_t last_sample_rows;
     // optional per-launch timing of the scan kernel (events on the caller's stream)
     bool timing;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timed;   // recorded, not yet read
@@ -103,6 +107,13 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
     if (k > 1) {
         // after the flag is raised every warp may still finish the tile it is on
         pl->cap = std::max(512, 2 * next_pow2(k));
+        // (a tuned tile height must leave that room: k kept keys plus one tile from every warp)
+        const int unit = mma ? 16 : (s_pass == 1 ? 16 : 4);
+        const int max_rows = (pl->cap - k) / (kMaxConsumerWarps + 1) / unit * unit;
+        if (pl->tile_rows > max_rows) {
+            pl->tile_rows = std::max(unit, max_rows);
+            pl->stage_bytes = align_up(pl->tile_rows * idx->d * 2, 128);
+        }
         // compact before the buffer is full, and already at about 4 k entries: a threshold only
         // rises when its list is compacted, and until then every push costs a shared atomic
         pl->soft_limit = std::min(pl->cap - (kMaxConsumerWarps + 1) * pl->tile_rows, std::max(4 * k, 64));
@@ -266,6 +277,11 @@ bool alloc_tc_workspace(ralm_index *idx, int queries) {
         idx->tc_thr = nullptr;
         return false;
     }
+    if (!idx->tc_gmax &&
+        device_alloc(&idx->tc_gmax, sizeof(float) * idx->num_sms * 4 * static_cast<size_t>(idx->max_s)) != cudaSuccess) {
+        idx->tc_gmax = nullptr;
+        return false;
+    }
     if (device_alloc(&idx->tc_cand, bytes) != cudaSuccess) {
         idx->tc_cand = nullptr;
         return false;
@@ -287,6 +303,7 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
     p.N = row_end;
     p.thr_init = thr_init;
     p.mode = mode;
+    p.gmax = idx->tc_gmax;
     p.d = idx->d;
     p.slack = static_cast<float>(idx->d) * (1.0f / 2097152.0f);  // as in the small-batch L2 scan
     p.norms = idx->norms;
@@ -307,22 +324,31 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
         p.nb = sp > kTcMaxN ? kTcMaxN : align_up(sp, pair ? 32 : 16);
         p.nhalves = (sp + p.nb - 1) / p.nb;
         const int nb_cta = pair ? p.nb / 2 : p.nb;
-        p.stage_bytes = kTcABytes + nb_cta * 128;
-        p.stages = std::min(kTcMaxStages, (idx->smem_optin - p.off_stage) / p.stage_bytes);
+        p.chunk_bytes = kTcABytes + nb_cta * 128;
+        // two K chunks per stage (half as many waits and commits per MMA) wherever the ring then
+        // still has three stages
+        const int room = idx->smem_optin - p.off_stage;
+        p.stage_chunks = (p.nchunks >= 2 && room / (2 * p.chunk_bytes) >= 3) ? 2 : 1;
+        p.stage_bytes = p.stage_chunks * p.chunk_bytes;
+        p.stages = std::min(kTcMaxStages, room / p.stage_bytes);
         if (p.stages < 2) return RALM_ERR_UNSUPPORTED;
         const int smem = p.off_stage + p.stages * p.stage_bytes;
         if (!encode_rows_map(&map_q, queries, sp, idx->d, nb_cta)) return RALM_ERR_CUDA;
+        void (*single)(CUtensorMap, CUtensorMap, TcParams) =
+            mode == 0 ? scan_tc_kernel<false, 0> : mode == 1 ? scan_tc_kernel<false, 1>
+            : mode == 2 ? scan_tc_kernel<false, 2> : scan_tc_kernel<false, 3>;
+        void (*paired)(CUtensorMap, CUtensorMap, TcParams) =
+            mode == 0 ? scan_tc_kernel<true, 0> : mode == 1 ? scan_tc_kernel<true, 1>
+            : mode == 2 ? scan_tc_kernel<true, 2> : scan_tc_kernel<true, 3>;
         if (!pair) {
             const int grid = static_cast<int>(std::min<long long>(idx->num_sms, p.ntiles));
-            if (cudaFuncSetAttribute(scan_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-                cudaSuccess)
+            if (cudaFuncSetAttribute(single, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
                 return RALM_ERR_CUDA;
-            scan_tc_kernel<false><<<grid, kTcThreads, smem, st>>>(map_x, map_q, p);
+            single<<<grid, kTcThreads, smem, st>>>(map_x, map_q, p);
             *grid_out = grid;
             return cudaGetLastError() == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
         }
-        if (cudaFuncSetAttribute(scan_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(paired, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return RALM_ERR_CUDA;
         cudaLaunchConfig_t cfg = {};
         cudaLaunchAttribute attr;
@@ -338,7 +364,7 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
         cfg.numAttrs = 1;
         if (idx->tc_clusters < 0) {
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, scan_tc_kernel<true>, &cfg) != cudaSuccess) {
+            if (cudaOccupancyMaxActiveClusters(&n, paired, &cfg) != cudaSuccess) {
                 cudaGetLastError();
                 n = 0;
             }
@@ -351,8 +377,7 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
         const int clusters = static_cast<int>(std::min<long long>(idx->tc_clusters, p.ntiles));
         cfg.gridDim = dim3(2 * clusters, 1, 1);
         *grid_out = 2 * clusters;
-        return cudaLaunchKernelEx(&cfg, scan_tc_kernel<true>, map_x, map_q, p) == cudaSuccess ? RALM_OK
-                                                                                              : RALM_ERR_CUDA;
+        return cudaLaunchKernelEx(&cfg, paired, map_x, map_q, p) == cudaSuccess ? RALM_OK : RALM_ERR_CUDA;
     }
 }
 
@@ -379,14 +404,17 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
                      (idx->variant == 0 &&
                       (s >= (l2 ? kTcAutoMinQueriesL2 : kTcAutoMinQueriesIp) || (!small_scan_fits && !l2))));
     if (tc) {
-        // Large corpora are scanned in two phases: a small sample first, whose merged top-k gives
-        // every query a score that k rows are known to reach; the rest then starts from those
-        // thresholds, so that hardly any score passes and the selection stays off the critical
-        // path. The sample's list rejoins the final merge (block index num_sms of `partial`).
+        // Large corpora are scanned in two phases: a small sample first, which gives every query a
+        // score that k rows are known to reach; the scan proper then starts from those thresholds,
+        // so that hardly any score passes and the selection stays off the critical path.
         const long long sample = tc_sample;
         const bool two_phase = tc_two_phase;
         int grid = 0;
         const int per_pass = std::min(kTcMaxQueries, idx->tc_cand_q);
+        idx->last_kernel = idx->variant == 4 ? 4 : 3;
+        idx->last_passes = (s + per_pass - 1) / per_pass;
+        idx->last_phases = two_phase ? 2 : 1;
+        idx->last_sample_rows = two_phase ? sample : 0;
         for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
             const int sp = std::min(per_pass, s - q0);
             const __half *qp = queries + static_cast<size_t>(q0) * idx->d;
@@ -395,19 +423,19 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             ralm_status_t rs = RALM_OK;
             if (two_phase) {
                 int grid1 = 0;
-                // L2: the sample is ranked by lower bounds of the tensor-core value and only yields
-                // thresholds; its rows are scanned again, exactly, by the main launch
-                rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, sample, nullptr, l2 ? 1 : 0,
+                // the sample launch keeps no lists: its selection warps write their best rank value
+                // per query (L2: best lower bound), and the k-th largest of a query's maxima is the
+                // threshold; the main launch then scans every row, the sample's too
+                rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, sample, nullptr, l2 ? 1 : 3,
                                     &grid1, st);
                 if (rs == RALM_OK) {
-                    merge_kernel<<<sp, kMergeThreads, 0, st>>>(
-                        idx->partial + static_cast<size_t>(q0) * k, grid1, s, k, 0, nullptr, nullptr,
-                        idx->partial + (static_cast<size_t>(idx->num_sms) * s + q0) * k, idx->tc_thr + q0);
+                    kth_of_maxima_kernel<<<sp, kMergeThreads, 0, st>>>(idx->tc_gmax + q0, grid1 * 4, s, k,
+                                                                       idx->tc_thr + q0);
                     if (cudaGetLastError() != cudaSuccess) rs = RALM_ERR_CUDA;
                 }
                 if (rs == RALM_OK)
-                    rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, l2 ? 0 : sample, idx->N,
-                                        idx->tc_thr, l2 ? 2 : 0, &grid, st);
+                    rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, idx->N, idx->tc_thr,
+                                        l2 ? 2 : 0, &grid, st);
                 idx->launches += 2;
             } else {
                 rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, idx->N, nullptr, 0, &grid, st);
@@ -416,8 +444,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             if (rs != RALM_OK) return rs;
             idx->launches++;
         }
-        merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, l2 ? 1 : 0, ids, scores, nullptr, nullptr,
-                                                  (two_phase && !l2) ? idx->num_sms : -1);
+        merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, l2 ? 1 : 0, ids, scores, nullptr, nullptr, -1);
         if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
         idx->launches++;
         return RALM_OK;
@@ -448,6 +475,10 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     // (two more launches: only worth it when the scan itself takes a millisecond or more)
     const bool two_phase = (k > 1 || use_q8) && idx->tc_thr && idx->tc_two_phase && sample * 32 <= idx->N;
     int grid = 0;
+    idx->last_kernel = use_q8 ? 5 : (mma ? 2 : 1);
+    idx->last_passes = (s + per_pass - 1) / per_pass;
+    idx->last_phases = two_phase ? 2 : 1;
+    idx->last_sample_rows = two_phase ? sample : 0;
     for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
         const int sp = std::min(per_pass, s - q0);
         ScanPlan pl;
@@ -669,6 +700,8 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->tune_warps = idx->tune_depth = idx->tune_rows = 0;
     idx->launches = 0;
     idx->timing = false;
+    idx->last_kernel = idx->last_passes = idx->last_phases = 0;
+    idx->last_sample_rows = 0;
     // one list per scan CTA and query, plus one more block for the list of a sample phase
     const size_t partial_bytes = sizeof(uint64_t) * (idx->num_sms + 1) * max_s * static_cast<size_t>(max_k);
     const size_t sk = static_cast<size_t>(max_s) * max_k;
@@ -676,6 +709,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->tc_cand_q = 0;
     idx->tc_clusters = -1;
     idx->tc_thr = nullptr;
+    idx->tc_gmax = nullptr;
     idx->tc_two_phase = true;
     idx->norms = nullptr;
     idx->x8 = nullptr;
@@ -740,6 +774,7 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
     cudaFree(idx->cache_keys);
     cudaFree(idx->tc_cand);
     cudaFree(idx->tc_thr);
+    cudaFree(idx->tc_gmax);
     cudaFree(idx->norms);
     cudaFree(idx->x8);
     cudaFree(idx->x8_bound);
@@ -796,7 +831,7 @@ ralm_status_t ralm_cache_search(ralm_index_t *idx, const int64_t *cache_ids, int
     const int Cp = next_pow2(C);
     if (static_cast<long long>(R) * q * Cp > RALM_MAX_CACHE_KEYS) return RALM_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const dim3 grid((Cp + kCacheSlotsPerCta - 1) / kCacheSlotsPerCta, R);
+    const dim3 grid(R, (Cp + kCacheSlotsPerCta - 1) / kCacheSlotsPerCta);
     cache_score_kernel<<<grid, kCacheThreads, 0, st>>>(idx->corpus, idx->N, idx->d,
                                                        idx->metric == RALM_L2, cache_ids, C, Cp,
                                                        static_cast<const __half *>(queries), q,
@@ -868,6 +903,7 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream) {
         return RALM_ERR_CUDA;
     if (word == kStatusTimeout) return RALM_ERR_TIMEOUT;
     if (word == kStatusBadCacheId) return RALM_ERR_BAD_CACHE_ID;
+    if (word == kStatusInternal) return RALM_ERR_INTERNAL;
     return word == 0 ? RALM_OK : RALM_ERR_CUDA;
 }
 
@@ -919,13 +955,16 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     if (metric != RALM_IP && metric != RALM_L2) return RALM_ERR_INVALID_ARG;
     if (s < 0 || k < 1) return RALM_ERR_INVALID_ARG;
     if (s > RALM_STATIC_MAX_S || k > RALM_STATIC_MAX_K) return RALM_ERR_STATIC_LIMIT;
-    if (s == 0) return RALM_OK;
-    if (!queries || !ids || !scores || !aligned16(queries)) return RALM_ERR_INVALID_ARG;
+    if (s > 0 && (!queries || !ids || !scores || !aligned16(queries))) return RALM_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (s == 0) {  // nothing to search; the caller's status word is still zeroed, as promised
+        if (device_status && cudaMemsetAsync(device_status, 0, sizeof(int), st) != cudaSuccess) return RALM_ERR_CUDA;
+        return RALM_OK;
+    }
     StaticDeviceState *dev = nullptr;
     ralm_status_t rs = static_state_for_current_device(&dev);
     if (rs != RALM_OK) return rs;
     if (dev->cc_major != 10) return RALM_ERR_UNSUPPORTED;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     int *status = device_status ? device_status : dev->status;
     // the scratch keeps whatever the previous call left; the partial lists are fully
     // rewritten by the scan, the status word is the one thing that must start at zero
@@ -949,6 +988,7 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.tc_cand_q = 0;
     view.tc_clusters = -1;
     view.tc_thr = nullptr;
+    view.tc_gmax = nullptr;
     view.tc_two_phase = false;
     view.spill = nullptr;
     view.spill_cap = 0;
@@ -961,6 +1001,8 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.h_ids = nullptr;
     view.h_scores = nullptr;
     view.launches = 0;
+    view.last_kernel = view.last_passes = view.last_phases = 0;
+    view.last_sample_rows = 0;
     view.timing = false;
     return search_device(&view, static_cast<const __half *>(queries), s, k, ids, scores, st);
 }
@@ -1006,6 +1048,33 @@ ralm_status_t ralm_index_read_timing(ralm_index_t *idx, double *total_ms, int64_
     return rs;
 }
 
+ralm_status_t ralm_index_read_timing_list(ralm_index_t *idx, double *ms, int64_t capacity, int64_t *count) {
+    if (!idx || !count || capacity < 0 || (capacity > 0 && !ms)) return RALM_ERR_INVALID_ARG;
+    int64_t n = 0;
+    ralm_status_t rs = RALM_OK;
+    for (auto &ev : idx->timed) {
+        float t = 0.f;
+        if (cudaEventSynchronize(ev.second) != cudaSuccess || cudaEventElapsedTime(&t, ev.first, ev.second) != cudaSuccess)
+            rs = RALM_ERR_CUDA;
+        else if (n < capacity)
+            ms[n++] = t;
+        idx->spare.push_back(ev);
+    }
+    idx->timed.clear();
+    *count = n;
+    return rs;
+}
+
+ralm_status_t ralm_index_last_dispatch(const ralm_index_t *idx, int32_t *kernel, int32_t *passes, int32_t *phases,
+                                       int64_t *sample_rows) {
+    if (!idx || !kernel || !passes || !phases || !sample_rows) return RALM_ERR_INVALID_ARG;
+    *kernel = idx->last_kernel;
+    *passes = idx->last_passes;
+    *phases = idx->last_phases;
+    *sample_rows = idx->last_sample_rows;
+    return RALM_OK;
+}
+
 const char *ralm_status_string(ralm_status_t status) {
     switch (status) {
         case RALM_OK: return "ok";
@@ -1015,6 +1084,7 @@ const char *ralm_status_string(ralm_status_t status) {
         case RALM_ERR_TIMEOUT: return "a device-side wait ran out";
         case RALM_ERR_UNSUPPORTED: return "unsupported device, shape or variant";
         case RALM_ERR_BAD_CACHE_ID: return "a cache id was outside [-1, N)";
+        case RALM_ERR_INTERNAL: return "a candidate list overflowed (library defect; results not valid)";
         case RALM_ERR_STATIC_LIMIT:
             return "s or k exceeds what the built-in scratch of ralm_search_static can hold";
     }

@@ -51,6 +51,7 @@ struct ScanParams {
     const float *norms;     // warp-MMA L2 with NRM: squared norm of every corpus row, fp32 [N]
                             // (8-bit scan: the per-row bound of its filter)
     const uint8_t *x8;      // 8-bit scan: the one-byte copy of the corpus, [N][d]
+    const float *sqnorms;   // 8-bit scan, L2: squared norm of every corpus row, fp32 [N]
     uint64_t *partial;      // [gridDim.x][s_total][k] sorted keys, 0 = empty
     uint64_t *spill;        // large k: candidate lists in global memory, [gridDim.x][8][cap]; the
                             // shared-memory candidate area then holds one sort scratch of cap keys
@@ -97,7 +98,7 @@ __device__ inline void compact_query(ScanHeader *hdr, uint64_t *cand, uint64_t *
                                      int k, int tid, int nthr, int bar_id) {
     uint64_t *list = cand + static_cast<size_t>(q) * cap;
     uint64_t *a = scratch ? scratch : list;
-    const int n = hdr->cnt[q];
+    const int n = hdr->cnt[q] < cap ? hdr->cnt[q] : cap;  // (cap: see push_candidate)
     const int P = next_pow2(n > 1 ? n : 2);
     if (scratch) {
         for (int i = tid; i < P; i += nthr) a[i] = (i < n) ? list[i] : 0ull;
@@ -197,10 +198,14 @@ __device__ __forceinline__ float2 h2_to_f2(uint32_t h2) {
     return __half22float2(*reinterpret_cast<const __half2 *>(&h2));
 }
 
+// The host sizes the lists so that slot < cap always holds (every warp pushes at most the rest of
+// its tile after the flag is up). Should that ever fail, the key is dropped and the status word
+// says so, rather than writing into the neighbouring list.
 __device__ __forceinline__ void push_candidate(ScanHeader *hdr, uint64_t *cand, int cap, int soft,
-                                               int q, uint64_t key) {
+                                               int q, uint64_t key, int *status) {
     const int slot = atomicAdd(&hdr->cnt[q], 1);
-    cand[static_cast<size_t>(q) * cap + slot] = key;
+    if (slot < cap) cand[static_cast<size_t>(q) * cap + slot] = key;
+    else atomicMax(status, kStatusInternal);
     if (slot >= soft) *reinterpret_cast<volatile int *>(&hdr->flag) = 1;
 }
 
@@ -548,7 +553,7 @@ scan_kernel(const ScanParams p) {
                                     if (TOP1) {
                                         atomicMax(&hdr->best[q], static_cast<unsigned long long>(key));
                                     } else if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q])) {
-                                        push_candidate(hdr, cand, p.cap, p.soft_limit, q, key);
+                                        push_candidate(hdr, cand, p.cap, p.soft_limit, q, key, p.status);
                                     }
                                 }
                             }
@@ -578,18 +583,18 @@ scan_kernel(const ScanParams p) {
                         if (r_lo < p.N) {
                             if (gq0 < p.s && acc[grp][0] >= th0)
                                 push_candidate(hdr, cand, p.cap, p.soft_limit, gq0,
-                                               make_key(acc[grp][0], static_cast<uint32_t>(r_lo)));
+                                               make_key(acc[grp][0], static_cast<uint32_t>(r_lo)), p.status);
                             if (gq1 < p.s && acc[grp][1] >= th1)
                                 push_candidate(hdr, cand, p.cap, p.soft_limit, gq1,
-                                               make_key(acc[grp][1], static_cast<uint32_t>(r_lo)));
+                                               make_key(acc[grp][1], static_cast<uint32_t>(r_lo)), p.status);
                         }
                         if (r_hi < p.N) {
                             if (gq0 < p.s && acc[grp][2] >= th0)
                                 push_candidate(hdr, cand, p.cap, p.soft_limit, gq0,
-                                               make_key(acc[grp][2], static_cast<uint32_t>(r_hi)));
+                                               make_key(acc[grp][2], static_cast<uint32_t>(r_hi)), p.status);
                             if (gq1 < p.s && acc[grp][3] >= th1)
                                 push_candidate(hdr, cand, p.cap, p.soft_limit, gq1,
-                                               make_key(acc[grp][3], static_cast<uint32_t>(r_hi)));
+                                               make_key(acc[grp][3], static_cast<uint32_t>(r_hi)), p.status);
                         }
                     }
                 }
@@ -650,7 +655,7 @@ scan_kernel(const ScanParams p) {
                             bestA[0] = key > bestA[0] ? key : bestA[0];
                         } else if (val >= hdr->thr[jq]) {
                             push_candidate(hdr, cand, p.cap, p.soft_limit, jq,
-                                           make_key(val, static_cast<uint32_t>(row)));
+                                           make_key(val, static_cast<uint32_t>(row)), p.status);
                         }
                     }
                 }

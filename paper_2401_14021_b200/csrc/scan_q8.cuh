@@ -20,6 +20,12 @@
 // from staged row q8_phys_row(m), which alternates between the two groups; the staged queries
 // get a pitch of 16 bytes modulo 128 for the same reason.
 //
+// L2 (squared distance) uses the same filter on x.q: with the rows' stored squared norms,
+//     -|x - q|^2 = 2 x.q - |x|^2 - |q|^2 <= 2 (q.x8 + |q| e_j) - |x|^2 - |q|^2
+// (plus the slack that bounds the rounding of the stored norms, as in the fp16 L2 scan), and a
+// pair that passes is scored again in the direct sum-of-squared-differences form from the fp16
+// row, which is the only value ranked and returned.
+//
 // Structure (producer warp, private stage rings per consumer warp, candidate buffers, compaction
 // meetings) is that of scan_kernel; the tile is 16 rows of d bytes. The host starts this kernel
 // from the thresholds of an fp16 scan of a small sample, without which nearly every pair would
@@ -118,15 +124,46 @@ __device__ __forceinline__ float warp_exact_ip(const __half *row, uint32_t q_add
     return v;
 }
 
+// Squared distance between one fp16 corpus row (global memory) and one staged query (stored in
+// the same (e0, e2, e1, e3) order), by the whole warp, in the direct form.
+__device__ __forceinline__ float warp_exact_l2(const __half *row, uint32_t q_addr, int d, int lane) {
+    float2 sum = make_float2(0.f, 0.f);
+    const uint4 *src = reinterpret_cast<const uint4 *>(row);
+    for (int piece = lane; piece * 8 < d; piece += 32) {
+        const uint4 xr = __ldg(src + piece);
+        const uint4 qr = lds128(q_addr + piece * 16);
+        const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
+        const uint32_t qw[4] = {qr.x, qr.y, qr.z, qr.w};
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const float2 x01 = h2_to_f2(xw[2 * e]), x23 = h2_to_f2(xw[2 * e + 1]);
+            const float2 q02 = h2_to_f2(qw[2 * e]), q13 = h2_to_f2(qw[2 * e + 1]);
+            const float d0 = x01.x - q02.x, d1 = x01.y - q13.x, d2 = x23.x - q02.y, d3 = x23.y - q13.y;
+            sum.x = fmaf(d0, d0, sum.x);
+            sum.y = fmaf(d1, d1, sum.y);
+            sum.x = fmaf(d2, d2, sum.x);
+            sum.y = fmaf(d3, d3, sum.y);
+        }
+    }
+    float v = sum.x + sum.y;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
 // p.x8: the 8-bit copy; p.norms: the per-row bound e_j; p.corpus: the fp16 rows (rescoring).
+// L2: squared distance (p.sqnorms: the rows' squared norms; p.l2_slack as in the fp16 L2 scan).
+// p.spill: candidate lists in global memory with one sort scratch in shared memory (large k).
 // NG groups of 8 queries per pass share every staged tile (NG = 1 or 2); p.tile_rows == 16;
 // d % 16 == 0.
-template <bool TOP1, int NG>
+template <bool TOP1, int NG, bool L2 = false>
 __global__ void __launch_bounds__(kScanThreads, 1)
 scan_q8_kernel(const ScanParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     ScanHeader *hdr = reinterpret_cast<ScanHeader *>(smem);
-    uint64_t *cand = reinterpret_cast<uint64_t *>(smem + p.off_cand);
+    uint64_t *scratch = p.spill ? reinterpret_cast<uint64_t *>(smem + p.off_cand) : nullptr;
+    uint64_t *cand = p.spill ? p.spill + static_cast<size_t>(blockIdx.x) * kScanMaxPassQueries * p.cap
+                             : reinterpret_cast<uint64_t *>(smem + p.off_cand);
     const int W = p.nwarps;
     const int S = W * p.depth;
     constexpr int T = 16;
@@ -187,8 +224,8 @@ scan_q8_kernel(const ScanParams p) {
         long long row0 = p.row_begin + (static_cast<long long>(blockIdx.x) + static_cast<long long>(w) * gridDim.x) * T;
         const long long row_step = static_cast<long long>(gridDim.x) * W * T;
 
-        // |q| of this lane's two queries (2t, 2t + 1), rounded up
-        float qn0[NG], qn1[NG];
+        // |q| of this lane's two queries (2t, 2t + 1), rounded up (and |q|^2 for L2)
+        float qn0[NG], qn1[NG], qs0[NG], qs1[NG];
 #pragma unroll
         for (int grp = 0; grp < NG; ++grp) {
             const int row_a = grp * kScanMaxQueries + 2 * t;
@@ -203,6 +240,8 @@ scan_q8_kernel(const ScanParams p) {
             const float up = 1.0f + 1.0f / 1024.0f;
             qn0[grp] = __fmul_ru(__fsqrt_ru(a2), up);
             qn1[grp] = __fmul_ru(__fsqrt_ru(b2), up);
+            qs0[grp] = a2;
+            qs1[grp] = b2;
         }
 
         int slot = 0;
@@ -231,18 +270,22 @@ scan_q8_kernel(const ScanParams p) {
         // The rows' bounds are fetched one tile ahead: the tile itself is usually resident by the
         // time its turn comes, and a load issued only then would stall the warp for a DRAM latency.
         const int ph_lo = q8_phys_row(g), ph_hi = q8_phys_row(g + 8);
-        float e_lo_next = 0.f, e_hi_next = 0.f;
+        float e_lo_next = 0.f, e_hi_next = 0.f, n_lo_next = 0.f, n_hi_next = 0.f;
         if (w < my_tiles) {
             if (row0 + ph_lo < p.N) e_lo_next = __ldg(p.norms + row0 + ph_lo);
             if (row0 + ph_hi < p.N) e_hi_next = __ldg(p.norms + row0 + ph_hi);
+            if (L2 && row0 + ph_lo < p.N) n_lo_next = __ldg(p.sqnorms + row0 + ph_lo);
+            if (L2 && row0 + ph_hi < p.N) n_hi_next = __ldg(p.sqnorms + row0 + ph_hi);
         }
         for (long long it = w; it < my_tiles; it += W, row0 += row_step) {
-            const float e_lo = e_lo_next, e_hi = e_hi_next;
-            e_lo_next = e_hi_next = 0.f;
+            const float e_lo = e_lo_next, e_hi = e_hi_next, n_lo = n_lo_next, n_hi = n_hi_next;
+            e_lo_next = e_hi_next = n_lo_next = n_hi_next = 0.f;
             if (it + W < my_tiles) {
                 const long long nrow = row0 + row_step;
                 if (nrow + ph_lo < p.N) e_lo_next = __ldg(p.norms + nrow + ph_lo);
                 if (nrow + ph_hi < p.N) e_hi_next = __ldg(p.norms + nrow + ph_hi);
+                if (L2 && nrow + ph_lo < p.N) n_lo_next = __ldg(p.sqnorms + nrow + ph_lo);
+                if (L2 && nrow + ph_hi < p.N) n_hi_next = __ldg(p.sqnorms + nrow + ph_hi);
             }
             if (*abort_flag) continue;
             const int st = w + slot * W;
@@ -269,7 +312,7 @@ scan_q8_kernel(const ScanParams p) {
                         while (!mbar_try_wait(full_bar, my_parity)) {}  // completed: returns at once
                         have_tile = true;
                     } else if (state == 2) {
-                        compaction_meeting(hdr, cand, nullptr, p.cap, p.s, p.k, w, lane, W);
+                        compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W);
                     } else if (state == 3) {
                         if (lane == 0) {
                             atomicMax(p.status, kStatusTimeout);
@@ -382,11 +425,25 @@ scan_q8_kernel(const ScanParams p) {
                     if (k0) th0 = fmaxf(th0, key_value(k0));
                     if (k1) th1 = fmaxf(th1, key_value(k1));
                 }
+                // upper bounds of the rank value: the score itself, or for L2 of -distance^2
+                float u[4];
+                u[0] = __fmaf_ru(qn0[grp], e_lo, acc[grp][0]);
+                u[1] = __fmaf_ru(qn1[grp], e_lo, acc[grp][1]);
+                u[2] = __fmaf_ru(qn0[grp], e_hi, acc[grp][2]);
+                u[3] = __fmaf_ru(qn1[grp], e_hi, acc[grp][3]);
+                if (L2) {
+                    const float sl = p.l2_slack;
+                    const float s00 = n_lo + qs0[grp], s01 = n_lo + qs1[grp], s10 = n_hi + qs0[grp], s11 = n_hi + qs1[grp];
+                    u[0] = __fmaf_ru(2.0f, u[0], __fmaf_ru(sl, s00, 0.0f - s00));
+                    u[1] = __fmaf_ru(2.0f, u[1], __fmaf_ru(sl, s01, 0.0f - s01));
+                    u[2] = __fmaf_ru(2.0f, u[2], __fmaf_ru(sl, s10, 0.0f - s10));
+                    u[3] = __fmaf_ru(2.0f, u[3], __fmaf_ru(sl, s11, 0.0f - s11));
+                }
                 bool pass[4];
-                pass[0] = r_lo < p.N && q0 < p.s && __fmaf_ru(qn0[grp], e_lo, acc[grp][0]) >= th0;
-                pass[1] = r_lo < p.N && q1 < p.s && __fmaf_ru(qn1[grp], e_lo, acc[grp][1]) >= th1;
-                pass[2] = r_hi < p.N && q0 < p.s && __fmaf_ru(qn0[grp], e_hi, acc[grp][2]) >= th0;
-                pass[3] = r_hi < p.N && q1 < p.s && __fmaf_ru(qn1[grp], e_hi, acc[grp][3]) >= th1;
+                pass[0] = r_lo < p.N && q0 < p.s && u[0] >= th0;
+                pass[1] = r_lo < p.N && q1 < p.s && u[1] >= th1;
+                pass[2] = r_hi < p.N && q0 < p.s && u[2] >= th0;
+                pass[3] = r_hi < p.N && q1 < p.s && u[3] >= th1;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     unsigned m = __ballot_sync(0xffffffffu, pass[i]);
@@ -396,14 +453,15 @@ scan_q8_kernel(const ScanParams p) {
                         const int row_local = q8_phys_row((src >> 2) + ((i & 2) ? 8 : 0));
                         const int q = grp * kScanMaxQueries + 2 * (src & 3) + (i & 1);
                         const long long row = row0 + row_local;
-                        const float val = warp_exact_ip(p.corpus + row * d, q_base_addr + q * q_pitch, d, lane);
+                        const float val = L2 ? 0.0f - warp_exact_l2(p.corpus + row * d, q_base_addr + q * q_pitch, d, lane)
+                                             : warp_exact_ip(p.corpus + row * d, q_base_addr + q * q_pitch, d, lane);
                         if (lane == 0) {
                             const uint64_t key = make_key(val, static_cast<uint32_t>(row));
                             if (TOP1) {
                                 if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q]))
                                     atomicMax(&hdr->best[q], static_cast<unsigned long long>(key));
                             } else if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q])) {
-                                push_candidate(hdr, cand, p.cap, p.soft_limit, q, key);
+                                push_candidate(hdr, cand, p.cap, p.soft_limit, q, key, p.status);
                             }
                         }
                     }
@@ -439,11 +497,11 @@ scan_q8_kernel(const ScanParams p) {
                     }
                 }
                 state = __shfl_sync(0xffffffffu, state, 0);
-                if (state == 1) compaction_meeting(hdr, cand, nullptr, p.cap, p.s, p.k, w, lane, W);
+                if (state == 1) compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W);
                 else if (state == 2) break;
             }
             named_barrier(1, cthreads);
-            compact_all(hdr, cand, nullptr, p.cap, p.s, p.k, 0, w, lane, W);
+            compact_all(hdr, cand, scratch, p.cap, p.s, p.k, 0, w, lane, W);
             named_barrier(1, cthreads);
             for (int q = 0; q < p.s; ++q) {
                 const int n = hdr->cnt[q];

@@ -5,13 +5,22 @@
 // per-CTA top-k selection so that the N x s score matrix never exists in memory.
 //
 // One persistent CTA per SM, 6 warps:
-//   warp 0      producer: one thread issues the TMA tile loads. A stage holds one K chunk
-//               (64 fp16 = 128 bytes per row, the 128-byte swizzle span) of 128 corpus rows
-//               and of up to 256 queries; stages form a ring guarded by full/empty mbarriers.
-//   warp 1      MMA: one thread issues tcgen05.mma (M = 128, N = 16..256, K = 16 per
-//               instruction, 4 per chunk). A work unit is (row tile, half of the queries);
-//               the two halves of TMEM (256 columns each) alternate between units, so one
-//               accumulator is drained while the next is being filled.
+//   warp 0      producer: issues the TMA tile loads. A K chunk is 64 fp16 = 128 bytes per row
+//               (the 128-byte swizzle span) of 128 corpus rows and of up to 256 queries; a
+//               stage holds up to two chunks; stages form a ring guarded by full/empty
+//               mbarriers.
+//   warp 1      MMA: issues tcgen05.mma (M = 128, N = 16..256, K = 16 per instruction, 4 per
+//               chunk) and one tcgen05.commit per stage. A work unit is (row tile, half of
+//               the queries); the two halves of TMEM (256 columns each) alternate between
+//               units, so one accumulator is drained while the next is being filled.
+//               Both warps run their loops with all 32 lanes converged and only the
+//               instruction that starts the asynchronous work sits under an elected lane:
+//               the waits, loop counters, addresses and descriptors then stay warp-uniform.
+//               (Run by a single lane inside a divergent branch, the same loop took ~190
+//               cycles per MMA and ~240 per wait + commit, whatever N was, and bounded the
+//               kernel: 4 MMAs per commit cost 857 cycles against 572 converged; with 8 per
+//               commit the converged loop is hidden behind the tensor pipe, 128 cycles per
+//               M = 256, N = 256, K = 16 instruction.)
 //   warps 2..5  selection: each warp owns one quarter of the TMEM lanes (32 corpus rows),
 //               reads the scores with tcgen05.ld, compares each with its query's threshold
 //               (the CTA's current k-th best, or a better bound handed in by the caller) and
@@ -70,17 +79,25 @@ struct TcParams {
                         // a CTA stages nb query rows per chunk, nb / 2 in a pair
     int nhalves;        // ceil(s / nb): 1 or 2
     int stages;
-    int stage_bytes;    // kTcABytes + (staged query rows) * 128, a multiple of 1024
+    int stage_chunks;   // K chunks per stage: 2, or 1 where the ring would otherwise be too short
+    int chunk_bytes;    // kTcABytes + (staged query rows) * 128, a multiple of 1024
+    int stage_bytes;    // stage_chunks * chunk_bytes
     int off_stage;      // shared-memory offset of the stage ring (1024-byte aligned)
     int cand_q;         // queries the candidate workspace was sized for (>= s)
-    // L2 (squared distance) on the same inner-product tiles. mode 0: inner product. The tensor-
-    // core value v = 2 x.q - |x|^2 - |q|^2 = -distance^2 cancels, so it is never ranked:
-    // mode 1 (sample launch): keys are the LOWER BOUNDS v - slack (|x|^2 + |q|^2); their merged
-    //         k-th value is a rank value that k rows are known to reach;
-    // mode 2 (main launch, over all rows): a pair passes the filter when v + slack (|x|^2 + |q|^2)
-    //         reaches the threshold, and is then scored again in the direct sum-of-squared-
-    //         differences form from global memory; only that value is ranked and returned.
+    // mode 0: inner product, scores ranked as they are.
+    // L2 (squared distance) runs on the same inner-product tiles: the tensor-core value
+    // v = 2 x.q - |x|^2 - |q|^2 = -distance^2 cancels, so it is never ranked;
+    // mode 2 (L2 main launch): a pair passes the filter when v + slack (|x|^2 + |q|^2) reaches the
+    //         threshold, and is then scored again in the direct sum-of-squared-differences form
+    //         from global memory; only that value is ranked and returned.
+    // Sample launches (mode 3 inner product, mode 1 L2) keep no lists at all: every selection
+    // warp keeps, per query, the best rank value among the rows it has seen (L2: the best LOWER
+    // BOUND v - slack (|x|^2 + |q|^2)) and writes these maxima to gmax. The warps' rows are
+    // disjoint, so the k-th largest of a query's maxima is a rank value that k different rows are
+    // known to reach: the threshold the main launch starts from. The main launch then scans all
+    // rows, the sample's too.
     int mode;
+    float *gmax;        // sample launches: [gridDim.x * 4][s_total] maxima, -inf where a warp saw no row
     int d;
     float slack;
     const float *norms;      // |x|^2 of every corpus row (fp32)
@@ -115,6 +132,28 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
         "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
         : "memory");
+}
+// One lane of a converged warp (the same one every time it is asked).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+// Bounded wait that also gives up when another warp of the CTA has started winding down. The
+// first probe is inline: the common case, a phase that completed long ago, costs one instruction.
+__device__ __forceinline__ bool tc_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag || clock64() - t0 > kWaitCycleLimit) return false;
+    }
 }
 __device__ __forceinline__ void tc_fence_before() {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -231,58 +270,59 @@ __device__ __forceinline__ void tc_compact_sorted(uint64_t *list, float *thr, in
 
 __device__ __forceinline__ void tc_compact_query(uint64_t *list, float *thr, int *cnt, int *sorted, int q,
                                                  int k, int lane) {
-    const int n = cnt[q];
+    const int n = cnt[q] < kTcCap ? cnt[q] : kTcCap;  // (the cap: see tc_append_octet)
     if (n <= 32) tc_compact_sorted<1>(list, thr, cnt, sorted, q, n, k, lane);
     else if (n <= 64) tc_compact_sorted<2>(list, thr, cnt, sorted, q, n, k, lane);
     else if (n <= 128) tc_compact_sorted<4>(list, thr, cnt, sorted, q, n, k, lane);
     else tc_compact_sorted<8>(list, thr, cnt, sorted, q, n, k, lane);
 }
 
-// The rare part of the selection: some score of this warp's 32 rows x 32 columns passes its
-// threshold. Out of line, and re-reading the scores from TMEM, so that the common path (no score
-// passes) stays a short loop with few live registers. The warp appends as a whole: lane L
-// learns which rows pass column L (one ballot per column that has any), reserves that many
-// slots of query L's list with ONE atomic instruction (32 different lists), and every passing
-// row then stores its key at its rank within the reservation.
-__device__ __noinline__ void tc_append_chunk(uint32_t taddr, const float *thr_chunk, int *cnt_chunk,
-                                             uint64_t *cand_chunk, uint32_t row, bool row_ok,
-                                             volatile int *dirty, int lane) {
-    uint32_t v[32];
-    tmem_ld32(taddr, v);
-    const float4 *t4 = reinterpret_cast<const float4 *>(thr_chunk);
-    uint32_t hit = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const float4 th = t4[i];
-        hit |= (__uint_as_float(v[4 * i + 0]) >= th.x ? 1u : 0u) << (4 * i + 0);
-        hit |= (__uint_as_float(v[4 * i + 1]) >= th.y ? 1u : 0u) << (4 * i + 1);
-        hit |= (__uint_as_float(v[4 * i + 2]) >= th.z ? 1u : 0u) << (4 * i + 2);
-        hit |= (__uint_as_float(v[4 * i + 3]) >= th.w ? 1u : 0u) << (4 * i + 3);
-    }
-    if (!row_ok) hit = 0;
+// Appending itself: every row (lane) whose bit b of `hit` is set stores key(v[b], row) in column
+// b's list. Only columns with a hit anywhere in the warp are visited (a warp-uniform branch per
+// column); each hit reserves its slot with its own shared-memory atomic.
+__device__ __forceinline__ void tc_store_hits(const uint32_t (&v)[32], uint32_t hit, int *cnt_chunk,
+                                              uint64_t *cand_chunk, uint32_t row, volatile int *dirty, int *status) {
     const uint32_t any_col = __reduce_or_sync(0xffffffffu, hit);
-    uint32_t mine = 0;
 #pragma unroll
     for (int b = 0; b < 32; ++b) {
         if (any_col & (1u << b)) {
-            const uint32_t m = __ballot_sync(0xffffffffu, (hit >> b) & 1u);
-            if (lane == b) mine = m;
+            if ((hit >> b) & 1u) {
+                const int slot = atomicAdd(&cnt_chunk[b], 1);
+                if (slot + 1 >= kTcSoft) *dirty = 1;
+                // (a list holds fewer than kTcSoft keys when a unit starts and gains at most 128 in
+                // one, so slot < kTcCap; should that ever fail the key is dropped and the status
+                // word says so, rather than writing into the neighbouring list)
+                if (slot < kTcCap) cand_chunk[static_cast<size_t>(b) * kTcCap + slot] = make_key(__uint_as_float(v[b]), row);
+                else atomicMax(status, kStatusInternal);
+            }
         }
     }
-    int base = 0;
-    if (mine) {
-        base = atomicAdd(&cnt_chunk[lane], __popc(mine));
-        if (base + __popc(mine) >= kTcSoft) *dirty = 1;
-    }
-    const uint32_t below = (1u << lane) - 1u;
+}
+
+// The rare part of the selection: some score among this warp's 32 rows x 8 columns (columns
+// c0 .. c0 + 7 of a block of 32) passes its threshold. Out of line, so that the common path (no
+// score passes) stays a short loop. thr_lane: the threshold of column `lane` of the block
+// (thresholds travel by shuffle, not through shared memory, whose loads are slow while TMA and the
+// tensor core keep it busy). Every row whose score passes stores key(score, row) in that
+// column's list, reserving its slot with its own shared-memory atomic.
+__device__ __noinline__ void tc_append_octet(uint32_t v0, uint32_t v1, uint32_t v2, uint32_t v3, uint32_t v4,
+                                             uint32_t v5, uint32_t v6, uint32_t v7, int c0, float thr_lane,
+                                             int *cnt_block, uint64_t *cand_block, uint32_t row, bool row_ok,
+                                             volatile int *dirty, int *status) {
+    const uint32_t v[8] = {v0, v1, v2, v3, v4, v5, v6, v7};
 #pragma unroll
-    for (int b = 0; b < 32; ++b) {
-        if (any_col & (1u << b)) {
-            const int base_b = __shfl_sync(0xffffffffu, base, b);
-            const uint32_t rows_b = __shfl_sync(0xffffffffu, mine, b);
-            if ((hit >> b) & 1u)
-                cand_chunk[static_cast<size_t>(b) * kTcCap + base_b + __popc(rows_b & below)] =
-                    make_key(__uint_as_float(v[b]), row);
+    for (int i = 0; i < 8; ++i) {
+        const float t = __shfl_sync(0xffffffffu, thr_lane, c0 + i);
+        if (row_ok && __uint_as_float(v[i]) >= t) {
+            const int slot = atomicAdd(&cnt_block[c0 + i], 1);
+            if (slot + 1 >= kTcSoft) *dirty = 1;
+            // (a list holds fewer than kTcSoft keys when a unit starts and gains at most 128 in
+            // one, so slot < kTcCap; should that ever fail the key is dropped and the status
+            // word says so, rather than writing into the neighbouring list)
+            if (slot < kTcCap)
+                cand_block[static_cast<size_t>(c0 + i) * kTcCap + slot] = make_key(__uint_as_float(v[i]), row);
+            else
+                atomicMax(status, kStatusInternal);
         }
     }
 }
@@ -312,14 +352,13 @@ __device__ __forceinline__ float tc_direct_l2(const __half *row, const __half *q
     return v;
 }
 
-// The rare part of the selection for L2 (see tc_append_chunk for the appending itself).
-// bound_sign = -1: sample launch, the value kept is the lower bound; +1: main launch, pairs that
-// pass the filter are scored again in the direct form and kept only if that value passes.
+// The rare part of the selection for L2 (main launch): pairs whose upper bound of -distance^2
+// reaches the threshold are scored again in the direct form and kept only if that value passes.
 __device__ __noinline__ void tc_append_chunk_l2(uint32_t taddr, const float *thr_chunk, const float *qn_chunk,
                                                 int *cnt_chunk, uint64_t *cand_chunk, uint32_t row, bool row_ok,
-                                                float nx, float slack, float bound_sign, const __half *corpus,
+                                                float nx, float slack, const __half *corpus,
                                                 const __half *queries_chunk, int d, volatile int *dirty,
-                                                int lane) {
+                                                int *status, int lane) {
     uint32_t v[32];
     tmem_ld32(taddr, v);
     uint32_t hit = 0;
@@ -327,57 +366,54 @@ __device__ __noinline__ void tc_append_chunk_l2(uint32_t taddr, const float *thr
     for (int b = 0; b < 32; ++b) {
         const float s2 = nx + qn_chunk[b];
         const float val = fmaf(2.0f, __uint_as_float(v[b]), 0.0f - s2);
-        const float bound = fmaf(bound_sign * slack, s2, val);
-        hit |= (bound >= thr_chunk[b] ? 1u : 0u) << b;
-        v[b] = __float_as_uint(bound);      // what the sample launch ranks
+        hit |= (fmaf(slack, s2, val) >= thr_chunk[b] ? 1u : 0u) << b;
     }
     if (!row_ok) hit = 0;
-    uint32_t any_col = __reduce_or_sync(0xffffffffu, hit);
-    if (bound_sign > 0.0f) {
+    const uint32_t any_col = __reduce_or_sync(0xffffffffu, hit);
 #pragma unroll
-        for (int b = 0; b < 32; ++b) {
-            if (any_col & (1u << b)) {
-                unsigned m = __ballot_sync(0xffffffffu, (hit >> b) & 1u);
-                while (m) {
-                    const int src = __ffs(m) - 1;
-                    m &= m - 1;
-                    const uint32_t row_src = __shfl_sync(0xffffffffu, row, src);
-                    const float dist = tc_direct_l2(corpus + static_cast<size_t>(row_src) * d,
-                                                    queries_chunk + static_cast<size_t>(b) * d, d, lane);
-                    if (lane == src) {
-                        const float exact = 0.0f - dist;
-                        v[b] = __float_as_uint(exact);
-                        if (!(exact >= thr_chunk[b])) hit &= ~(1u << b);
-                    }
+    for (int b = 0; b < 32; ++b) {
+        if (any_col & (1u << b)) {
+            unsigned m = __ballot_sync(0xffffffffu, (hit >> b) & 1u);
+            while (m) {
+                const int src = __ffs(m) - 1;
+                m &= m - 1;
+                const uint32_t row_src = __shfl_sync(0xffffffffu, row, src);
+                const float dist = tc_direct_l2(corpus + static_cast<size_t>(row_src) * d,
+                                                queries_chunk + static_cast<size_t>(b) * d, d, lane);
+                if (lane == src) {
+                    const float exact = 0.0f - dist;
+                    v[b] = __float_as_uint(exact);
+                    if (!(exact >= thr_chunk[b])) hit &= ~(1u << b);
                 }
             }
         }
-        any_col = __reduce_or_sync(0xffffffffu, hit);
     }
-    uint32_t mine = 0;
+    tc_store_hits(v, hit, cnt_chunk, cand_chunk, row, dirty, status);
+}
+
+// One block of 32 queries of a sample launch: for every column the best rank value among this
+// warp's 32 rows (as order-preserving bits, 0 = no row), folded into lane c's running maximum
+// for column c.
+__device__ __forceinline__ void tc_fold_block_maxima(const uint32_t (&v)[32], bool row_ok, uint32_t &best, int lane) {
 #pragma unroll
-    for (int b = 0; b < 32; ++b) {
-        if (any_col & (1u << b)) {
-            const uint32_t m = __ballot_sync(0xffffffffu, (hit >> b) & 1u);
-            if (lane == b) mine = m;
-        }
+    for (int c = 0; c < 32; ++c) {
+        const uint32_t mine = row_ok ? ordered_bits(__uint_as_float(v[c]) + 0.0f) : 0u;
+        const uint32_t m = __reduce_max_sync(0xffffffffu, mine);
+        if (lane == c) best = m > best ? m : best;
     }
-    int base = 0;
-    if (mine) {
-        base = atomicAdd(&cnt_chunk[lane], __popc(mine));
-        if (base + __popc(mine) >= kTcSoft) *dirty = 1;
-    }
-    const uint32_t below = (1u << lane) - 1u;
+}
+
+// Lane L's copy of the thresholds of queries L, L + 32, ... of both halves (+inf where there
+// is none): tl[h][j] belongs to query h * nb + j * 32 + L.
+__device__ __forceinline__ void tc_load_lane_thresholds(float (&tl)[2][kTcMaxN / 32], const float *thr, int nb,
+                                                        int nhalves, int lane) {
 #pragma unroll
-    for (int b = 0; b < 32; ++b) {
-        if (any_col & (1u << b)) {
-            const int base_b = __shfl_sync(0xffffffffu, base, b);
-            const uint32_t rows_b = __shfl_sync(0xffffffffu, mine, b);
-            if ((hit >> b) & 1u)
-                cand_chunk[static_cast<size_t>(b) * kTcCap + base_b + __popc(rows_b & below)] =
-                    make_key(__uint_as_float(v[b]), row);
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int j = 0; j < kTcMaxN / 32; ++j) {
+            const int q = h * nb + j * 32 + lane;
+            tl[h][j] = (h < nhalves && j * 32 < nb && q < kTcMaxQueries) ? thr[q] : INFINITY;
         }
-    }
 }
 
 // ---- CTA-pair helpers (PAIR = true: two CTAs of a cluster work as one MMA unit) -----------
@@ -392,8 +428,13 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
 }
+// Arrival on a barrier of the pair's other CTA. The barrier only hands a TMEM accumulator back, and
+// the reads it follows are ordered by tcgen05.wait::ld and the tcgen05 fence; the arrival's own release
+// stays at CTA scope. (With cluster scope it also waited for this thread's earlier global stores to be
+// visible across the cluster: about 2500 cycles per unit while TMA traffic is heavy, more than the
+// scores take to read.)
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void cluster_barrier() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -429,7 +470,9 @@ __device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t a_desc
 // 128 r .. 128 r + 127 and half of the query rows of each K chunk, the leader (rank 0) issues
 // one M = 256 MMA for both, and each CTA finds the scores of its own 128 rows in its own
 // TMEM. Per CTA and chunk this stages 16 KB + nb/2 query rows instead of 16 KB + nb.
-template <bool PAIR>
+// MODE: TcParams::mode as a compile-time constant, so that each launch carries only its own
+// selection code (the loops over 32-column blocks are fully unrolled).
+template <bool PAIR, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_q,
                const TcParams p) {
@@ -438,7 +481,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     float *thr = reinterpret_cast<float *>(tc_smem + kTcOffThr);
     int *cnt = reinterpret_cast<int *>(tc_smem + kTcOffCnt);
     int *sorted = reinterpret_cast<int *>(tc_smem + kTcOffSorted);
-    const int warp = threadIdx.x >> 5;
+    // (through a shuffle, so that the compiler knows the warp index to be the same in all lanes)
+    const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x >> 5), 0);
     const int lane = threadIdx.x & 31;
     const int S = p.stages;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;   // 0 = leader of the pair
@@ -471,7 +515,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         sorted[q] = 0;
     }
     float *qn = reinterpret_cast<float *>(tc_smem + kTcOffQn);
-    if (p.mode != 0) {
+    if (MODE == 1 || MODE == 2) {
         for (int q = threadIdx.x; q < kTcMaxQueries; q += kTcThreads) {
             float acc = 0.f;
             if (q < p.s) {
@@ -512,64 +556,77 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            // bytes that land per stage and phase on the barrier the MMA thread waits on: a
-            // pair's loads all report to the leader's barrier
-            const uint32_t stage_tx = static_cast<uint32_t>(kTcABytes + nb_cta * 128) * (PAIR ? 2u : 1u);
-            int st = 0;
-            uint32_t lap = 0;
-            long long issued = 0;
-            bool ok = true, stop = false;
-            for (long long u = 0; u < my_units && !stop; ++u) {
-                const long long tile = p.tile0 + group + (u / p.nhalves) * ngroups;
-                const int half = static_cast<int>(u % p.nhalves);
-                const int row_y = static_cast<int>(tile * kGroupRows + rank * kTcTileM);
-                // a pair splits the N of this unit's MMA, not nb: the follower supplies the upper
-                // half of the (rounded) queries this half really has
-                const int nq_u = (p.s - half * p.nb < p.nb) ? (p.s - half * p.nb) : p.nb;
-                const int query_y = half * p.nb + (PAIR ? static_cast<int>(rank) * (((nq_u + 31) & ~31) / 2) : 0);
-                for (int c = 0; c < p.nchunks; ++c) {
-                    ok = mbar_wait_bounded(smem_u32(&hdr->empty[st]), (lap & 1) ^ 1);
-                    if (!ok || *abort_flag) {
-                        stop = true;
-                        break;
-                    }
+        // All lanes run the loop; the elected lane issues the copies.
+        const bool elected = elect_one();
+        // bytes that land per chunk on the barrier the MMA warp waits on: a pair's loads all
+        // report to the leader's barrier
+        const uint32_t chunk_tx = static_cast<uint32_t>(kTcABytes + nb_cta * 128) * (PAIR ? 2u : 1u);
+        const uint32_t chunk_bytes = static_cast<uint32_t>(p.chunk_bytes);
+        const int nchunks = p.nchunks, SC = p.stage_chunks;
+        int st = 0;
+        uint32_t lap = 0;
+        long long issued = 0;
+        bool ok = true;
+        for (long long u = 0; u < my_units && ok; ++u) {
+            const long long tile = p.tile0 + group + (u / p.nhalves) * ngroups;
+            const int half = static_cast<int>(u % p.nhalves);
+            const int row_y = static_cast<int>(tile * kGroupRows + rank * kTcTileM);
+            // a pair splits the N of this unit's MMA, not nb: the follower supplies the upper
+            // half of the (rounded) queries this half really has
+            const int nq_u = (p.s - half * p.nb < p.nb) ? (p.s - half * p.nb) : p.nb;
+            const int query_y = half * p.nb + (PAIR ? static_cast<int>(rank) * (((nq_u + 31) & ~31) / 2) : 0);
+            for (int c = 0; c < nchunks; c += SC) {
+                const int kc = (nchunks - c < SC) ? (nchunks - c) : SC;
+                ok = tc_wait(smem_u32(&hdr->empty[st]), (lap & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                if (elected) {
                     const uint32_t bar = smem_u32(&hdr->full[st]);
                     const uint32_t dst = stage_base + static_cast<uint32_t>(st) * p.stage_bytes;
                     if (PAIR) {
                         const uint32_t lead_bar = map_to_cta(bar, 0);
-                        if (leader) mbar_arrive_expect_tx(bar, stage_tx);
-                        tma_load_2d_pair(dst, &map_x, c * kTcChunkK, row_y, lead_bar);
-                        tma_load_2d_pair(dst + kTcABytes, &map_q, c * kTcChunkK, query_y, lead_bar);
+                        if (leader) mbar_arrive_expect_tx(bar, chunk_tx * kc);
+                        for (int j = 0; j < kc; ++j) {
+                            tma_load_2d_pair(dst + j * chunk_bytes, &map_x, (c + j) * kTcChunkK, row_y, lead_bar);
+                            tma_load_2d_pair(dst + j * chunk_bytes + kTcABytes, &map_q, (c + j) * kTcChunkK, query_y,
+                                             lead_bar);
+                        }
                     } else {
-                        mbar_arrive_expect_tx(bar, stage_tx);
-                        tma_load_2d(dst, &map_x, c * kTcChunkK, row_y, bar);
-                        tma_load_2d(dst + kTcABytes, &map_q, c * kTcChunkK, query_y, bar);
-                    }
-                    ++issued;
-                    if (++st == S) {
-                        st = 0;
-                        ++lap;
+                        mbar_arrive_expect_tx(bar, chunk_tx * kc);
+                        for (int j = 0; j < kc; ++j) {
+                            tma_load_2d(dst + j * chunk_bytes, &map_x, (c + j) * kTcChunkK, row_y, bar);
+                            tma_load_2d(dst + j * chunk_bytes + kTcABytes, &map_q, (c + j) * kTcChunkK, query_y, bar);
+                        }
                     }
                 }
+                ++issued;
+                if (++st == S) {
+                    st = 0;
+                    ++lap;
+                }
             }
-            if (!ok && !*abort_flag) {
-                atomicMax(p.status, kStatusTimeout);
-                *abort_flag = 1;
-            }
-            if (*abort_flag && (!PAIR || leader)) {
-                // winding down early: let every copy already issued land before exit (a pair's
-                // follower cannot watch the leader's barrier; its copies land in its own shared
-                // memory, which stays allocated until both CTAs have passed the final barrier,
-                // and a wait has already run out by then)
-                const long long first = issued > S ? issued - S : 0;
-                for (long long it = first; it < issued; ++it)
-                    mbar_wait_bounded(smem_u32(&hdr->full[it % S]), static_cast<uint32_t>((it / S) & 1));
-            }
+        }
+        if (!ok && lane == 0 && !*abort_flag) {
+            atomicMax(p.status, kStatusTimeout);
+            *abort_flag = 1;
+        }
+        __syncwarp();
+        if (*abort_flag && (!PAIR || leader)) {
+            // winding down early: let every copy already issued land before exit (a pair's
+            // follower cannot watch the leader's barrier; its copies land in its own shared
+            // memory, which stays allocated until both CTAs have passed the final barrier,
+            // and a wait has already run out by then)
+            const long long first = issued > S ? issued - S : 0;
+            for (long long it = first; it < issued; ++it)
+                mbar_wait_bounded(smem_u32(&hdr->full[it % S]), static_cast<uint32_t>((it / S) & 1));
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0 && leader) {
+        // The leader CTA's warp, all lanes converged; the elected lane issues MMAs and commits.
+        if (leader) {
+            const bool elected = elect_one();
+            const uint64_t desc_fixed = tc_smem_desc(0);
+            const uint32_t chunk_desc = static_cast<uint32_t>(p.chunk_bytes) >> 4;
+            const int nchunks = p.nchunks, SC = p.stage_chunks;
             int st = 0;
             uint32_t lap = 0;
             bool ok = true;
@@ -581,45 +638,60 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const uint32_t idesc = tc_idesc(n_mma, kGroupRows);
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * kTcMaxN);
                 // the selection warps must have drained this accumulator's previous unit
-                ok = mbar_wait_bounded(smem_u32(&hdr->tmem_empty[acc]), static_cast<uint32_t>(((u >> 1) & 1) ^ 1));
-                if (!ok || *abort_flag) break;
+                ok = tc_wait(smem_u32(&hdr->tmem_empty[acc]), static_cast<uint32_t>(((u >> 1) & 1) ^ 1), abort_flag);
+                if (!ok) break;
                 tc_fence_after();
-                for (int c = 0; c < p.nchunks; ++c) {
+                uint32_t accumulate = 0;
+                for (int c = 0; c < nchunks; c += SC) {
+                    const int kc = (nchunks - c < SC) ? (nchunks - c) : SC;
                     // (the mbarrier wait orders the TMA writes before the MMAs that read them; no
                     // tcgen05 fence here: it is only needed where tcgen05 work of other threads,
                     // the selection warps' loads, has to be ordered, as above)
-                    ok = mbar_wait_bounded(smem_u32(&hdr->full[st]), lap & 1);
-                    if (!ok || *abort_flag) break;
-                    const uint32_t a_addr = stage_base + static_cast<uint32_t>(st) * p.stage_bytes;
-                    const uint32_t b_addr = a_addr + kTcABytes;
+                    ok = tc_wait(smem_u32(&hdr->full[st]), lap & 1, abort_flag);
+                    if (!ok) break;
+                    if (elected) {
+                        const uint32_t a_addr = stage_base + static_cast<uint32_t>(st) * p.stage_bytes;
+                        const uint64_t a_desc = desc_fixed | ((a_addr & 0x3FFFFu) >> 4);
+                        const uint64_t b_desc = desc_fixed | (((a_addr + kTcABytes) & 0x3FFFFu) >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < kTcChunkK / 16; ++kk) {
-                        if (PAIR)
-                            tc_mma_f16_pair(d_tmem, tc_smem_desc(a_addr + kk * 32), tc_smem_desc(b_addr + kk * 32),
-                                            idesc, (c | kk) != 0 ? 1u : 0u);
-                        else
-                            tc_mma_f16(d_tmem, tc_smem_desc(a_addr + kk * 32), tc_smem_desc(b_addr + kk * 32),
-                                       idesc, (c | kk) != 0 ? 1u : 0u);
+                        for (int j = 0; j < 2; ++j) {
+                            if (j < kc) {
+#pragma unroll
+                                for (int kk = 0; kk < kTcChunkK / 16; ++kk) {
+                                    // (a K step of 16 is 32 bytes further along the 128-byte rows)
+                                    const uint32_t step = j * chunk_desc + kk * 2;
+                                    if (PAIR) tc_mma_f16_pair(d_tmem, a_desc + step, b_desc + step, idesc, accumulate);
+                                    else tc_mma_f16(d_tmem, a_desc + step, b_desc + step, idesc, accumulate);
+                                    accumulate = 1;
+                                }
+                            }
+                        }
+                        // stage reusable (in both CTAs of a pair) once these MMAs are done
+                        if (PAIR) tc_commit_pair(smem_u32(&hdr->empty[st]));
+                        else tc_commit(smem_u32(&hdr->empty[st]));
                     }
-                    // stage reusable (in both CTAs of a pair) once these MMAs are done
-                    if (PAIR) tc_commit_pair(smem_u32(&hdr->empty[st]));
-                    else tc_commit(smem_u32(&hdr->empty[st]));
+                    accumulate = 1;
                     if (++st == S) {
                         st = 0;
                         ++lap;
                     }
                 }
-                if (!ok || *abort_flag) break;
-                if (PAIR) tc_commit_pair(smem_u32(&hdr->tmem_full[acc]));
-                else tc_commit(smem_u32(&hdr->tmem_full[acc]));
+                if (!ok) break;
+                if (elected) {
+                    if (PAIR) tc_commit_pair(smem_u32(&hdr->tmem_full[acc]));
+                    else tc_commit(smem_u32(&hdr->tmem_full[acc]));
+                }
             }
-            if (!ok && !*abort_flag) {
+            if (!ok && lane == 0 && !*abort_flag) {
                 atomicMax(p.status, kStatusTimeout);
                 *abort_flag = 1;
             }
+            __syncwarp();
             // every MMA issued above must have completed before the TMEM is given back
-            if (PAIR) tc_commit_pair(smem_u32(&hdr->drain));
-            else tc_commit(smem_u32(&hdr->drain));
+            if (elected) {
+                if (PAIR) tc_commit_pair(smem_u32(&hdr->drain));
+                else tc_commit(smem_u32(&hdr->drain));
+            }
             mbar_wait_bounded(smem_u32(&hdr->drain), 0);
         }
     } else {
@@ -627,7 +699,23 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const int ew = warp - 2;        // 0..3
         const int quarter = warp & 3;   // the TMEM lanes this warp may read: 32 * quarter ..
         uint64_t *my_cand = p.cand + static_cast<size_t>(blockIdx.x) * p.cand_q * kTcCap;
+        constexpr bool sample = MODE == 1 || MODE == 3;
+        constexpr bool l2 = MODE == 1 || MODE == 2;
         bool ok = true;
+        // Per-query values live in registers, spread over the lanes: lane L holds those of queries
+        // L, L + 32, ... and column c's value reaches every row by a shuffle from lane c. The
+        // common path then reads no shared memory, whose loads take several times longer while
+        // TMA and the tensor core keep it busy (440 against 100 cycles per block of 32 queries).
+        // tl: thresholds (main launches; reloaded after a compaction meeting, the only place where
+        // they move). qnl: |q|^2 (L2). best: running maxima of a sample launch.
+        float tl[2][kTcMaxN / 32], qnl[2][kTcMaxN / 32];
+        uint32_t best[2][kTcMaxN / 32];
+        tc_load_lane_thresholds(tl, thr, p.nb, p.nhalves, lane);
+        if (l2) tc_load_lane_thresholds(qnl, qn, p.nb, p.nhalves, lane);
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int j = 0; j < kTcMaxN / 32; ++j) best[h][j] = 0u;
         for (long long u = 0; u < my_units; ++u) {
             const long long tile = p.tile0 + group + (u / p.nhalves) * ngroups;
             const int half = static_cast<int>(u % p.nhalves);
@@ -655,52 +743,77 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const bool row_ok = row < p.N;
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                        static_cast<uint32_t>(acc * kTcMaxN);
-                const float nx = (p.mode != 0 && row_ok) ? __ldg(p.norms + row) : 0.f;
-                const float bound_sign = p.mode == 1 ? -1.0f : 1.0f;
-                for (int j = 0; p.mode != 0 && j * 32 < nq; ++j) {
-                    // L2: the same loop on the bound of -distance^2 (see TcParams::mode)
-                    uint32_t v[32];
-                    tmem_ld32(t_row + j * 32, v);
-                    const float4 *t4 = reinterpret_cast<const float4 *>(thr + qb + j * 32);
-                    const float4 *n4 = reinterpret_cast<const float4 *>(qn + qb + j * 32);
-                    const float sl = bound_sign * p.slack;
-                    bool p0 = false, p1 = false, p2 = false, p3 = false;
+                const float nx = (l2 && row_ok) ? __ldg(p.norms + row) : 0.f;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float4 th = t4[i];
-                        const float4 nq4 = n4[i];
-                        const float s0 = nx + nq4.x, s1 = nx + nq4.y, s2 = nx + nq4.z, s3 = nx + nq4.w;
-                        p0 |= fmaf(sl, s0, fmaf(2.0f, __uint_as_float(v[4 * i + 0]), 0.0f - s0)) >= th.x;
-                        p1 |= fmaf(sl, s1, fmaf(2.0f, __uint_as_float(v[4 * i + 1]), 0.0f - s1)) >= th.y;
-                        p2 |= fmaf(sl, s2, fmaf(2.0f, __uint_as_float(v[4 * i + 2]), 0.0f - s2)) >= th.z;
-                        p3 |= fmaf(sl, s3, fmaf(2.0f, __uint_as_float(v[4 * i + 3]), 0.0f - s3)) >= th.w;
-                    }
-                    if (__any_sync(0xffffffffu, row_ok && (p0 | p1 | p2 | p3)))
-                        tc_append_chunk_l2(t_row + j * 32, thr + qb + j * 32, qn + qb + j * 32, cnt + qb + j * 32,
-                                           my_cand + static_cast<size_t>(qb + j * 32) * kTcCap,
-                                           static_cast<uint32_t>(row), row_ok, nx, p.slack, bound_sign, p.corpus,
-                                           p.queries + static_cast<size_t>(qb + j * 32) * p.d, p.d, dirty, lane);
-                }
-                for (int j = 0; p.mode == 0 && j * 32 < nq; ++j) {
-                    uint32_t v[32];
-                    tmem_ld32(t_row + j * 32, v);
-                    const float4 *t4 = reinterpret_cast<const float4 *>(thr + qb + j * 32);
-                    // common case: nothing passes. Four independent predicate chains.
-                    bool p0 = false, p1 = false, p2 = false, p3 = false;
+                for (int j = 0; j < kTcMaxN / 32; ++j) {
+                    if (j * 32 < nq) {
+                        uint32_t v[32];
+                        tmem_ld32(t_row + j * 32, v);
+                        if (sample) {
+                            if (l2) {
+                                // the LOWER bound of -distance^2 (see TcParams::mode)
+                                const float my_qn = half ? qnl[1][j] : qnl[0][j];
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float4 th = t4[i];
-                        p0 |= __uint_as_float(v[4 * i + 0]) >= th.x;
-                        p1 |= __uint_as_float(v[4 * i + 1]) >= th.y;
-                        p2 |= __uint_as_float(v[4 * i + 2]) >= th.z;
-                        p3 |= __uint_as_float(v[4 * i + 3]) >= th.w;
+                                for (int c = 0; c < 32; ++c) {
+                                    const float s2 = nx + __shfl_sync(0xffffffffu, my_qn, c);
+                                    const float val = fmaf(2.0f, __uint_as_float(v[c]), 0.0f - s2);
+                                    v[c] = __float_as_uint(fmaf(0.0f - p.slack, s2, val));
+                                }
+                            }
+                            if (half) tc_fold_block_maxima(v, row_ok, best[1][j], lane);
+                            else tc_fold_block_maxima(v, row_ok, best[0][j], lane);
+                        } else if (l2) {
+                            // the UPPER bound of -distance^2 against the thresholds
+                            const float my_thr = half ? tl[1][j] : tl[0][j];
+                            const float my_qn = half ? qnl[1][j] : qnl[0][j];
+                            bool p0 = false, p1 = false;
+#pragma unroll
+                            for (int c = 0; c < 32; c += 2) {
+                                const float s0 = nx + __shfl_sync(0xffffffffu, my_qn, c);
+                                const float s1 = nx + __shfl_sync(0xffffffffu, my_qn, c + 1);
+                                p0 |= fmaf(p.slack, s0, fmaf(2.0f, __uint_as_float(v[c]), 0.0f - s0)) >=
+                                      __shfl_sync(0xffffffffu, my_thr, c);
+                                p1 |= fmaf(p.slack, s1, fmaf(2.0f, __uint_as_float(v[c + 1]), 0.0f - s1)) >=
+                                      __shfl_sync(0xffffffffu, my_thr, c + 1);
+                            }
+                            if (__any_sync(0xffffffffu, row_ok && (p0 | p1)))
+                                tc_append_chunk_l2(t_row + j * 32, thr + qb + j * 32, qn + qb + j * 32, cnt + qb + j * 32,
+                                                   my_cand + static_cast<size_t>(qb + j * 32) * kTcCap,
+                                                   static_cast<uint32_t>(row), row_ok, nx, p.slack, p.corpus,
+                                                   p.queries + static_cast<size_t>(qb + j * 32) * p.d, p.d, dirty, p.status, lane);
+                        } else {
+                            // common case: nothing passes. Four independent predicate chains, one per
+                            // eight columns, so that the rare case only revisits the eight it concerns.
+                            const float my_thr = half ? tl[1][j] : tl[0][j];
+                            bool p0 = false, p1 = false, p2 = false, p3 = false;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                p0 |= __uint_as_float(v[i]) >= __shfl_sync(0xffffffffu, my_thr, i);
+                                p1 |= __uint_as_float(v[8 + i]) >= __shfl_sync(0xffffffffu, my_thr, 8 + i);
+                                p2 |= __uint_as_float(v[16 + i]) >= __shfl_sync(0xffffffffu, my_thr, 16 + i);
+                                p3 |= __uint_as_float(v[24 + i]) >= __shfl_sync(0xffffffffu, my_thr, 24 + i);
+                            }
+                            if (__any_sync(0xffffffffu, row_ok && (p0 | p1 | p2 | p3))) {
+                                int *cnt_block = cnt + qb + j * 32;
+                                uint64_t *cand_block = my_cand + static_cast<size_t>(qb + j * 32) * kTcCap;
+                                const uint32_t r32 = static_cast<uint32_t>(row);
+                                if (__any_sync(0xffffffffu, row_ok && p0))
+                                    tc_append_octet(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], 0, my_thr, cnt_block,
+                                                    cand_block, r32, row_ok, dirty, p.status);
+                                if (__any_sync(0xffffffffu, row_ok && p1))
+                                    tc_append_octet(v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15], 8, my_thr,
+                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status);
+                                if (__any_sync(0xffffffffu, row_ok && p2))
+                                    tc_append_octet(v[16], v[17], v[18], v[19], v[20], v[21], v[22], v[23], 16, my_thr,
+                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status);
+                                if (__any_sync(0xffffffffu, row_ok && p3))
+                                    tc_append_octet(v[24], v[25], v[26], v[27], v[28], v[29], v[30], v[31], 24, my_thr,
+                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status);
+                            }
+                        }
                     }
-                    if (__any_sync(0xffffffffu, row_ok && (p0 | p1 | p2 | p3)))
-                        tc_append_chunk(t_row + j * 32, thr + qb + j * 32, cnt + qb + j * 32,
-                                        my_cand + static_cast<size_t>(qb + j * 32) * kTcCap,
-                                        static_cast<uint32_t>(row), row_ok, dirty, lane);
                 }
-                // accumulator drained: hand it back to the MMA thread (the pair's leader)
+                // accumulator drained: hand it back to the MMA warp (the pair's leader)
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
@@ -708,6 +821,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     else mbar_arrive(smem_u32(&hdr->tmem_empty[acc]));
                 }
             }
+            if (sample) continue;   // no lists, nothing to compact
             // All four warps meet after every unit (also when winding down, so that nobody is
             // left waiting) so that every push of the unit is visible; each then reads the
             // unit's flag. Three flags in rotation make one barrier enough: unit u's flag is
@@ -728,18 +842,32 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     }
                 }
                 named_barrier(1, 128);  // thresholds and counts settled before the next unit's pushes
+                tc_load_lane_thresholds(tl, thr, p.nb, p.nhalves, lane);
             }
         }
-        // ---- CTA result: every list sorted and cut to k, written as this CTA's partial lists
-        for (int base = 0; base < p.s; base += 128) {
-            const int q0 = base + ew * 32;
-            for (int b = 0; b < 32 && q0 + b < p.s; ++b) {
-                const int q = q0 + b;
-                uint64_t *list = my_cand + static_cast<size_t>(q) * kTcCap;
-                if (cnt[q] != sorted[q]) tc_compact_query(list, thr, cnt, sorted, q, p.k, lane);
-                const int n = cnt[q];
-                uint64_t *dst = p.partial + (static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
-                for (int i = lane; i < p.k; i += 32) dst[i] = (i < n) ? list[i] : 0ull;
+        if (sample) {
+            // ---- this warp's best rank value per query (-inf if it saw no row)
+            float *dst = p.gmax + (static_cast<size_t>(blockIdx.x) * 4 + ew) * p.s_total + p.q_base;
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int j = 0; j < kTcMaxN / 32; ++j) {
+                    const int q = h * p.nb + j * 32 + lane;
+                    if (h < p.nhalves && j * 32 < p.nb && q < p.s)
+                        dst[q] = best[h][j] ? from_ordered_bits(best[h][j]) : -INFINITY;
+                }
+        } else {
+            // ---- CTA result: every list sorted and cut to k, written as this CTA's partial lists
+            for (int base = 0; base < p.s; base += 128) {
+                const int q0 = base + ew * 32;
+                for (int b = 0; b < 32 && q0 + b < p.s; ++b) {
+                    const int q = q0 + b;
+                    uint64_t *list = my_cand + static_cast<size_t>(q) * kTcCap;
+                    if (cnt[q] != sorted[q]) tc_compact_query(list, thr, cnt, sorted, q, p.k, lane);
+                    const int n = cnt[q];
+                    uint64_t *dst = p.partial + (static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
+                    for (int i = lane; i < p.k; i += 32) dst[i] = (i < n) ? list[i] : 0ull;
+                }
             }
         }
     }

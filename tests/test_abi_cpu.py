@@ -34,8 +34,8 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_status_strings(lib):
     lib.ralm_status_string.restype = ctypes.c_char_p
-    seen = {lib.ralm_status_string(i) for i in range(7)}
-    assert len(seen) == 7 and all(seen)
+    seen = {lib.ralm_status_string(i) for i in range(9)}
+    assert len(seen) == 9 and all(seen)
 
 
 def test_host_side_argument_checks_need_no_gpu(lib):

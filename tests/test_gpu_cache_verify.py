@@ -7,7 +7,7 @@ import torch
 
 import oracle
 import workloads
-from parity import check_lists
+from parity import Counts, check_lists
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -25,16 +25,14 @@ def _check_cache(ralm, idx, x, cache, q, metric, k):
     xn, qn = x.cpu().numpy(), q.cpu().numpy()
     oi, osc = oracle.cache_search(xn, cache.cpu().numpy(), qn, metric, k)
     gi, gs = ids.cpu().numpy(), scores.cpu().numpy()
-    strict = band = 0
+    counts = Counts()
     for r in range(cache.shape[0]):
         for u in range(q.shape[1]):
-            a, b = check_lists(gi[r, u], gs[r, u], oi[r, u], osc[r, u],
-                               lambda j: oracle.pair_score(xn[j], qn[r, u], metric), metric,
-                               scale=float(np.abs(osc[r, u][np.isfinite(osc[r, u])]).max(initial=1.0)),
-                               n_valid=xn.shape[0])
-            strict += a
-            band += b
-    return ids, strict, band
+            counts += check_lists(gi[r, u], gs[r, u], oi[r, u], osc[r, u],
+                                  lambda j: oracle.pair_score(xn[j], qn[r, u], metric), metric,
+                                  scale=float(np.abs(osc[r, u][np.isfinite(osc[r, u])]).max(initial=1.0)),
+                                  n_valid=xn.shape[0])
+    return ids, counts
 
 
 @pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
@@ -67,6 +65,23 @@ def test_cache_integer_inputs_bit_exact_with_duplicates_and_empty():
         assert np.array_equal(ids.cpu().numpy(), oi)
         assert np.array_equal(scores.cpu().numpy().astype(np.float64), osc)
         assert (ids[1] == -1).all()
+
+
+def test_cache_search_with_more_requests_than_a_grid_dimension_holds():
+    """100 000 requests of 8 slots (the key buffer's limit is R * q * C <= 2^20): the request index
+    must not sit in a grid dimension that stops at 65 535."""
+    ralm = _ralm()
+    R, C, d = 100_000, 8, 64
+    x = workloads.integer_valued((500, d), seed=66, lo=-3, hi=3, device=DEV)
+    q = workloads.integer_valued((R, 1, d), seed=67, lo=-3, hi=3, device=DEV)
+    cache = torch.randint(0, 500, (R, C), device=DEV, generator=torch.Generator(DEV).manual_seed(2))
+    idx = ralm.Index(x, oracle.IP, 8, 2)
+    ids, scores = ralm.cache_search(idx, cache, q, 2)
+    torch.cuda.synchronize()
+    assert idx.device_status() == 0
+    oi, osc = oracle.cache_search(x.cpu().numpy(), cache.cpu().numpy(), q.cpu().numpy(), oracle.IP, 2)
+    assert np.array_equal(ids.cpu().numpy(), oi)
+    assert np.array_equal(scores.cpu().numpy().astype(np.float64), osc)
 
 
 def test_cache_over_all_ids_equals_search():

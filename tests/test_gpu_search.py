@@ -213,7 +213,7 @@ def test_tcgen05_scan_parity(N, d, s, k):
     x, _ = workloads.mixture_corpus(N, d, 64, seed=600 + d, device=DEV)
     q, src = workloads.noisy_copy_queries(x, s, seed=601 + d)
     ids, scores = _run(x, q, oracle.IP, k)
-    strict, band = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k)
     assert ids[:, 0].tolist() == src.tolist()
     ids8, scores8 = _run(x, q, oracle.IP, k, 2)          # the 8-queries-per-pass scan on the same batch
     assert torch.equal(ids[:, 0], ids8[:, 0])
@@ -249,13 +249,13 @@ def test_tcgen05_scan_l2_parity_and_duplicates():
     q, src = workloads.noisy_copy_queries(x, s, seed=96)
     q[:4] = x[src[:4]]                                   # exact copies: distance exactly 0, ranked first
     ids, scores = _run(x, q, oracle.L2, k)               # 64 queries: the large-batch scan by itself
-    strict, band = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, k)
+    counts = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, k)
     assert ids[:, 0].tolist() == src.tolist()
     assert (scores[:4, 0] == 0).all()
     ids8, scores8 = _run(x, q, oracle.L2, k, 2)          # eight queries per pass on the same batch
     assert torch.equal(ids[:, 0], ids8[:, 0])
     torch.testing.assert_close(scores, scores8, rtol=1e-4, atol=1e-4)
-    print("L2 large batch: strict=%d band=%d" % (strict, band))
+    print("L2 large batch: %s" % counts)
 
 
 @pytest.mark.parametrize("metric", [oracle.IP, oracle.L2])
@@ -323,8 +323,12 @@ def test_config_c1():
     for k in c.k_values:
         for variant in (2, 1):
             ids, scores = _run(x, q, oracle.IP, k, variant)
-            strict, band = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k)
+            counts = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k)
             assert ids[:, 0].tolist() == src.tolist()
+            # a swap between rows whose fp64 scores differ by more than fp32 rounding explains
+            # is accepted by the 2e-3 rule but is not expected: none may occur
+            assert counts.wide == 0, "C1 k=%d variant=%d: %s" % (k, variant, counts)
+            print("C1 s=4 k=%d variant=%d %s" % (k, variant, counts))
 
 
 @pytest.mark.parametrize("s", [1, 2, 4, 8])
@@ -333,9 +337,10 @@ def test_config_c2(s, c2_corpus):
     q, src = workloads.noisy_copy_queries(x, s, workloads.seed_for(2, "queries"))
     for k in (1, 20):
         ids, scores = _run(x, q, oracle.IP, k)
-        strict, band = check_search(ids, scores, xn, q.cpu().numpy(), oracle.IP, k)
+        counts = check_search(ids, scores, xn, q.cpu().numpy(), oracle.IP, k)
         assert ids[:, 0].tolist() == src.tolist()
-        print("C2 s=%d k=%d strict=%d band=%d" % (s, k, strict, band))
+        assert counts.wide == 0, "C2 s=%d k=%d: %s" % (s, k, counts)
+        print("C2 s=%d k=%d %s" % (s, k, counts))
 
 
 @pytest.fixture(scope="module")
@@ -352,6 +357,7 @@ def test_knn_lm_shape_l2_k1024():
     q, src = workloads.noisy_copy_queries(x, 4, workloads.seed_for(4, "queries"))
     for variant in (2, 1):
         ids, scores = _run(x, q, oracle.L2, 1024, variant)
-        strict, band = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, 1024)
+        counts = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, 1024)
         assert ids[:, 0].tolist() == src.tolist()
-        print("C4/50 variant=%d strict=%d band=%d" % (variant, strict, band))
+        assert counts.wide == 0, "C4/50 variant=%d: %s" % (variant, counts)
+        print("C4/50 variant=%d %s" % (variant, counts))

@@ -96,7 +96,41 @@ def test_shards_on_one_gpu_reproduce_the_unsharded_search(metric, k, G):
     got_ids, got_scores = ralm.merge_lists(torch.stack(ids), torch.stack(scores),
                                            torch.tensor(offsets, dtype=torch.int64, device=DEV), metric)
     torch.cuda.synchronize()
+    # the reference is the oracle over the WHOLE corpus (integer data: ids and scores bit for bit,
+    # ties across shard boundaries included); the library's own unsharded search must agree too
+    import oracle
+    from parity import check_search
+    check_search(got_ids, got_scores, x.cpu().numpy(), q.cpu().numpy(), metric, k, exact=True)
     assert torch.equal(got_ids, want_ids) and torch.equal(got_scores, want_scores)
+
+
+@pytest.mark.gpu
+def test_shards_of_real_valued_rows_against_the_oracle():
+    """Mixture rows (near ties, fp32 rounding): the merged answer of 4 shards against the oracle's
+    ranking of the whole corpus, by the near-tie rule."""
+    import paper_2401_14021_b200 as ralm
+    import oracle
+    from parity import check_search
+    from paper_2401_14021_b200.sharded import shard_rows
+    N, d, s, k, G = 120_000, 256, 8, 20, 4
+    x, _ = workloads.mixture_corpus(N, d, 64, seed=35, device=DEV)
+    q, src = workloads.noisy_copy_queries(x, s, seed=36)
+    ids, scores, offsets = [], [], []
+    for g in range(G):
+        lo, hi = shard_rows(N, G, g)
+        shard = ralm.Index(x[lo:hi], ralm.IP, s, k)
+        i, sc = ralm.search(shard, q, k)
+        torch.cuda.synchronize()
+        ids.append(i)
+        scores.append(sc)
+        offsets.append(lo)
+        shard.close()
+    got_ids, got_scores = ralm.merge_lists(torch.stack(ids), torch.stack(scores),
+                                           torch.tensor(offsets, dtype=torch.int64, device=DEV), ralm.IP)
+    torch.cuda.synchronize()
+    counts = check_search(got_ids, got_scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k)
+    assert got_ids[:, 0].tolist() == src.tolist()
+    assert counts.wide == 0, str(counts)
 
 
 @pytest.mark.gpu

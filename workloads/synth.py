@@ -56,34 +56,50 @@ def _gen(seed: int, chunk: int, device) -> torch.Generator:
     return g
 
 
+def _range(N: int, row_range) -> Tuple[int, int]:
+    lo, hi = (0, N) if row_range is None else row_range
+    if not 0 <= lo <= hi <= N:
+        raise ValueError("row_range outside the corpus")
+    return lo, hi
+
+
 def unit_gaussian_corpus(N: int, d: int, seed: int, device="cpu",
-                         chunk_rows: int = CHUNK_ROWS) -> torch.Tensor:
-    """Rows i.i.d. N(0, I_d), scaled to unit length in fp32, rounded to fp16."""
-    out = torch.empty((N, d), dtype=torch.float16, device=device)
+                         chunk_rows: int = CHUNK_ROWS, row_range=None) -> torch.Tensor:
+    """Rows i.i.d. N(0, I_d), scaled to unit length in fp32, rounded to fp16.
+    row_range = (lo, hi): only those rows of the N-row corpus (the same bytes the whole corpus
+    holds there: every chunk is generated from its own seed)."""
+    r_lo, r_hi = _range(N, row_range)
+    out = torch.empty((r_hi - r_lo, d), dtype=torch.float16, device=device)
     for b, lo in enumerate(range(0, N, chunk_rows)):
         hi = min(N, lo + chunk_rows)
+        if hi <= r_lo or lo >= r_hi:
+            continue
         u = torch.randn((hi - lo, d), generator=_gen(seed, b, device), device=device,
                         dtype=torch.float32)
         u /= u.norm(dim=1, keepdim=True).clamp_min(1e-20)
-        out[lo:hi] = u.to(torch.float16)
+        a, z = max(lo, r_lo), min(hi, r_hi)
+        out[a - r_lo:z - r_lo] = u[a - lo:z - lo].to(torch.float16)
     return out
 
 
 def mixture_corpus(N: int, d: int, n_centres: int, seed: int, device="cpu",
                    sigma_within: float = 0.2, normalise: bool = True,
                    lognormal_sigma: float = 0.0, clustered_order: bool = False,
-                   chunk_rows: int = CHUNK_ROWS) -> Tuple[torch.Tensor, torch.Tensor]:
+                   chunk_rows: int = CHUNK_ROWS, row_range=None) -> Tuple[torch.Tensor, torch.Tensor]:
     """Gaussian-mixture corpus.
 
     Centres c_m ~ N(0, I_d). Row j picks a centre a_j uniformly and independently (so row
     order is NOT clustered unless `clustered_order`, which sorts the assignment to build
     the adversarial ordering), u_j = c_{a_j} + sigma_within * eps_j. Then either
     x_j = fp16(u_j / |u_j|) or, unnormalised, x_j = fp16(u_j * exp(lognormal_sigma * z_j)).
-    Returns (corpus [N][d] fp16, assignment [N] int32).
+    Returns (corpus [N][d] fp16, assignment [N] int32). With row_range = (lo, hi) the corpus
+    holds only those rows of the N-row corpus (the same bytes: every chunk is generated from its
+    own seed); the assignment is still that of all N rows.
     """
+    r_lo, r_hi = _range(N, row_range)
     centres = torch.randn((n_centres, d), generator=_gen(seed, 1_000_000, device),
                           device=device, dtype=torch.float32)
-    out = torch.empty((N, d), dtype=torch.float16, device=device)
+    out = torch.empty((r_hi - r_lo, d), dtype=torch.float16, device=device)
     assign = torch.empty((N,), dtype=torch.int32, device=device)
     for b, lo in enumerate(range(0, N, chunk_rows)):
         hi = min(N, lo + chunk_rows)
@@ -91,6 +107,9 @@ def mixture_corpus(N: int, d: int, n_centres: int, seed: int, device="cpu",
         a = torch.randint(0, n_centres, (hi - lo,), generator=g, device=device)
         if clustered_order:
             a = (torch.arange(lo, hi, device=device) * n_centres) // max(N, 1)
+        assign[lo:hi] = a.to(torch.int32)
+        if hi <= r_lo or lo >= r_hi:
+            continue
         u = torch.randn((hi - lo, d), generator=g, device=device, dtype=torch.float32)
         u.mul_(sigma_within).add_(centres[a])
         if normalise:
@@ -98,21 +117,28 @@ def mixture_corpus(N: int, d: int, n_centres: int, seed: int, device="cpu",
         if lognormal_sigma > 0.0:
             z = torch.randn((hi - lo, 1), generator=g, device=device, dtype=torch.float32)
             u *= torch.exp(lognormal_sigma * z)
-        out[lo:hi] = u.to(torch.float16)
-        assign[lo:hi] = a.to(torch.int32)
+        first, last = max(lo, r_lo), min(hi, r_hi)
+        out[first - r_lo:last - r_lo] = u[first - lo:last - lo].to(torch.float16)
         del u, a
     return out, assign
 
 
 def noisy_copy_queries(corpus: torch.Tensor, s: int, seed: int, sigma: float = 0.1,
-                       relative: bool = True) -> Tuple[torch.Tensor, torch.Tensor]:
+                       relative: bool = True, n_rows: Optional[int] = None,
+                       fetch=None) -> Tuple[torch.Tensor, torch.Tensor]:
     """s queries, each a noisy copy of a distinct random corpus row.
+
+    When the corpus is spread over several holders, `corpus` is any tensor on the right device
+    with d columns, `n_rows` the row count of the whole corpus and `fetch(ids)` returns its rows
+    `ids` (fp16 [len(ids)][d]); the queries are then the same as for the corpus in one piece.
 
     relative=True: noise std per coordinate = sigma * |x_src| / sqrt(d) (noise of expected
     norm sigma * |x_src|). relative=False: noise std = sigma per coordinate.
     Returns (queries [s][d] fp16, source ids [s] int64).
     """
     N, d = corpus.shape
+    if n_rows is not None:
+        N = n_rows
     device = corpus.device
     g = _gen(seed, 0, device)
     if s <= N:
@@ -120,7 +146,7 @@ def noisy_copy_queries(corpus: torch.Tensor, s: int, seed: int, sigma: float = 0
             _distinct_randint(N, s, g, device)
     else:
         src = torch.randint(0, N, (s,), generator=g, device=device)
-    x = corpus[src].to(torch.float32)
+    x = (corpus[src] if fetch is None else fetch(src)).to(torch.float32)
     eps = torch.randn((s, d), generator=g, device=device, dtype=torch.float32)
     if relative:
         scale = sigma * x.norm(dim=1, keepdim=True) / (d ** 0.5)
