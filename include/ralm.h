@@ -211,20 +211,23 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
  * variable RALM_FORCE_VARIANT=<1..4> applies the same pin to every index at creation. */
 ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant);
 
-/* Optional for inner-product indexes: build a one-byte-per-element copy of the corpus (E5M2,
- * N * d bytes, plus one fp32 bound per row) that ralm_search then streams instead of the fp16 rows
- * for batches of up to 8 queries with k <= 256, and of 9..16 queries with k <= 64, under the
- * automatic variant (other shapes take the fp16 scans). The copy only
- * FILTERS: by the Cauchy-Schwarz inequality the score of the rounded row is within
- * |q| * |x - x8| of the true one, a (row, query) pair whose upper bound cannot reach the score
- * that k rows are already known to reach is dropped, and every other pair is scored again from
- * the fp16 row, which is the value that is ranked and returned. Results are those of the fp16
- * scan (what the paper's exact dense retriever returns, Section 5.1); the bytes streamed per
- * batch drop to about half. The copy is used on corpora large enough for the sample phase that
+/* Optional: build a one-byte-per-element copy of the corpus (E5M2, N * d bytes, plus one fp32
+ * bound per row) that ralm_search then streams instead of the fp16 rows for batches of up to 8
+ * queries (any k the index allows) and of 9..16 queries with k <= 64, under the automatic variant
+ * (other shapes take the fp16 scans). The copy only
+ * FILTERS: by the Cauchy-Schwarz inequality the inner product with the rounded row is within
+ * |q| * |x - x8| of the true one, which bounds the score (inner product) or, with the rows' stored
+ * squared norms, the squared distance (L2) from the right side; a (row, query) pair whose bound
+ * cannot reach the value that k rows are already known to reach is dropped, and every other pair
+ * is scored again from the fp16 row (L2: in the direct sum-of-squared-differences form), which is
+ * the value that is ranked and returned. Results are those of the fp16
+ * scan (what the paper's exact dense retriever returns, Section 5.1; the KNN-LM datastore's
+ * neighbours and distances, Section 5.3); the bytes streamed per batch drop to about half. The
+ * copy is used on corpora large enough for the sample phase that
  * gives the filter its thresholds (about 2.4 M rows); smaller ones keep the fp16 scan unless
  * `force` is non-zero (a testing aid: correct, but slow without thresholds to start from).
  * One pass over the corpus on the default stream, synchronous; allocates device memory.
- * Errors: UNSUPPORTED for L2 indexes or d % 16 != 0; OOM. Calling it again only updates `force`. */
+ * Errors: UNSUPPORTED for d % 16 != 0; OOM. Calling it again only updates `force`. */
 ralm_status_t ralm_index_enable_q8(ralm_index_t *idx, int32_t force);
 
 /* Override the scan kernel's launch shape on this index (benchmarking aid; 0 keeps the

@@ -34,6 +34,7 @@ struct ralm_index {
     uint64_t *cache_keys;  // [RALM_MAX_CACHE_KEYS]
     uint64_t *spill;       // large k: candidate lists of the small-batch scan, [num_sms][8][spill_cap]
     int spill_cap;
+    uint32_t *pub;         // large k: thresholds the scan CTAs publish to each other, [num_sms][max_s]
     float *norms;          // L2: squared norm of every corpus row (fp32 [N]), or null
     uint8_t *x8;           // inner product, optional: one-byte (E5M2) copy of the corpus, [N][d]
     float *x8_bound;       // per row: bound on |q.x - q.x8| per unit of |q| (see scan_q8.cuh)
@@ -67,6 +68,7 @@ struct ScanPlan {
 };
 
 constexpr int kSmemCandBytes = 32 * 1024;  // candidate lists larger than this leave shared memory
+constexpr int kPubMinK = 128;              // from this k on the scan CTAs share thresholds (ScanParams::pub)
 
 int align_up(int v, int a) { return (v + a - 1) / a * a; }
 
@@ -135,13 +137,19 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
 
 // Shared-memory layout of one CTA of the 8-bit scan: 16-row tiles of d bytes, 8 or 16 staged
 // queries, candidate lists in shared memory: k <= kQ8MaxK for up to 8 queries, k <= kQ8MaxKWide
-// (lists of 256 slots) for 9..16, which keeps them within kSmemCandBytes.
+// (lists of 256 slots) for 9..16, which keeps them within kSmemCandBytes. Larger k (up to 8
+// queries) keeps the lists in global memory, as the fp16 scan does, when the index has them.
 constexpr int kQ8MaxK = 256;
 constexpr int kQ8MaxKWide = 64;
 constexpr int kQ8MaxQueries = 2 * kScanMaxQueries;
 bool plan_scan_q8(const ralm_index *idx, int s_pass, int k, ScanPlan *pl) {
     const int q_rows = s_pass > kScanMaxQueries ? kQ8MaxQueries : kScanMaxQueries;
-    if (s_pass > kQ8MaxQueries || k > (q_rows > kScanMaxQueries ? kQ8MaxKWide : kQ8MaxK)) return false;
+    // (lists beyond 256 slots go to global memory whenever the index has room for them there: with
+    // 512 slots in shared memory the stage ring loses a consumer warp, and this scan is bound by
+    // those; with more, the lists do not fit at all)
+    const bool spill = q_rows == kScanMaxQueries && k > kQ8MaxKWide && idx->spill &&
+                       std::max(512, 2 * next_pow2(k)) <= idx->spill_cap;
+    if (s_pass > kQ8MaxQueries || (k > (q_rows > kScanMaxQueries ? kQ8MaxKWide : kQ8MaxK) && !spill)) return false;
     pl->tile_rows = 16;
     pl->stage_bytes = align_up(pl->tile_rows * idx->d + kQ8TileBytesExtra, 128);
     pl->off_q = kScanHeaderBytes;
@@ -155,7 +163,8 @@ bool plan_scan_q8(const ralm_index *idx, int s_pass, int k, ScanPlan *pl) {
         // consumer warps, and this scan is bound by them: 2.59 against 2.35 ms on 21 M x 768)
         pl->cap = (q_rows > kScanMaxQueries || k <= kQ8MaxKWide) ? 256 : std::max(512, 2 * next_pow2(k));
         pl->soft_limit = std::min(pl->cap - (kMaxConsumerWarps + 1) * pl->tile_rows, std::max(4 * k, 64));
-        off += q_rows * pl->cap * 8;
+        pl->spill = spill;
+        off += (spill ? 1 : q_rows) * pl->cap * 8;   // spilled lists: one sort scratch stays here
     }
     pl->off_stage = align_up(off, 128);
     const int fit = std::min(kMaxStages, (idx->smem_optin - pl->off_stage) / pl->stage_bytes);
@@ -463,7 +472,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     ScanPlan pl8;
     // (only where a sample phase is possible: without thresholds nearly every pair passes the filter)
     const long long q8_sample = (std::max<long long>(idx->N / 128, 4LL * idx->num_sms * kTcTileM) + 255) / 256 * 256;
-    const bool use_q8 = idx->x8 && idx->metric == RALM_IP && idx->variant == 0 && s <= kQ8MaxQueries &&
+    const bool use_q8 = idx->x8 && (idx->metric == RALM_IP || idx->norms) && idx->variant == 0 && s <= kQ8MaxQueries &&
                         (idx->x8_force || (idx->tc_thr && idx->tc_two_phase && q8_sample * 32 <= idx->N)) &&
                         plan_scan_q8(idx, s, k, &pl8);
     const int per_pass = use_q8 ? kQ8MaxQueries : mma ? (wide ? wide_pass : kScanMaxQueries) : kFmaQueriesPerPass;
@@ -488,6 +497,9 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
         p.queries = queries + static_cast<size_t>(q0) * idx->d;
         p.norms = idx->norms;
         p.x8 = nullptr;
+        p.sqnorms = nullptr;
+        p.pub = nullptr;
+        p.pub_rank = 0;
         p.spill = pl.spill ? idx->spill : nullptr;
         p.partial = idx->partial;
         p.status = idx->status;
@@ -518,6 +530,11 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             // the same grid whatever the tile height of the pass: the merge reads one list per CTA
             const int g = static_cast<int>(std::min<long long>(idx->num_sms, (end - begin + 15) / 16));
             *grid_out = g;
+            p.pub = (idx->pub && k >= kPubMinK && g > 1) ? idx->pub : nullptr;
+            p.pub_rank = p.pub ? (k + g - 1) / g : 0;
+            if (p.pub && cudaMemsetAsync(idx->pub, 0, sizeof(uint32_t) * idx->num_sms * static_cast<size_t>(idx->max_s), st) !=
+                             cudaSuccess)
+                return cudaErrorUnknown;
             if (mma && idx->metric == RALM_L2 && idx->norms && sp > kScanMaxQueries)
                 return (k == 1) ? launch_scan<true, true, 16, 1, true, true>(p, g, pl.smem_bytes, st)
                                 : launch_scan<true, true, 16, 1, false, true>(p, g, pl.smem_bytes, st);
@@ -543,7 +560,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             ScanParams p8 = p;
             p8.x8 = idx->x8;
             p8.norms = idx->x8_bound;
-            p8.spill = nullptr;
+            p8.sqnorms = idx->norms;
+            p8.spill = pl8.spill ? idx->spill : nullptr;
             p8.cap = pl8.cap;
             p8.soft_limit = pl8.soft_limit;
             p8.tile_rows = pl8.tile_rows;
@@ -559,8 +577,17 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             p8.ntiles = (end - begin + pl8.tile_rows - 1) / pl8.tile_rows;
             const int g = static_cast<int>(std::min<long long>(idx->num_sms, (end - begin + 15) / 16));
             *grid_out = g;
+            p8.pub = (idx->pub && k >= kPubMinK && g > 1) ? idx->pub : nullptr;
+            p8.pub_rank = p8.pub ? (k + g - 1) / g : 0;
+            if (p8.pub && cudaMemsetAsync(idx->pub, 0, sizeof(uint32_t) * idx->num_sms * static_cast<size_t>(idx->max_s), st) !=
+                              cudaSuccess)
+                return cudaErrorUnknown;
             auto kern = (k == 1) ? scan_q8_kernel<true, 1> : scan_q8_kernel<false, 1>;
             if (sp > kScanMaxQueries) kern = (k == 1) ? scan_q8_kernel<true, 2> : scan_q8_kernel<false, 2>;
+            if (idx->metric == RALM_L2) {
+                kern = (k == 1) ? scan_q8_kernel<true, 1, true> : scan_q8_kernel<false, 1, true>;
+                if (sp > kScanMaxQueries) kern = (k == 1) ? scan_q8_kernel<true, 2, true> : scan_q8_kernel<false, 2, true>;
+            }
             cudaError_t ke = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, pl8.smem_bytes);
             if (ke != cudaSuccess) return ke;
             kern<<<g, 32 * (pl8.nwarps + 1), pl8.smem_bytes, st>>>(p8);
@@ -717,6 +744,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->x8_force = false;
     idx->spill = nullptr;
     idx->spill_cap = 0;
+    idx->pub = nullptr;
     cudaError_t first_error = cudaSuccess;
     auto alloc = [&first_error](auto **ptr, size_t bytes) {
         if (first_error == cudaSuccess) first_error = device_alloc(ptr, bytes);
@@ -728,6 +756,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
         idx->spill_cap = std::max(512, 2 * next_pow2(max_k));
         alloc(&idx->spill, sizeof(uint64_t) * idx->num_sms * kScanMaxPassQueries * static_cast<size_t>(idx->spill_cap));
     }
+    if (max_k >= kPubMinK) alloc(&idx->pub, sizeof(uint32_t) * idx->num_sms * static_cast<size_t>(max_s));
     if (metric == RALM_L2 && N > 0) alloc(&idx->norms, sizeof(float) * N);
     ScanPlan probe;
     const bool small_scan_fits = plan_scan(idx, true, kScanMaxQueries, 1, &probe);
@@ -779,6 +808,7 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
     cudaFree(idx->x8);
     cudaFree(idx->x8_bound);
     cudaFree(idx->spill);
+    cudaFree(idx->pub);
     cudaFree(idx->status);
     cudaFree(idx->h_queries);
     cudaFree(idx->h_ids);
@@ -921,7 +951,7 @@ ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant) {
 
 ralm_status_t ralm_index_enable_q8(ralm_index_t *idx, int32_t force) {
     if (!idx) return RALM_ERR_INVALID_ARG;
-    if (idx->metric != RALM_IP || idx->d % 16 != 0) return RALM_ERR_UNSUPPORTED;
+    if (idx->d % 16 != 0 || (idx->metric == RALM_L2 && idx->N > 0 && !idx->norms)) return RALM_ERR_UNSUPPORTED;
     idx->x8_force = force != 0;
     if (idx->x8 || idx->N == 0) return RALM_OK;
     ScanPlan probe;
@@ -933,6 +963,19 @@ ralm_status_t ralm_index_enable_q8(ralm_index_t *idx, int32_t force) {
         cudaGetLastError();
         cudaFree(x8);
         return RALM_ERR_OOM;
+    }
+    if (!idx->spill && idx->max_k > kQ8MaxKWide) {
+        // candidate lists of more than 256 slots live in global memory for this scan
+        const int cap = std::max(512, 2 * next_pow2(idx->max_k));
+        if (device_alloc(&idx->spill, sizeof(uint64_t) * idx->num_sms * kScanMaxPassQueries * static_cast<size_t>(cap)) !=
+            cudaSuccess) {
+            cudaGetLastError();
+            idx->spill = nullptr;
+            cudaFree(x8);
+            cudaFree(bound);
+            return RALM_ERR_OOM;
+        }
+        idx->spill_cap = cap;
     }
     const int blocks = static_cast<int>(std::min<long long>((idx->N + 7) / 8, 32LL * idx->num_sms));
     quantize_rows_kernel<<<blocks, 256>>>(idx->corpus, idx->N, idx->d, x8, bound);
@@ -992,6 +1035,7 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.tc_two_phase = false;
     view.spill = nullptr;
     view.spill_cap = 0;
+    view.pub = nullptr;
     view.norms = nullptr;  // no index, no stored norms: the scan derives them on the tensor cores
     view.x8 = nullptr;
     view.x8_bound = nullptr;

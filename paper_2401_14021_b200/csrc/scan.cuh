@@ -76,6 +76,13 @@ struct ScanParams {
     int off_cand;
     int off_stage;
     float l2_slack;  // warp-MMA L2: filter slack per unit of (|x|^2 + |q|^2)
+    // Large k: thresholds shared between the CTAs of a launch. After every compaction a CTA
+    // publishes, per query, the rank value of its pub_rank-th best row (as order-preserving bits,
+    // 0 = nothing yet) in pub[blockIdx.x * s_total + q_base + q]. pub_rank * gridDim.x >= k, the
+    // CTAs' rows are disjoint, so the lowest published value of a query is reached by k different
+    // rows, and every CTA may raise its threshold to it. Null: off.
+    uint32_t *pub;
+    int pub_rank;
 };
 
 struct ScanHeader {
@@ -94,8 +101,13 @@ static_assert(sizeof(ScanHeader) <= kScanHeaderBytes, "header too large");
 // Sort query q's candidates, keep the best k, raise the threshold. Called by a group of
 // `nthr` threads with ranks `tid`, synchronised through group_sync(bar_id). With a scratch
 // area the list (which then lives in global memory) is sorted there and its head copied back.
+struct PubCtx {
+    uint32_t *mine;   // this CTA's row of published values (indexed by the pass's query), or null
+    int rank;         // which of its best rows a CTA publishes
+};
+
 __device__ inline void compact_query(ScanHeader *hdr, uint64_t *cand, uint64_t *scratch, int cap, int q,
-                                     int k, int tid, int nthr, int bar_id) {
+                                     int k, int tid, int nthr, int bar_id, PubCtx pub = PubCtx{nullptr, 0}) {
     uint64_t *list = cand + static_cast<size_t>(q) * cap;
     uint64_t *a = scratch ? scratch : list;
     const int n = hdr->cnt[q] < cap ? hdr->cnt[q] : cap;  // (cap: see push_candidate)
@@ -113,16 +125,37 @@ __device__ inline void compact_query(ScanHeader *hdr, uint64_t *cand, uint64_t *
     }
     if (tid == 0) {
         hdr->cnt[q] = n < k ? n : k;
-        hdr->thr[q] = (n >= k) ? key_value(a[k - 1]) : -INFINITY;
+        // (never below a threshold taken over from the other CTAs)
+        const float kth = (n >= k) ? key_value(a[k - 1]) : -INFINITY;
+        hdr->thr[q] = fmaxf(hdr->thr[q], kth);
+        if (pub.mine && n >= pub.rank)
+            *reinterpret_cast<volatile uint32_t *>(pub.mine + q) = ordered_bits(key_value(a[pub.rank - 1]));
     }
     group_sync(bar_id, nthr);
+}
+
+// Large k: raise every query's threshold to the lowest value the CTAs of the launch have
+// published for it (see ScanParams::pub), once all of them have published one. Called by one
+// warp between the barriers of a compaction meeting.
+__device__ inline void adopt_published_thresholds(ScanHeader *hdr, const uint32_t *pub, int nblocks, int s_total,
+                                                  int q_base, int s, int lane) {
+    for (int q = 0; q < s; ++q) {
+        uint32_t lowest = 0xFFFFFFFFu;
+        for (int c = lane; c < nblocks; c += 32) {
+            const uint32_t v = __ldcg(pub + static_cast<size_t>(c) * s_total + q_base + q);
+            lowest = v < lowest ? v : lowest;
+        }
+        lowest = __reduce_min_sync(0xffffffffu, lowest);
+        if (lane == 0 && lowest != 0u) hdr->thr[q] = fmaxf(hdr->thr[q], from_ordered_bits(lowest));
+    }
+    __syncwarp();
 }
 
 // All W consumer warps (this one is w) compact every query that holds more than `min_count`
 // candidates; the queries are spread over groups of warps that sort in parallel. Must be
 // called by all W * 32 consumer threads, with no push in flight.
 __device__ inline void compact_all(ScanHeader *hdr, uint64_t *cand, uint64_t *scratch, int cap, int s,
-                                   int k, int min_count, int w, int lane, int W) {
+                                   int k, int min_count, int w, int lane, int W, PubCtx pub = PubCtx{nullptr, 0}) {
     int list[kScanMaxPassQueries];
     int nq = 0;
 #pragma unroll
@@ -143,16 +176,22 @@ __device__ inline void compact_all(ScanHeader *hdr, uint64_t *cand, uint64_t *sc
 #pragma unroll
         for (int j = 0; j < kScanMaxPassQueries; ++j)
             if (j == i) q = list[j];
-        compact_query(hdr, cand, scratch, cap, q, k, tid, G * 32, bar_id);
+        compact_query(hdr, cand, scratch, cap, q, k, tid, G * 32, bar_id, pub);
     }
 }
 
 // The meeting itself: barrier, compact, lower the flag, barrier.
 __device__ __forceinline__ void compaction_meeting(ScanHeader *hdr, uint64_t *cand, uint64_t *scratch,
                                                    const int cap, const int s, const int k, int w,
-                                                   int lane, int W) {
+                                                   int lane, int W, const ScanParams &p) {
     named_barrier(1, W * 32);
-    compact_all(hdr, cand, scratch, cap, s, k, k, w, lane, W);
+    PubCtx pub{p.pub ? p.pub + static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base : nullptr, p.pub_rank};
+    // (with shared thresholds every list that can already publish is sorted, not only the full ones)
+    compact_all(hdr, cand, scratch, cap, s, k, p.pub ? p.pub_rank - 1 : k, w, lane, W, pub);
+    if (p.pub) {
+        named_barrier(1, W * 32);   // every compaction of this meeting has written its threshold
+        if (w == 0) adopt_published_thresholds(hdr, p.pub, gridDim.x, p.s_total, p.q_base, s, lane);
+    }
     if (w == 0 && lane == 0) *reinterpret_cast<volatile int *>(&hdr->flag) = 0;
     named_barrier(1, W * 32);
 }
@@ -403,8 +442,15 @@ scan_kernel(const ScanParams p) {
         long long row0 =
             p.row_begin + (static_cast<long long>(blockIdx.x) + static_cast<long long>(w) * gridDim.x) * T;
         const long long row_step = static_cast<long long>(gridDim.x) * W * T;
+        // shared thresholds (large k): lists fill too slowly to call meetings by themselves, so the
+        // first consumer warp calls one after 64, 128, 256, ... of its tiles
+        long long tiles_done = 0, next_meeting = 64;
         for (long long it = w; it < my_tiles; it += W, row0 += row_step) {
             if (*abort_flag) continue;
+            if (!TOP1 && p.pub && w == 0 && ++tiles_done == next_meeting) {
+                next_meeting *= 2;
+                if (lane == 0) *compact_flag = 1;
+            }
             // this warp's private ring: only this warp ever waits on these stages, in order,
             // so a parity wait can never be satisfied by an older phase
             const int st = w + slot * W;
@@ -438,7 +484,7 @@ scan_kernel(const ScanParams p) {
                         while (!mbar_try_wait(full_bar, my_parity)) {}  // completed: returns at once
                         have_tile = true;
                     } else if (state == 2) {
-                        compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W);
+                        compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W, p);
                     } else if (state == 3) {
                         if (lane == 0) {
                             atomicMax(p.status, kStatusTimeout);
@@ -699,7 +745,7 @@ scan_kernel(const ScanParams p) {
                     }
                 }
                 state = __shfl_sync(0xffffffffu, state, 0);
-                if (state == 1) compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W);
+                if (state == 1) compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W, p);
                 else if (state == 2) break;
             }
             named_barrier(1, cthreads);

@@ -98,51 +98,48 @@ quantize_rows_kernel(const __half *__restrict__ corpus, long long N, int d, uint
     }
 }
 
-// Exact inner product of one fp16 corpus row (global memory) with one staged query, by the
-// whole warp. The staged query has every group of four elements stored as (e0, e2, e1, e3).
-__device__ __forceinline__ float warp_exact_ip(const __half *row, uint32_t q_addr, int d, int lane) {
+// One fp16 corpus row (global memory) against one staged query, by the whole warp: the exact
+// inner product, or for L2 the squared distance in the direct sum-of-squared-differences form.
+// The staged query has every group of four elements stored as (e0, e2, e1, e3). The row is not
+// in any cache (only its one-byte copy was streamed), so the loads of four steps are issued
+// together: one DRAM latency per 1024 elements instead of four.
+template <bool L2>
+__device__ __forceinline__ float warp_exact_score(const __half *row, uint32_t q_addr, int d, int lane) {
     float2 sum = make_float2(0.f, 0.f);
     const uint4 *src = reinterpret_cast<const uint4 *>(row);
-    for (int piece = lane; piece * 8 < d; piece += 32) {
-        const uint4 xr = __ldg(src + piece);
-        const uint4 qr = lds128(q_addr + piece * 16);
-        const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
-        const uint32_t qw[4] = {qr.x, qr.y, qr.z, qr.w};
+    const int pieces = d >> 3;
+    for (int base = 0; base < pieces; base += 128) {
+        uint4 xr[4];
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const float2 x01 = h2_to_f2(xw[2 * e]), x23 = h2_to_f2(xw[2 * e + 1]);
-            const float2 q02 = h2_to_f2(qw[2 * e]), q13 = h2_to_f2(qw[2 * e + 1]);
-            sum.x = fmaf(x01.x, q02.x, sum.x);
-            sum.y = fmaf(x01.y, q13.x, sum.y);
-            sum.x = fmaf(x23.x, q02.y, sum.x);
-            sum.y = fmaf(x23.y, q13.y, sum.y);
+        for (int u = 0; u < 4; ++u) {
+            const int piece = base + u * 32 + lane;
+            xr[u] = piece < pieces ? __ldg(src + piece) : make_uint4(0, 0, 0, 0);
         }
-    }
-    float v = sum.x + sum.y;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-
-// Squared distance between one fp16 corpus row (global memory) and one staged query (stored in
-// the same (e0, e2, e1, e3) order), by the whole warp, in the direct form.
-__device__ __forceinline__ float warp_exact_l2(const __half *row, uint32_t q_addr, int d, int lane) {
-    float2 sum = make_float2(0.f, 0.f);
-    const uint4 *src = reinterpret_cast<const uint4 *>(row);
-    for (int piece = lane; piece * 8 < d; piece += 32) {
-        const uint4 xr = __ldg(src + piece);
-        const uint4 qr = lds128(q_addr + piece * 16);
-        const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
-        const uint32_t qw[4] = {qr.x, qr.y, qr.z, qr.w};
+        for (int u = 0; u < 4; ++u) {
+            const int piece = base + u * 32 + lane;
+            if (piece < pieces) {
+                const uint4 qr = lds128(q_addr + piece * 16);
+                const uint32_t xw[4] = {xr[u].x, xr[u].y, xr[u].z, xr[u].w};
+                const uint32_t qw[4] = {qr.x, qr.y, qr.z, qr.w};
 #pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const float2 x01 = h2_to_f2(xw[2 * e]), x23 = h2_to_f2(xw[2 * e + 1]);
-            const float2 q02 = h2_to_f2(qw[2 * e]), q13 = h2_to_f2(qw[2 * e + 1]);
-            const float d0 = x01.x - q02.x, d1 = x01.y - q13.x, d2 = x23.x - q02.y, d3 = x23.y - q13.y;
-            sum.x = fmaf(d0, d0, sum.x);
-            sum.y = fmaf(d1, d1, sum.y);
-            sum.x = fmaf(d2, d2, sum.x);
-            sum.y = fmaf(d3, d3, sum.y);
+                for (int e = 0; e < 2; ++e) {
+                    const float2 x01 = h2_to_f2(xw[2 * e]), x23 = h2_to_f2(xw[2 * e + 1]);
+                    const float2 q02 = h2_to_f2(qw[2 * e]), q13 = h2_to_f2(qw[2 * e + 1]);
+                    if (L2) {
+                        const float d0 = x01.x - q02.x, d1 = x01.y - q13.x, d2 = x23.x - q02.y, d3 = x23.y - q13.y;
+                        sum.x = fmaf(d0, d0, sum.x);
+                        sum.y = fmaf(d1, d1, sum.y);
+                        sum.x = fmaf(d2, d2, sum.x);
+                        sum.y = fmaf(d3, d3, sum.y);
+                    } else {
+                        sum.x = fmaf(x01.x, q02.x, sum.x);
+                        sum.y = fmaf(x01.y, q13.x, sum.y);
+                        sum.x = fmaf(x23.x, q02.y, sum.x);
+                        sum.y = fmaf(x23.y, q13.y, sum.y);
+                    }
+                }
+            }
         }
     }
     float v = sum.x + sum.y;
@@ -277,6 +274,7 @@ scan_q8_kernel(const ScanParams p) {
             if (L2 && row0 + ph_lo < p.N) n_lo_next = __ldg(p.sqnorms + row0 + ph_lo);
             if (L2 && row0 + ph_hi < p.N) n_hi_next = __ldg(p.sqnorms + row0 + ph_hi);
         }
+        long long tiles_done = 0, next_meeting = 64;
         for (long long it = w; it < my_tiles; it += W, row0 += row_step) {
             const float e_lo = e_lo_next, e_hi = e_hi_next, n_lo = n_lo_next, n_hi = n_hi_next;
             e_lo_next = e_hi_next = n_lo_next = n_hi_next = 0.f;
@@ -288,6 +286,11 @@ scan_q8_kernel(const ScanParams p) {
                 if (L2 && nrow + ph_hi < p.N) n_hi_next = __ldg(p.sqnorms + nrow + ph_hi);
             }
             if (*abort_flag) continue;
+            // (shared thresholds, large k: meetings after 64, 128, 256, ... tiles, as in scan_kernel)
+            if (!TOP1 && p.pub && w == 0 && ++tiles_done == next_meeting) {
+                next_meeting *= 2;
+                if (lane == 0) *compact_flag = 1;
+            }
             const int st = w + slot * W;
             const int cur_slot = slot;
             const uint32_t full_bar = smem_u32(&hdr->full[st]);
@@ -312,7 +315,7 @@ scan_q8_kernel(const ScanParams p) {
                         while (!mbar_try_wait(full_bar, my_parity)) {}  // completed: returns at once
                         have_tile = true;
                     } else if (state == 2) {
-                        compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W);
+                        compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W, p);
                     } else if (state == 3) {
                         if (lane == 0) {
                             atomicMax(p.status, kStatusTimeout);
@@ -453,8 +456,8 @@ scan_q8_kernel(const ScanParams p) {
                         const int row_local = q8_phys_row((src >> 2) + ((i & 2) ? 8 : 0));
                         const int q = grp * kScanMaxQueries + 2 * (src & 3) + (i & 1);
                         const long long row = row0 + row_local;
-                        const float val = L2 ? 0.0f - warp_exact_l2(p.corpus + row * d, q_base_addr + q * q_pitch, d, lane)
-                                             : warp_exact_ip(p.corpus + row * d, q_base_addr + q * q_pitch, d, lane);
+                        const float exact = warp_exact_score<L2>(p.corpus + row * d, q_base_addr + q * q_pitch, d, lane);
+                        const float val = L2 ? 0.0f - exact : exact;
                         if (lane == 0) {
                             const uint64_t key = make_key(val, static_cast<uint32_t>(row));
                             if (TOP1) {
@@ -497,7 +500,7 @@ scan_q8_kernel(const ScanParams p) {
                     }
                 }
                 state = __shfl_sync(0xffffffffu, state, 0);
-                if (state == 1) compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W);
+                if (state == 1) compaction_meeting(hdr, cand, scratch, p.cap, p.s, p.k, w, lane, W, p);
                 else if (state == 2) break;
             }
             named_barrier(1, cthreads);

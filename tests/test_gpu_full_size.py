@@ -270,6 +270,21 @@ def test_c4_full_size_l2_k1024():
     assert ids[:, 0].tolist() == src.tolist()
     counts, n_sub = _sampled_parity(x, q, ids, scores, oracle.L2, 1024, 14, 16_384, seed=3400)
     print("C4: %s over a %d-row sub-corpus" % (counts, n_sub))
+    # the same search through the 8-bit filter copy (51 GB more): identical neighbours, distances
+    # from the same direct form
+    free, _ = torch.cuda.mem_get_info()
+    if free > c.N * c.d + (6 << 30):
+        idx.enable_q8()
+        ids8, scores8 = ralm.search(idx, q, 1024)
+        torch.cuda.synchronize()
+        assert idx.device_status() == 0
+        assert idx.last_dispatch()["kernel_name"] == "scan_q8_kernel"
+        counts8, n_sub = _sampled_parity(x, q, ids8, scores8, oracle.L2, 1024, 14, 16_384, seed=3401)
+        print("C4 8-bit scan: %s over a %d-row sub-corpus" % (counts8, n_sub))
+        assert torch.equal(ids8[:, 0], ids[:, 0])
+        torch.testing.assert_close(scores8, scores, rtol=1e-5, atol=1e-4)
+    else:
+        print("C4 8-bit scan: skipped, %.0f GB free" % (free / 1e9))
     idx.close()
     # 64 concurrent queries, k = 20: L2 on the large-batch scan (lower-bound sample, filter, rescoring)
     q64, src64 = workloads.noisy_copy_queries(x, 64, workloads.seed_for(4, "queries") + 5)

@@ -16,9 +16,9 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def _search(x, q, k, q8):
+def _search(x, q, k, q8, metric=oracle.IP):
     import paper_2401_14021_b200 as ralm
-    idx = ralm.Index(x, oracle.IP, max_s=max(1, q.shape[0]), max_k=k)
+    idx = ralm.Index(x, metric, max_s=max(1, q.shape[0]), max_k=k)
     if q8:
         # (forced: most of these corpora are too small for the sample phase, without which the
         # library would keep the fp16 scan)
@@ -128,13 +128,55 @@ def test_q8_is_refused_where_it_does_not_apply_and_falls_back_where_it_cannot_se
         idx.enable_q8()
     idx.close()
     x = workloads.integer_valued((500, 32), seed=1501, lo=-3, hi=3, device=DEV)
-    idx = ralm.Index(x, oracle.L2, max_s=4, max_k=4)      # the filter is an inner-product bound
-    with pytest.raises(ralm.RalmError):
-        idx.enable_q8()
-    idx.close()
-    # k beyond the 8-bit scan's limits (256 up to 8 queries, 64 up to 16) and batches of more than
-    # 16 queries take the fp16 scans
+    # k beyond the 8-bit scan's limits (up to 8 queries: 256, more where the index keeps its lists in
+    # global memory; 9..16 queries: 64) and batches of more than 16 queries take the fp16 scans
     q = workloads.integer_valued((20, 32), seed=1502, lo=-3, hi=3, device=DEV)
     for s, k in ((4, 300), (12, 65), (20, 5)):
         ids, scores, _ = _search(x, q[:s].contiguous(), k, q8=True)
         check_search(ids, scores, x.cpu().numpy(), q[:s].cpu().numpy(), oracle.IP, k, exact=True)
+
+
+# ---- L2 (the KNN-LM datastore's metric): the same filter on x.q bounds the squared distance from
+# below; what passes is scored again in the direct form. Integer rows: distances are exact
+# integers, ties abound, ids and distances must equal the oracle's bit for bit, also with lists
+# that live in global memory (k > 256) and with planted zero-distance copies.
+@pytest.mark.parametrize("N,d,s,k", [(1, 16, 1, 1), (17, 64, 8, 1), (33, 48, 2, 40), (5000, 768, 4, 5),
+                                     (3001, 1024, 4, 1024), (40_000, 208, 8, 300), (100_003, 768, 8, 1),
+                                     (2_500_000, 64, 8, 20), (2_450_001, 32, 3, 600), (5000, 768, 16, 5),
+                                     (2_450_000, 32, 13, 20)])
+def test_q8_l2_integer_inputs_are_bit_exact(N, d, s, k):
+    x = workloads.integer_valued((N, d), seed=1500 + N % 1000 + d, lo=-20, hi=20, device=DEV)
+    q = workloads.integer_valued((s, d), seed=1600 + N % 1000 + d, lo=-20, hi=20, device=DEV)
+    if N > s:
+        q[0] = x[N // 2]                       # an exact copy: distance 0, ranked first
+    ids, scores, _ = _search(x, q, k, q8=True, metric=oracle.L2)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, k, exact=True)
+
+
+@pytest.mark.parametrize("N,d,s,k", [(120_001, 1024, 4, 1024), (2_450_000, 128, 8, 1), (2_450_000, 128, 4, 20),
+                                     (2_450_000, 128, 16, 20)])
+def test_q8_l2_unnormalised_rows_match_the_oracle_and_the_fp16_scan(N, d, s, k):
+    """Rows shaped like the KNN-LM keys (mixture, unnormalised, log-normal norms): the band rule
+    against the oracle, the planted source first, and the fp16 L2 scan's ranking and distances."""
+    x, _ = workloads.mixture_corpus(N, d, 256, seed=1700 + d, device=DEV, normalise=False, lognormal_sigma=0.3)
+    q, src = workloads.noisy_copy_queries(x, s, seed=1701 + d)
+    ids, scores, launches = _search(x, q, k, q8=True, metric=oracle.L2)
+    counts = check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, k)
+    assert counts.wide == 0, str(counts)
+    assert ids[:, 0].tolist() == src.tolist()
+    ids16, scores16, _ = _search(x, q, k, q8=False, metric=oracle.L2)
+    assert torch.equal(ids[:, 0], ids16[:, 0])
+    torch.testing.assert_close(scores, scores16, rtol=1e-5, atol=1e-5)
+
+
+def test_q8_l2_dispatch_is_the_8bit_scan():
+    import paper_2401_14021_b200 as ralm
+    x, _ = workloads.mixture_corpus(50_000, 128, 64, seed=1800, device=DEV, normalise=False, lognormal_sigma=0.3)
+    q, _ = workloads.noisy_copy_queries(x, 4, seed=1801)
+    idx = ralm.Index(x, oracle.L2, max_s=4, max_k=8)
+    ralm.search(idx, q, 8)
+    assert idx.last_dispatch()["kernel"] == 2          # the fp16 warp-MMA scan
+    idx.enable_q8(force=True)
+    ralm.search(idx, q, 8)
+    assert idx.last_dispatch()["kernel_name"] == "scan_q8_kernel"
+    idx.close()
