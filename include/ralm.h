@@ -76,7 +76,7 @@ typedef enum {
  * buffers, a status word; for L2 the squared norm of every row (4 N bytes, computed here in one
  * pass over the corpus); for max_k > 256 spilled candidate lists (about 19 MB at k = 1024); for
  * max_s >= 9 the candidate lists of the large-batch scan (about 300 KB per query, 155 MB at 512
- * queries). Synchronous.
+ * queries; twice that for max_k > 64). Synchronous.
  * Errors: INVALID_ARG (null pointer, misaligned corpus, bad sizes), OOM, CUDA,
  * UNSUPPORTED (device is not compute capability 10.x). */
 ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_metric_t metric,
@@ -202,7 +202,7 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
 /* Pin the scan variant used by ralm_search on this index (benchmarking aid).
  *   0 = automatic, 1 = FMA scan (fp32 FMAs, d <= 1024, 4 queries per pass), 2 = warp-MMA scan
  *   (8 queries per pass, 16 for larger batches, 32 for inner product; for L2 the tensor-core
- *   value only filters and the ranked distance is the direct sum of squared differences), 3 = tcgen05 scan (up to 512 queries per pass, k <= 64,
+ *   value only filters and the ranked distance is the direct sum of squared differences), 3 = tcgen05 scan (up to 512 queries per pass, k <= 256,
  *   d >= 64; pairs of CTAs share each MMA; for L2 the tensor-core value again only filters,
  *   and the corpus must be large enough to scan a sample first, about 600 K rows), 4 = tcgen05
  *   scan with single CTAs. Automatic: warp-MMA up to 32 queries (inner product) or 16 (L2), the

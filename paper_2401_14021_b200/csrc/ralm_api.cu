@@ -43,8 +43,8 @@ struct ralm_index {
     float *tc_gmax;        // tcgen05 scan, sample launch: [num_sms * 4][max_s] maxima per selection warp
     bool tc_two_phase;     // sample phase enabled (tuning aid)
     int tc_clusters;       // CTA pairs the device runs at once (-1 = not asked yet)
-    uint64_t *tc_cand;     // tcgen05 scan: [num_sms][tc_cand_q][kTcCap] candidate lists, or null
-    int tc_cand_q;
+    uint64_t *tc_cand;     // tcgen05 scan: [num_sms][tc_cand_q][tc_cand_cap] candidate lists, or null
+    int tc_cand_q, tc_cand_cap;
     int *status;
     // staging for the host-buffer entry point
     __half *h_queries;
@@ -273,6 +273,7 @@ bool encode_rows_map(CUtensorMap *map, const void *base, long long rows, int d, 
 
 bool tc_can_serve(const ralm_index *idx, int k) {
     return (idx->metric == RALM_IP || idx->norms != nullptr) && idx->tc_cand != nullptr && k <= kTcMaxK &&
+           (k <= kTcSmallK || idx->tc_cand_cap >= kTcCapLarge) &&
            idx->d >= kTcChunkK;
 }
 
@@ -281,7 +282,8 @@ bool alloc_tc_workspace(ralm_index *idx, int queries) {
     if (idx->tc_cand) cudaFree(idx->tc_cand);
     idx->tc_cand = nullptr;
     idx->tc_cand_q = 0;
-    const size_t bytes = sizeof(uint64_t) * idx->num_sms * static_cast<size_t>(queries) * kTcCap;
+    const int cap = idx->max_k > kTcSmallK ? kTcCapLarge : kTcCapSmall;
+    const size_t bytes = sizeof(uint64_t) * idx->num_sms * static_cast<size_t>(queries) * cap;
     if (!idx->tc_thr && device_alloc(&idx->tc_thr, sizeof(float) * idx->max_s) != cudaSuccess) {
         idx->tc_thr = nullptr;
         return false;
@@ -296,6 +298,7 @@ bool alloc_tc_workspace(ralm_index *idx, int queries) {
         return false;
     }
     idx->tc_cand_q = queries;
+    idx->tc_cand_cap = cap;
     return true;
 }
 
@@ -308,6 +311,9 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
     p.partial = idx->partial;
     p.cand = idx->tc_cand;
     p.cand_q = idx->tc_cand_q;
+    // (lists of 256 slots whenever k allows, also in a workspace sized for more)
+    p.cap = k > kTcSmallK ? kTcCapLarge : kTcCapSmall;
+    p.soft = k > kTcSmallK ? kTcSoftLarge : kTcSoftSmall;
     p.status = idx->status;
     p.N = row_end;
     p.thr_init = thr_init;
@@ -734,6 +740,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     const size_t sk = static_cast<size_t>(max_s) * max_k;
     idx->tc_cand = nullptr;
     idx->tc_cand_q = 0;
+    idx->tc_cand_cap = 0;
     idx->tc_clusters = -1;
     idx->tc_thr = nullptr;
     idx->tc_gmax = nullptr;
@@ -1029,6 +1036,7 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.cache_keys = nullptr;
     view.tc_cand = nullptr;
     view.tc_cand_q = 0;
+    view.tc_cand_cap = 0;
     view.tc_clusters = -1;
     view.tc_thr = nullptr;
     view.tc_gmax = nullptr;

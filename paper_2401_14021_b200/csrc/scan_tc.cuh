@@ -55,16 +55,18 @@ constexpr int kTcChunkK = 64;    // fp16 per K chunk (128 bytes: one swizzle spa
 constexpr int kTcMaxQueries = 2 * kTcMaxN;
 constexpr int kTcABytes = kTcTileM * kTcChunkK * 2;
 constexpr int kTcMaxStages = 12;
-constexpr int kTcCap = 256;      // candidate slots per (CTA, query)
-constexpr int kTcSoft = 120;     // a list holding this many is compacted before the next unit (at most
-                                 // 128 more arrive in a unit; just under 128 so that the usual sort is
-                                 // one of 128 keys)
-constexpr int kTcMaxK = 64;      // k <= about kTcSoft / 2 keeps compactions rare
+// Candidate lists per (CTA, query): `cap` slots; a list holding `soft` keys or more is compacted
+// before the next unit, in which at most 128 more arrive (soft + 128 <= cap). k <= 64: 256 slots
+// and soft 120, just under 128 so that the usual sort is one of 128 keys; k <= 256: 512 slots.
+constexpr int kTcCapSmall = 256, kTcSoftSmall = 120, kTcSmallK = 64;
+constexpr int kTcCapLarge = 512, kTcSoftLarge = 380;
+constexpr int kTcMaxK = 256;
 constexpr int kTcTmemCols = 512;
 
 struct TcParams {
     uint64_t *partial;  // [gridDim.x][s_total][k] sorted keys, 0 = empty
-    uint64_t *cand;     // [gridDim.x][cand_q][kTcCap] candidate lists
+    uint64_t *cand;     // [gridDim.x][cand_q][cap] candidate lists
+    int cap, soft;      // slots per list; fill level that asks for a compaction (see kTcCapSmall)
     int *status;
     long long N;        // rows of this launch end here (the whole corpus, or the end of a sample)
     long long tile0;    // first row tile (of 128 rows, 256 for pairs) of this launch
@@ -113,7 +115,7 @@ struct TcHeader {
     uint64_t drain;
     uint32_t tmem_base;
     int abort;
-    int dirty[3];  // [u % 3]: some candidate list reached kTcSoft during unit u
+    int dirty[3];  // [u % 3]: some candidate list reached the soft limit during unit u
 };
 constexpr int kTcHeaderBytes = 512;
 static_assert(sizeof(TcHeader) <= kTcHeaderBytes, "header too large");
@@ -269,30 +271,29 @@ __device__ __forceinline__ void tc_compact_sorted(uint64_t *list, float *thr, in
 }
 
 __device__ __forceinline__ void tc_compact_query(uint64_t *list, float *thr, int *cnt, int *sorted, int q,
-                                                 int k, int lane) {
-    const int n = cnt[q] < kTcCap ? cnt[q] : kTcCap;  // (the cap: see tc_append_octet)
+                                                 int k, int cap, int lane) {
+    const int n = cnt[q] < cap ? cnt[q] : cap;  // (the cap: see tc_append_octet)
     if (n <= 32) tc_compact_sorted<1>(list, thr, cnt, sorted, q, n, k, lane);
     else if (n <= 64) tc_compact_sorted<2>(list, thr, cnt, sorted, q, n, k, lane);
     else if (n <= 128) tc_compact_sorted<4>(list, thr, cnt, sorted, q, n, k, lane);
-    else tc_compact_sorted<8>(list, thr, cnt, sorted, q, n, k, lane);
+    else if (n <= 256) tc_compact_sorted<8>(list, thr, cnt, sorted, q, n, k, lane);
+    else tc_compact_sorted<16>(list, thr, cnt, sorted, q, n, k, lane);
 }
 
 // Appending itself: every row (lane) whose bit b of `hit` is set stores key(v[b], row) in column
 // b's list. Only columns with a hit anywhere in the warp are visited (a warp-uniform branch per
 // column); each hit reserves its slot with its own shared-memory atomic.
 __device__ __forceinline__ void tc_store_hits(const uint32_t (&v)[32], uint32_t hit, int *cnt_chunk,
-                                              uint64_t *cand_chunk, uint32_t row, volatile int *dirty, int *status) {
+                                              uint64_t *cand_chunk, uint32_t row, volatile int *dirty, int *status, int cap,
+                                              int soft) {
     const uint32_t any_col = __reduce_or_sync(0xffffffffu, hit);
 #pragma unroll
     for (int b = 0; b < 32; ++b) {
         if (any_col & (1u << b)) {
             if ((hit >> b) & 1u) {
                 const int slot = atomicAdd(&cnt_chunk[b], 1);
-                if (slot + 1 >= kTcSoft) *dirty = 1;
-                // (a list holds fewer than kTcSoft keys when a unit starts and gains at most 128 in
-                // one, so slot < kTcCap; should that ever fail the key is dropped and the status
-                // word says so, rather than writing into the neighbouring list)
-                if (slot < kTcCap) cand_chunk[static_cast<size_t>(b) * kTcCap + slot] = make_key(__uint_as_float(v[b]), row);
+                if (slot + 1 >= soft) *dirty = 1;
+                if (slot < cap) cand_chunk[static_cast<size_t>(b) * cap + slot] = make_key(__uint_as_float(v[b]), row);
                 else atomicMax(status, kStatusInternal);
             }
         }
@@ -308,19 +309,19 @@ __device__ __forceinline__ void tc_store_hits(const uint32_t (&v)[32], uint32_t 
 __device__ __noinline__ void tc_append_octet(uint32_t v0, uint32_t v1, uint32_t v2, uint32_t v3, uint32_t v4,
                                              uint32_t v5, uint32_t v6, uint32_t v7, int c0, float thr_lane,
                                              int *cnt_block, uint64_t *cand_block, uint32_t row, bool row_ok,
-                                             volatile int *dirty, int *status) {
+                                             volatile int *dirty, int *status, int cap, int soft) {
     const uint32_t v[8] = {v0, v1, v2, v3, v4, v5, v6, v7};
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const float t = __shfl_sync(0xffffffffu, thr_lane, c0 + i);
         if (row_ok && __uint_as_float(v[i]) >= t) {
             const int slot = atomicAdd(&cnt_block[c0 + i], 1);
-            if (slot + 1 >= kTcSoft) *dirty = 1;
-            // (a list holds fewer than kTcSoft keys when a unit starts and gains at most 128 in
-            // one, so slot < kTcCap; should that ever fail the key is dropped and the status
+            if (slot + 1 >= soft) *dirty = 1;
+            // (a list holds fewer than `soft` keys when a unit starts and gains at most 128 in
+            // one, so slot < cap; should that ever fail the key is dropped and the status
             // word says so, rather than writing into the neighbouring list)
-            if (slot < kTcCap)
-                cand_block[static_cast<size_t>(c0 + i) * kTcCap + slot] = make_key(__uint_as_float(v[i]), row);
+            if (slot < cap)
+                cand_block[static_cast<size_t>(c0 + i) * cap + slot] = make_key(__uint_as_float(v[i]), row);
             else
                 atomicMax(status, kStatusInternal);
         }
@@ -358,7 +359,7 @@ __device__ __noinline__ void tc_append_chunk_l2(uint32_t taddr, const float *thr
                                                 int *cnt_chunk, uint64_t *cand_chunk, uint32_t row, bool row_ok,
                                                 float nx, float slack, const __half *corpus,
                                                 const __half *queries_chunk, int d, volatile int *dirty,
-                                                int *status, int lane) {
+                                                int *status, int cap, int soft, int lane) {
     uint32_t v[32];
     tmem_ld32(taddr, v);
     uint32_t hit = 0;
@@ -388,7 +389,7 @@ __device__ __noinline__ void tc_append_chunk_l2(uint32_t taddr, const float *thr
             }
         }
     }
-    tc_store_hits(v, hit, cnt_chunk, cand_chunk, row, dirty, status);
+    tc_store_hits(v, hit, cnt_chunk, cand_chunk, row, dirty, status, cap, soft);
 }
 
 // One block of 32 queries of a sample launch: for every column the best rank value among this
@@ -698,7 +699,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         // ------------------------------------------------------------------ selection
         const int ew = warp - 2;        // 0..3
         const int quarter = warp & 3;   // the TMEM lanes this warp may read: 32 * quarter ..
-        uint64_t *my_cand = p.cand + static_cast<size_t>(blockIdx.x) * p.cand_q * kTcCap;
+        uint64_t *my_cand = p.cand + static_cast<size_t>(blockIdx.x) * p.cand_q * p.cap;
         constexpr bool sample = MODE == 1 || MODE == 3;
         constexpr bool l2 = MODE == 1 || MODE == 2;
         bool ok = true;
@@ -778,9 +779,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                             }
                             if (__any_sync(0xffffffffu, row_ok && (p0 | p1)))
                                 tc_append_chunk_l2(t_row + j * 32, thr + qb + j * 32, qn + qb + j * 32, cnt + qb + j * 32,
-                                                   my_cand + static_cast<size_t>(qb + j * 32) * kTcCap,
+                                                   my_cand + static_cast<size_t>(qb + j * 32) * p.cap,
                                                    static_cast<uint32_t>(row), row_ok, nx, p.slack, p.corpus,
-                                                   p.queries + static_cast<size_t>(qb + j * 32) * p.d, p.d, dirty, p.status, lane);
+                                                   p.queries + static_cast<size_t>(qb + j * 32) * p.d, p.d, dirty, p.status, p.cap, p.soft, lane);
                         } else {
                             // common case: nothing passes. Four independent predicate chains, one per
                             // eight columns, so that the rare case only revisits the eight it concerns.
@@ -795,20 +796,20 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                             }
                             if (__any_sync(0xffffffffu, row_ok && (p0 | p1 | p2 | p3))) {
                                 int *cnt_block = cnt + qb + j * 32;
-                                uint64_t *cand_block = my_cand + static_cast<size_t>(qb + j * 32) * kTcCap;
+                                uint64_t *cand_block = my_cand + static_cast<size_t>(qb + j * 32) * p.cap;
                                 const uint32_t r32 = static_cast<uint32_t>(row);
                                 if (__any_sync(0xffffffffu, row_ok && p0))
                                     tc_append_octet(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], 0, my_thr, cnt_block,
-                                                    cand_block, r32, row_ok, dirty, p.status);
+                                                    cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft);
                                 if (__any_sync(0xffffffffu, row_ok && p1))
                                     tc_append_octet(v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15], 8, my_thr,
-                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status);
+                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft);
                                 if (__any_sync(0xffffffffu, row_ok && p2))
                                     tc_append_octet(v[16], v[17], v[18], v[19], v[20], v[21], v[22], v[23], 16, my_thr,
-                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status);
+                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft);
                                 if (__any_sync(0xffffffffu, row_ok && p3))
                                     tc_append_octet(v[24], v[25], v[26], v[27], v[28], v[29], v[30], v[31], 24, my_thr,
-                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status);
+                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft);
                             }
                         }
                     }
@@ -833,12 +834,12 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             if (need) {
                 for (int base = 0; base < p.s; base += 128) {
                     const int q = base + ew * 32 + lane;
-                    unsigned m = __ballot_sync(0xffffffffu, q < p.s && cnt[q] >= kTcSoft);
+                    unsigned m = __ballot_sync(0xffffffffu, q < p.s && cnt[q] >= p.soft);
                     while (m) {
                         const int b = __ffs(m) - 1;
                         m &= m - 1;
                         const int qq = base + ew * 32 + b;
-                        tc_compact_query(my_cand + static_cast<size_t>(qq) * kTcCap, thr, cnt, sorted, qq, p.k, lane);
+                        tc_compact_query(my_cand + static_cast<size_t>(qq) * p.cap, thr, cnt, sorted, qq, p.k, p.cap, lane);
                     }
                 }
                 named_barrier(1, 128);  // thresholds and counts settled before the next unit's pushes
@@ -862,8 +863,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const int q0 = base + ew * 32;
                 for (int b = 0; b < 32 && q0 + b < p.s; ++b) {
                     const int q = q0 + b;
-                    uint64_t *list = my_cand + static_cast<size_t>(q) * kTcCap;
-                    if (cnt[q] != sorted[q]) tc_compact_query(list, thr, cnt, sorted, q, p.k, lane);
+                    uint64_t *list = my_cand + static_cast<size_t>(q) * p.cap;
+                    if (cnt[q] != sorted[q]) tc_compact_query(list, thr, cnt, sorted, q, p.k, p.cap, lane);
                     const int n = cnt[q];
                     uint64_t *dst = p.partial + (static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
                     for (int i = lane; i < p.k; i += 32) dst[i] = (i < n) ? list[i] : 0ull;

@@ -196,10 +196,12 @@ def test_argument_errors():
 @pytest.mark.parametrize("N,d,s,k", [(1, 64, 1, 1), (129, 72, 3, 1), (300, 128, 9, 64), (1000, 64, 16, 5),
                                      (5000, 768, 100, 20), (257, 64, 257, 2), (3000, 256, 600, 7),
                                      (2000, 128, 300, 5), (700, 64, 40, 3), (300, 4096, 12, 3),
-                                     (40_000, 768, 512, 20)])
+                                     (40_000, 768, 512, 20), (3000, 128, 40, 65), (20_000, 64, 300, 128),
+                                     (50_000, 128, 70, 256), (200, 64, 33, 256), (700_001, 64, 40, 200)])
 def test_tcgen05_scan_integer_inputs_are_bit_exact(N, d, s, k):
     """The large-batch scan pinned explicitly (variant 3), including shapes with a ragged last
-    K chunk (d % 64 != 0), a ragged row tile, a second query half and a second pass."""
+    K chunk (d % 64 != 0), a ragged row tile, a second query half, a second pass, k beyond 64
+    (candidate lists of 512 slots) and more neighbours than rows."""
     x = workloads.integer_valued((N, d), seed=400 + N, lo=-3, hi=3, device=DEV)
     q = workloads.integer_valued((s, d), seed=500 + N, lo=-3, hi=3, device=DEV)
     for variant in (3, 4):                 # CTA pairs, single CTAs
