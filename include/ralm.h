@@ -87,7 +87,7 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx);
 
 /* C.retrieve(q_1..q_s): exact top-k of s queries over the whole corpus, one stream of the
  * corpus from HBM per pass (up to 32 queries on the small-batch scan, up to 512 on the
- * large-batch scan).
+ * large-batch scan, which takes over from 17 inner-product or 9 L2 queries on large corpora).
  *   queries DEVICE fp16 [s][d], 16-byte aligned.     0 <= s <= max_s
  *   ids     DEVICE int64 [s][k]  (written)           1 <= k <= max_k
  *   scores  DEVICE fp32  [s][k]  (written)
@@ -205,8 +205,9 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
  *   value only filters and the ranked distance is the direct sum of squared differences), 3 = tcgen05 scan (up to 512 queries per pass, k <= 256,
  *   d >= 64; pairs of CTAs share each MMA; for L2 the tensor-core value again only filters,
  *   and the corpus must be large enough to scan a sample first, about 600 K rows), 4 = tcgen05
- *   scan with single CTAs. Automatic: warp-MMA up to 32 queries (inner product) or 16 (L2), the
- *   tcgen05 scan beyond that where it applies.
+ *   scan with single CTAs. Automatic: warp-MMA up to 16 queries (inner product; 32 on corpora
+ *   too small for a sample launch, about 600 K rows) or 8 (L2), the tcgen05 scan beyond that
+ *   where it applies.
  * UNSUPPORTED if the variant cannot serve the index's metric or dimension. The environment
  * variable RALM_FORCE_VARIANT=<1..4> applies the same pin to every index at creation. */
 ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant);

@@ -22,7 +22,8 @@ class RalmError(RuntimeError):
 
 
 def lib_path() -> str:
-    return os.path.join(_HERE, "libralm.so")
+    """The compiled library; RALM_LIBRARY names another build of it (the bounds-checking one)."""
+    return os.environ.get("RALM_LIBRARY") or os.path.join(_HERE, "libralm.so")
 
 
 def load_library() -> ctypes.CDLL:

@@ -13,6 +13,28 @@ constexpr int kStatusBadCacheId = 6;
 constexpr int kStatusInternal = 8;  // a candidate list was asked to hold more than its capacity
 
 // ---------------------------------------------------------------------------------
+// Debug build (-DRALM_DEBUG_BOUNDS, `python -m paper_2401_14021_b200.build --debug`): every index
+// into a global array that a scan computes is checked against the array's extent; a violation
+// records kStatusInternal in the status word, a store is skipped and a load is redirected to
+// element 0. Nothing traps. The release build compiles the checks away.
+// ---------------------------------------------------------------------------------
+struct Extents {
+    long long rows;     // rows of the whole corpus (norms, bounds and the 8-bit copy have as many)
+    long long partial;  // keys in the partial-list array
+    long long lists;    // keys in the candidate lists that live in global memory (0: none)
+    long long aux;      // elements of the sample launch's maxima (tcgen05 scan)
+};
+#ifdef RALM_DEBUG_BOUNDS
+__device__ __forceinline__ bool in_bounds(long long i, long long n, int *status) {
+    if (i >= 0 && i < n) return true;
+    atomicMax(status, kStatusInternal);
+    return false;
+}
+#else
+__device__ __forceinline__ bool in_bounds(long long, long long, int *) { return true; }
+#endif
+
+// ---------------------------------------------------------------------------------
 // Ranking keys. Every candidate is one 64-bit key whose unsigned order IS the ranking:
 //   high 32 bits: order-preserving image of the "rank value" v (larger v ranks first),
 //                 v = score for inner product, v = -distance^2 for L2;

@@ -31,6 +31,7 @@ struct ralm_index {
     int variant;  // 0 auto, 1 FMA, 2 warp-MMA, 3 tcgen05
     int tune_warps, tune_depth, tune_rows;  // 0 = library default
     uint64_t *partial;   // [num_sms][max_s][max_k]
+    long long partial_keys;  // keys the array holds
     uint64_t *cache_keys;  // [RALM_MAX_CACHE_KEYS]
     uint64_t *spill;       // large k: candidate lists of the small-batch scan, [num_sms][8][spill_cap]
     int spill_cap;
@@ -72,6 +73,16 @@ constexpr int kPubMinK = 128;              // from this k on the scan CTAs share
 
 int align_up(int v, int a) { return (v + a - 1) / a * a; }
 
+// Extents of an index's global arrays (checked by the debug build's kernels).
+Extents index_extents(const ralm_index *idx, long long list_keys) {
+    Extents e;
+    e.rows = idx->N;
+    e.partial = idx->partial_keys;
+    e.lists = list_keys;
+    e.aux = idx->tc_gmax ? static_cast<long long>(idx->num_sms) * 4 * idx->max_s : 0;
+    return e;
+}
+
 // Every device allocation of the library goes through here, so that a test can make the n-th
 // one fail (ralm_debug_fail_allocation) and check that creation reports it and frees the rest.
 std::atomic<int> g_fail_allocation_in{0};
@@ -97,7 +108,7 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
         const int unit = s_pass == 1 ? 16 : 4;  // rows per reduction group of the FMA flavour
         pl->tile_rows = std::max(unit, idx->tune_rows / unit * unit);
     }
-    pl->stage_bytes = align_up(pl->tile_rows * idx->d * 2, 128);
+    pl->stage_bytes = align_up(pl->tile_rows * idx->d * 2 + (mma ? kTileShiftBytes : 0), 128);
     pl->off_q = kScanHeaderBytes;
     // (the warp-MMA flavour stages 8 query rows, or 16 when a pass carries more than 8)
     const int q_rows = s_pass > 16 ? 32 : (s_pass > kScanMaxQueries ? 16 : kScanMaxQueries);
@@ -114,7 +125,7 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
         const int max_rows = (pl->cap - k) / (kMaxConsumerWarps + 1) / unit * unit;
         if (pl->tile_rows > max_rows) {
             pl->tile_rows = std::max(unit, max_rows);
-            pl->stage_bytes = align_up(pl->tile_rows * idx->d * 2, 128);
+            pl->stage_bytes = align_up(pl->tile_rows * idx->d * 2 + (mma ? kTileShiftBytes : 0), 128);
         }
         // compact before the buffer is full, and already at about 4 k entries: a threshold only
         // rises when its list is compacted, and until then every push costs a shared atomic
@@ -319,6 +330,7 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
     p.thr_init = thr_init;
     p.mode = mode;
     p.gmax = idx->tc_gmax;
+    p.ext = index_extents(idx, static_cast<long long>(idx->num_sms) * idx->tc_cand_q * idx->tc_cand_cap);
     p.d = idx->d;
     p.slack = static_cast<float>(idx->d) * (1.0f / 2097152.0f);  // as in the small-batch L2 scan
     p.norms = idx->norms;
@@ -397,8 +409,13 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
 }
 
 constexpr int kTcAutoMinQueries = 9;     // batches the 8-query scan cannot serve in one pass
-constexpr int kTcAutoMinQueriesIp = 33;  // inner product: the small-batch scan takes up to 32 in one pass
-constexpr int kTcAutoMinQueriesL2 = 17;  // L2: up to 16
+// From how many queries the automatic variant takes the tcgen05 scan (measured on 21 M x 768 and
+// 50 M x 1024): inner product 24 queries 4.6 against 5.3 ms for the four-group warp-MMA pass, 16
+// queries 4.7 against 4.3-4.7; L2 9 queries 14.9 against 16.4 ms. On corpora too small for a sample
+// launch the small-batch scan keeps batches of up to 32 inner-product queries.
+constexpr int kTcAutoMinQueriesIp = 17;
+constexpr int kTcAutoMinQueriesIpSmall = 33;
+constexpr int kTcAutoMinQueriesL2 = 9;
 
 ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k, int64_t *ids,
                             float *scores, cudaStream_t st) {
@@ -417,7 +434,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     const bool tc = tc_can_serve(idx, k) && (!l2 || tc_two_phase) &&
                     (idx->variant == 3 || idx->variant == 4 ||
                      (idx->variant == 0 &&
-                      (s >= (l2 ? kTcAutoMinQueriesL2 : kTcAutoMinQueriesIp) || (!small_scan_fits && !l2))));
+                      (s >= (l2 ? kTcAutoMinQueriesL2 : (tc_two_phase ? kTcAutoMinQueriesIp : kTcAutoMinQueriesIpSmall)) ||
+                       (!small_scan_fits && !l2))));
     if (tc) {
         // Large corpora are scanned in two phases: a small sample first, which gives every query a
         // score that k rows are known to reach; the scan proper then starts from those thresholds,
@@ -506,6 +524,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
         p.sqnorms = nullptr;
         p.pub = nullptr;
         p.pub_rank = 0;
+        p.ext = index_extents(idx, idx->spill ? static_cast<long long>(idx->num_sms) * kScanMaxPassQueries * idx->spill_cap : 0);
         p.spill = pl.spill ? idx->spill : nullptr;
         p.partial = idx->partial;
         p.status = idx->status;
@@ -757,6 +776,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
         if (first_error == cudaSuccess) first_error = device_alloc(ptr, bytes);
     };
     alloc(&idx->partial, partial_bytes);
+    idx->partial_keys = static_cast<long long>(partial_bytes / sizeof(uint64_t));
     alloc(&idx->tc_thr, sizeof(float) * max_s);
     const int pass_queries = std::min(max_s, kScanMaxPassQueries);
     if (max_k > 1 && std::max(512, 2 * next_pow2(max_k)) * 8 * pass_queries > kSmemCandBytes) {
@@ -1033,6 +1053,7 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.variant = 0;
     view.tune_warps = view.tune_depth = view.tune_rows = 0;
     view.partial = dev->partial;
+    view.partial_keys = static_cast<long long>(RALM_STATIC_MAX_BLOCKS) * RALM_STATIC_MAX_S * RALM_STATIC_MAX_K;
     view.cache_keys = nullptr;
     view.tc_cand = nullptr;
     view.tc_cand_q = 0;

@@ -83,6 +83,7 @@ struct ScanParams {
     // rows, and every CTA may raise its threshold to it. Null: off.
     uint32_t *pub;
     int pub_rank;
+    Extents ext;     // extents of the global arrays, for the debug build's checks
 };
 
 struct ScanHeader {
@@ -216,6 +217,20 @@ __device__ __forceinline__ void transpose_reduce(float (&a)[V], int lane) {
     for (int o = 16 / V; o > 0; o >>= 1) a[0] += __shfl_xor_sync(0xffffffffu, a[0], o);
 }
 
+// Shared-memory banks, warp-MMA flavour: a lane reads 16 bytes of two rows per step and the
+// lanes of a quarter warp hold two different rows, which collide when a row is a multiple of 128
+// bytes long (768 and 1024 dimensions both are). So a tile is staged as two copies of 8 rows,
+// the second shifted by kTileShiftBytes, and MMA row m takes its data from staged row
+// staged_row(m), which alternates between the two groups (rows m and m + 1 then sit 64 bytes
+// apart modulo 128).
+constexpr int kTileShiftBytes = 64;
+__host__ __device__ __forceinline__ int staged_row(int m) {
+    return ((m & 1) << 3) + ((m & 8) >> 1) + ((m & 7) >> 1);
+}
+__host__ __device__ __forceinline__ int staged_row_offset(int row, int row_bytes) {
+    return row * row_bytes + ((row & 8) ? kTileShiftBytes : 0);
+}
+
 __device__ __forceinline__ void mma_m16n8k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
                                              uint32_t a3, uint32_t b0, uint32_t b1) {
     asm volatile(
@@ -241,9 +256,11 @@ __device__ __forceinline__ float2 h2_to_f2(uint32_t h2) {
 // its tile after the flag is up). Should that ever fail, the key is dropped and the status word
 // says so, rather than writing into the neighbouring list.
 __device__ __forceinline__ void push_candidate(ScanHeader *hdr, uint64_t *cand, int cap, int soft,
-                                               int q, uint64_t key, int *status) {
+                                               int q, uint64_t key, int *status, long long list_room = 1LL << 62) {
     const int slot = atomicAdd(&hdr->cnt[q], 1);
-    if (slot < cap) cand[static_cast<size_t>(q) * cap + slot] = key;
+    // (list_room: keys between `cand` and the end of the global list array; debug build only)
+    if (slot < cap && in_bounds(static_cast<long long>(q) * cap + slot, list_room, status))
+        cand[static_cast<size_t>(q) * cap + slot] = key;
     else atomicMax(status, kStatusInternal);
     if (slot >= soft) *reinterpret_cast<volatile int *>(&hdr->flag) = 1;
 }
@@ -287,6 +304,8 @@ scan_kernel(const ScanParams p) {
     uint64_t *scratch = p.spill ? reinterpret_cast<uint64_t *>(smem + p.off_cand) : nullptr;
     uint64_t *cand = p.spill ? p.spill + static_cast<size_t>(blockIdx.x) * kScanMaxPassQueries * p.cap
                              : reinterpret_cast<uint64_t *>(smem + p.off_cand);
+    const long long list_room = p.spill ? p.ext.lists - static_cast<long long>(blockIdx.x) * kScanMaxPassQueries * p.cap
+                                        : 1LL << 62;
     const int W = p.nwarps;
     const int S = W * p.depth;
     const int T = p.tile_rows;
@@ -330,51 +349,71 @@ scan_kernel(const ScanParams p) {
 
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
-        if (lane == 0) {
-            long long issued = 0;
-            bool ok = true;
-            // tile `it` belongs to consumer warp cw = it % W; it is that warp's (it / W)-th
-            // tile and goes to slot (it / W) % depth of the warp's private ring, for the
-            // use-th time. The counters advance incrementally: no division on this path.
-            int cw = 0, slot = 0;
-            uint32_t use = 0;
-            long long row0 = p.row_begin + static_cast<long long>(blockIdx.x) * T;
-            const long long row_step = static_cast<long long>(gridDim.x) * T;
-            const uint32_t stage_base = smem_u32(smem + p.off_stage);
-            for (long long it = 0; it < my_tiles; ++it) {
-                const int st = cw + slot * W;
-                if (use > 0) {
-                    ok = mbar_wait_bounded(smem_u32(&hdr->empty[st]), (use - 1) & 1);
-                    if (!ok) break;
-                }
-                if (*abort_flag) break;
+        // All 32 lanes run the loop (waits, counters and addresses stay warp-uniform); one elected
+        // lane issues the copies.
+        uint32_t elected;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "elect.sync _|p, 0xffffffff;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(elected));
+        long long issued = 0;
+        bool ok = true;
+        // tile `it` belongs to consumer warp cw = it % W; it is that warp's (it / W)-th
+        // tile and goes to slot (it / W) % depth of the warp's private ring, for the
+        // use-th time. The counters advance incrementally: no division on this path.
+        int cw = 0, slot = 0;
+        uint32_t use = 0;
+        long long row0 = p.row_begin + static_cast<long long>(blockIdx.x) * T;
+        const long long row_step = static_cast<long long>(gridDim.x) * T;
+        const uint32_t stage_base = smem_u32(smem + p.off_stage);
+        const uint32_t row_bytes = static_cast<uint32_t>(d * 2);
+        for (long long it = 0; it < my_tiles; ++it) {
+            const int st = cw + slot * W;
+            if (use > 0) {
+                const uint32_t ebar = smem_u32(&hdr->empty[st]);
+                if (!mbar_try_wait(ebar, (use - 1) & 1)) ok = mbar_wait_bounded(ebar, (use - 1) & 1);
+                if (!ok) break;
+            }
+            if (*abort_flag) break;
+            if (elected) {
                 const long long rows = (p.N - row0 < T) ? (p.N - row0) : T;
-                const uint32_t bytes = static_cast<uint32_t>(rows) * static_cast<uint32_t>(d * 2);
+                const uint32_t bytes = static_cast<uint32_t>(rows) * row_bytes;
                 const uint32_t bar = smem_u32(&hdr->full[st]);
+                const uint32_t dst = stage_base + static_cast<uint32_t>(st) * p.stage_bytes;
+                const long long src_row = in_bounds(row0 + rows - 1, p.ext.rows, p.status) ? row0 : 0;
                 mbar_arrive_expect_tx(bar, bytes);
-                bulk_load(stage_base + static_cast<uint32_t>(st) * p.stage_bytes, p.corpus + row0 * d,
-                          bytes, bar);
-                issued = it + 1;
-                row0 += row_step;
-                if (++cw == W) {
-                    cw = 0;
-                    if (++slot == p.depth) {
-                        slot = 0;
-                        ++use;
-                    }
+                if (MMA) {
+                    // rows 0..7 and rows 8..15 as two copies, the second kTileShiftBytes further
+                    const uint32_t first = rows < 8 ? bytes : 8u * row_bytes;
+                    bulk_load(dst, p.corpus + src_row * d, first, bar);
+                    if (bytes > first)
+                        bulk_load(dst + first + kTileShiftBytes, p.corpus + (src_row + 8) * d, bytes - first, bar);
+                } else {
+                    bulk_load(dst, p.corpus + src_row * d, bytes, bar);
                 }
             }
-            if (!ok) {
-                atomicMax(p.status, kStatusTimeout);
-                *abort_flag = 1;
-            }
-            if (*abort_flag) {
-                // winding down early: let every copy already issued land before exit
-                for (long long it = (issued > S ? issued - S : 0); it < issued; ++it) {
-                    const long long local = it / W;
-                    mbar_wait_bounded(smem_u32(&hdr->full[(it % W) + (local % p.depth) * W]),
-                                      (local / p.depth) & 1);
+            issued = it + 1;
+            row0 += row_step;
+            if (++cw == W) {
+                cw = 0;
+                if (++slot == p.depth) {
+                    slot = 0;
+                    ++use;
                 }
+            }
+        }
+        if (!ok && lane == 0) {
+            atomicMax(p.status, kStatusTimeout);
+            *abort_flag = 1;
+        }
+        __syncwarp();
+        if (*abort_flag) {
+            // winding down early: let every copy already issued land before exit
+            for (long long it = (issued > S ? issued - S : 0); it < issued; ++it) {
+                const long long local = it / W;
+                mbar_wait_bounded(smem_u32(&hdr->full[(it % W) + (local % p.depth) * W]),
+                                  (local / p.depth) & 1);
             }
         }
     } else if (warp - 1 < W) {
@@ -437,6 +476,7 @@ scan_kernel(const ScanParams p) {
             }
         }
 
+        const int ph_lo = staged_row(g), ph_hi = staged_row(g + 8);
         int slot = 0;         // position in this warp's private ring
         uint32_t parity = 0;  // phase parity of the ring's current lap
         long long row0 =
@@ -456,10 +496,11 @@ scan_kernel(const ScanParams p) {
             const int st = w + slot * W;
             const uint32_t full_bar = smem_u32(&hdr->full[st]);
             const uint32_t my_parity = parity;
-            float pn_lo = 0.f, pn_hi = 0.f;  // stored norms of rows g and g + 8, in flight during the wait
+            // (MMA rows g and g + 8 are the tile's rows ph_lo and ph_hi: see staged_row)
+            float pn_lo = 0.f, pn_hi = 0.f;  // stored norms of those rows, in flight during the wait
             if (MMA && L2 && NRM) {
-                if (row0 + g < p.N) pn_lo = __ldg(p.norms + row0 + g);
-                if (row0 + g + 8 < p.N) pn_hi = __ldg(p.norms + row0 + g + 8);
+                if (row0 + ph_lo < p.N && in_bounds(row0 + ph_lo, p.ext.rows, p.status)) pn_lo = __ldg(p.norms + row0 + ph_lo);
+                if (row0 + ph_hi < p.N && in_bounds(row0 + ph_hi, p.ext.rows, p.status)) pn_hi = __ldg(p.norms + row0 + ph_hi);
             }
             if (++slot == p.depth) {
                 slot = 0;
@@ -511,8 +552,8 @@ scan_kernel(const ScanParams p) {
                 float nhi[4] = {0.f, 0.f, 0.f, 0.f}, nhi_b[4] = {0.f, 0.f, 0.f, 0.f};
                 const int nchunks = (d + 31) >> 5;
                 const uint32_t q_addr = q_base_addr + g * q_pitch;
-                const uint32_t a_lo_addr = stage_addr + g * d * 2;
-                const uint32_t a_hi_addr = stage_addr + (g + 8) * d * 2;
+                const uint32_t a_lo_addr = stage_addr + staged_row_offset(ph_lo, d * 2);
+                const uint32_t a_hi_addr = stage_addr + staged_row_offset(ph_hi, d * 2);
 #pragma unroll 4
                 for (int c = 0; c < nchunks; ++c) {
                     // logical k (2t, 2t+1, 2t+8, 2t+9 of two MMAs) <- physical halves
@@ -547,7 +588,7 @@ scan_kernel(const ScanParams p) {
                 }
                 // acc[0]: (row g, query 2t)     acc[1]: (row g, query 2t+1)
                 // acc[2]: (row g+8, query 2t)   acc[3]: (row g+8, query 2t+1)
-                const long long r_lo = row0 + g, r_hi = row0 + g + 8;
+                const long long r_lo = row0 + ph_lo, r_hi = row0 + ph_hi;
                 const int q0 = 2 * t;  // this lane's first query within a group; the second is q0 + 1
                 if (L2) {
                     // |x|^2 - 2 x.q + |q|^2 from the tensor cores is only a FILTER (it cancels):
@@ -589,9 +630,9 @@ scan_kernel(const ScanParams p) {
                             while (m) {
                                 const int src = __ffs(m) - 1;
                                 m &= m - 1;
-                                const int row_local = (src >> 2) + ((i & 2) ? 8 : 0);
+                                const int row_local = staged_row((src >> 2) + ((i & 2) ? 8 : 0));
                                 const int q = grp * kScanMaxQueries + 2 * (src & 3) + (i & 1);
-                                const float dist = warp_direct_l2(stage_addr + row_local * d * 2,
+                                const float dist = warp_direct_l2(stage_addr + staged_row_offset(row_local, d * 2),
                                                                   q_base_addr + q * q_pitch, d, lane);
                                 if (lane == 0) {
                                     const float val = 0.0f - dist;
@@ -599,7 +640,7 @@ scan_kernel(const ScanParams p) {
                                     if (TOP1) {
                                         atomicMax(&hdr->best[q], static_cast<unsigned long long>(key));
                                     } else if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q])) {
-                                        push_candidate(hdr, cand, p.cap, p.soft_limit, q, key, p.status);
+                                        push_candidate(hdr, cand, p.cap, p.soft_limit, q, key, p.status, list_room);
                                     }
                                 }
                             }
@@ -629,18 +670,18 @@ scan_kernel(const ScanParams p) {
                         if (r_lo < p.N) {
                             if (gq0 < p.s && acc[grp][0] >= th0)
                                 push_candidate(hdr, cand, p.cap, p.soft_limit, gq0,
-                                               make_key(acc[grp][0], static_cast<uint32_t>(r_lo)), p.status);
+                                               make_key(acc[grp][0], static_cast<uint32_t>(r_lo)), p.status, list_room);
                             if (gq1 < p.s && acc[grp][1] >= th1)
                                 push_candidate(hdr, cand, p.cap, p.soft_limit, gq1,
-                                               make_key(acc[grp][1], static_cast<uint32_t>(r_lo)), p.status);
+                                               make_key(acc[grp][1], static_cast<uint32_t>(r_lo)), p.status, list_room);
                         }
                         if (r_hi < p.N) {
                             if (gq0 < p.s && acc[grp][2] >= th0)
                                 push_candidate(hdr, cand, p.cap, p.soft_limit, gq0,
-                                               make_key(acc[grp][2], static_cast<uint32_t>(r_hi)), p.status);
+                                               make_key(acc[grp][2], static_cast<uint32_t>(r_hi)), p.status, list_room);
                             if (gq1 < p.s && acc[grp][3] >= th1)
                                 push_candidate(hdr, cand, p.cap, p.soft_limit, gq1,
-                                               make_key(acc[grp][3], static_cast<uint32_t>(r_hi)), p.status);
+                                               make_key(acc[grp][3], static_cast<uint32_t>(r_hi)), p.status, list_room);
                         }
                     }
                 }
@@ -701,7 +742,7 @@ scan_kernel(const ScanParams p) {
                             bestA[0] = key > bestA[0] ? key : bestA[0];
                         } else if (val >= hdr->thr[jq]) {
                             push_candidate(hdr, cand, p.cap, p.soft_limit, jq,
-                                           make_key(val, static_cast<uint32_t>(row)), p.status);
+                                           make_key(val, static_cast<uint32_t>(row)), p.status, list_room);
                         }
                     }
                 }
@@ -723,7 +764,7 @@ scan_kernel(const ScanParams p) {
                 if (bestA[0]) atomicMax(&hdr->best[jq], static_cast<unsigned long long>(bestA[0]));
             }
             named_barrier(1, cthreads);
-            if (ctid < p.s)
+            if (ctid < p.s && in_bounds(static_cast<long long>(blockIdx.x) * p.s_total + p.q_base + ctid, p.ext.partial, p.status))
                 p.partial[static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + ctid] =
                     hdr->best[ctid];
         } else {
@@ -753,10 +794,11 @@ scan_kernel(const ScanParams p) {
             named_barrier(1, cthreads);
             for (int q = 0; q < p.s; ++q) {
                 const int n = hdr->cnt[q];
-                uint64_t *dst =
-                    p.partial + (static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
+                const long long first = (static_cast<long long>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
+                uint64_t *dst = p.partial + first;
                 for (int i = ctid; i < p.k; i += cthreads)
-                    dst[i] = (i < n) ? cand[static_cast<size_t>(q) * p.cap + i] : 0ull;
+                    if (in_bounds(first + i, p.ext.partial, p.status))
+                        dst[i] = (i < n) ? cand[static_cast<size_t>(q) * p.cap + i] : 0ull;
             }
         }
     }

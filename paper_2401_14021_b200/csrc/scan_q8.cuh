@@ -161,6 +161,8 @@ scan_q8_kernel(const ScanParams p) {
     uint64_t *scratch = p.spill ? reinterpret_cast<uint64_t *>(smem + p.off_cand) : nullptr;
     uint64_t *cand = p.spill ? p.spill + static_cast<size_t>(blockIdx.x) * kScanMaxPassQueries * p.cap
                              : reinterpret_cast<uint64_t *>(smem + p.off_cand);
+    const long long list_room = p.spill ? p.ext.lists - static_cast<long long>(blockIdx.x) * kScanMaxPassQueries * p.cap
+                                        : 1LL << 62;
     const int W = p.nwarps;
     const int S = W * p.depth;
     constexpr int T = 16;
@@ -256,9 +258,10 @@ scan_q8_kernel(const ScanParams p) {
             // rows 0..7 and rows 8..15 as two copies, the second 64 bytes further
             const uint32_t first = rows < 8 ? bytes : static_cast<uint32_t>(8 * d);
             const uint32_t dst = stage_base + static_cast<uint32_t>(st_) * p.stage_bytes;
-            bulk_load(dst, p.x8 + first_row * d, first, bar);
+            const long long src_row = in_bounds(first_row + rows - 1, p.ext.rows, p.status) ? first_row : 0;
+            bulk_load(dst, p.x8 + src_row * d, first, bar);
             if (bytes > first)
-                bulk_load(dst + first + kQ8TileBytesExtra, p.x8 + (first_row + 8) * d, bytes - first, bar);
+                bulk_load(dst + first + kQ8TileBytesExtra, p.x8 + (src_row + 8) * d, bytes - first, bar);
         };
         long long issued = 0, landed = 0;   // of this warp's tiles (lane 0 issues; all lanes count alike)
         for (; issued < p.depth && issued < n_mine; ++issued)
@@ -456,6 +459,7 @@ scan_q8_kernel(const ScanParams p) {
                         const int row_local = q8_phys_row((src >> 2) + ((i & 2) ? 8 : 0));
                         const int q = grp * kScanMaxQueries + 2 * (src & 3) + (i & 1);
                         const long long row = row0 + row_local;
+                        if (!in_bounds(row, p.ext.rows, p.status)) continue;
                         const float exact = warp_exact_score<L2>(p.corpus + row * d, q_base_addr + q * q_pitch, d, lane);
                         const float val = L2 ? 0.0f - exact : exact;
                         if (lane == 0) {
@@ -464,7 +468,7 @@ scan_q8_kernel(const ScanParams p) {
                                 if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q]))
                                     atomicMax(&hdr->best[q], static_cast<unsigned long long>(key));
                             } else if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q])) {
-                                push_candidate(hdr, cand, p.cap, p.soft_limit, q, key, p.status);
+                                push_candidate(hdr, cand, p.cap, p.soft_limit, q, key, p.status, list_room);
                             }
                         }
                     }
@@ -481,7 +485,7 @@ scan_q8_kernel(const ScanParams p) {
         // ------------------------------------------------------------ CTA result
         if (TOP1) {
             named_barrier(1, cthreads);
-            if (ctid < p.s)
+            if (ctid < p.s && in_bounds(static_cast<long long>(blockIdx.x) * p.s_total + p.q_base + ctid, p.ext.partial, p.status))
                 p.partial[static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + ctid] = hdr->best[ctid];
         } else {
             __syncwarp();
@@ -508,9 +512,11 @@ scan_q8_kernel(const ScanParams p) {
             named_barrier(1, cthreads);
             for (int q = 0; q < p.s; ++q) {
                 const int n = hdr->cnt[q];
-                uint64_t *dst = p.partial + (static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
+                const long long first = (static_cast<long long>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
+                uint64_t *dst = p.partial + first;
                 for (int i = ctid; i < p.k; i += cthreads)
-                    dst[i] = (i < n) ? cand[static_cast<size_t>(q) * p.cap + i] : 0ull;
+                    if (in_bounds(first + i, p.ext.partial, p.status))
+                        dst[i] = (i < n) ? cand[static_cast<size_t>(q) * p.cap + i] : 0ull;
             }
         }
     }

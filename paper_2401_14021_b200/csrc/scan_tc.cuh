@@ -100,6 +100,7 @@ struct TcParams {
     // rows, the sample's too.
     int mode;
     float *gmax;        // sample launches: [gridDim.x * 4][s_total] maxima, -inf where a warp saw no row
+    Extents ext;        // extents of the global arrays, for the debug build's checks
     int d;
     float slack;
     const float *norms;      // |x|^2 of every corpus row (fp32)
@@ -285,7 +286,7 @@ __device__ __forceinline__ void tc_compact_query(uint64_t *list, float *thr, int
 // column); each hit reserves its slot with its own shared-memory atomic.
 __device__ __forceinline__ void tc_store_hits(const uint32_t (&v)[32], uint32_t hit, int *cnt_chunk,
                                               uint64_t *cand_chunk, uint32_t row, volatile int *dirty, int *status, int cap,
-                                              int soft) {
+                                              int soft, long long room) {
     const uint32_t any_col = __reduce_or_sync(0xffffffffu, hit);
 #pragma unroll
     for (int b = 0; b < 32; ++b) {
@@ -293,8 +294,9 @@ __device__ __forceinline__ void tc_store_hits(const uint32_t (&v)[32], uint32_t 
             if ((hit >> b) & 1u) {
                 const int slot = atomicAdd(&cnt_chunk[b], 1);
                 if (slot + 1 >= soft) *dirty = 1;
-                if (slot < cap) cand_chunk[static_cast<size_t>(b) * cap + slot] = make_key(__uint_as_float(v[b]), row);
-                else atomicMax(status, kStatusInternal);
+                if (slot >= cap) atomicMax(status, kStatusInternal);
+                else if (in_bounds(static_cast<long long>(b) * cap + slot, room, status))
+                    cand_chunk[static_cast<size_t>(b) * cap + slot] = make_key(__uint_as_float(v[b]), row);
             }
         }
     }
@@ -309,7 +311,9 @@ __device__ __forceinline__ void tc_store_hits(const uint32_t (&v)[32], uint32_t 
 __device__ __noinline__ void tc_append_octet(uint32_t v0, uint32_t v1, uint32_t v2, uint32_t v3, uint32_t v4,
                                              uint32_t v5, uint32_t v6, uint32_t v7, int c0, float thr_lane,
                                              int *cnt_block, uint64_t *cand_block, uint32_t row, bool row_ok,
-                                             volatile int *dirty, int *status, int cap, int soft) {
+                                             volatile int *dirty, int *status, int cap, int soft,
+                                             long long room) {
+    // (room: keys between cand_block and the end of the list array; checked in the debug build)
     const uint32_t v[8] = {v0, v1, v2, v3, v4, v5, v6, v7};
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -320,10 +324,10 @@ __device__ __noinline__ void tc_append_octet(uint32_t v0, uint32_t v1, uint32_t 
             // (a list holds fewer than `soft` keys when a unit starts and gains at most 128 in
             // one, so slot < cap; should that ever fail the key is dropped and the status
             // word says so, rather than writing into the neighbouring list)
-            if (slot < cap)
-                cand_block[static_cast<size_t>(c0 + i) * cap + slot] = make_key(__uint_as_float(v[i]), row);
-            else
+            if (slot >= cap)
                 atomicMax(status, kStatusInternal);
+            else if (in_bounds(static_cast<long long>(c0 + i) * cap + slot, room, status))
+                cand_block[static_cast<size_t>(c0 + i) * cap + slot] = make_key(__uint_as_float(v[i]), row);
         }
     }
 }
@@ -359,7 +363,7 @@ __device__ __noinline__ void tc_append_chunk_l2(uint32_t taddr, const float *thr
                                                 int *cnt_chunk, uint64_t *cand_chunk, uint32_t row, bool row_ok,
                                                 float nx, float slack, const __half *corpus,
                                                 const __half *queries_chunk, int d, volatile int *dirty,
-                                                int *status, int cap, int soft, int lane) {
+                                                int *status, int cap, int soft, long long room, int lane) {
     uint32_t v[32];
     tmem_ld32(taddr, v);
     uint32_t hit = 0;
@@ -389,7 +393,7 @@ __device__ __noinline__ void tc_append_chunk_l2(uint32_t taddr, const float *thr
             }
         }
     }
-    tc_store_hits(v, hit, cnt_chunk, cand_chunk, row, dirty, status, cap, soft);
+    tc_store_hits(v, hit, cnt_chunk, cand_chunk, row, dirty, status, cap, soft, room);
 }
 
 // One block of 32 queries of a sample launch: for every column the best rank value among this
@@ -700,6 +704,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const int ew = warp - 2;        // 0..3
         const int quarter = warp & 3;   // the TMEM lanes this warp may read: 32 * quarter ..
         uint64_t *my_cand = p.cand + static_cast<size_t>(blockIdx.x) * p.cand_q * p.cap;
+        const long long cand_room = p.ext.lists - static_cast<long long>(blockIdx.x) * p.cand_q * p.cap;
         constexpr bool sample = MODE == 1 || MODE == 3;
         constexpr bool l2 = MODE == 1 || MODE == 2;
         bool ok = true;
@@ -744,7 +749,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const bool row_ok = row < p.N;
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                        static_cast<uint32_t>(acc * kTcMaxN);
-                const float nx = (l2 && row_ok) ? __ldg(p.norms + row) : 0.f;
+                const float nx = (l2 && row_ok && in_bounds(row, p.ext.rows, p.status)) ? __ldg(p.norms + row) : 0.f;
 #pragma unroll
                 for (int j = 0; j < kTcMaxN / 32; ++j) {
                     if (j * 32 < nq) {
@@ -781,7 +786,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                                 tc_append_chunk_l2(t_row + j * 32, thr + qb + j * 32, qn + qb + j * 32, cnt + qb + j * 32,
                                                    my_cand + static_cast<size_t>(qb + j * 32) * p.cap,
                                                    static_cast<uint32_t>(row), row_ok, nx, p.slack, p.corpus,
-                                                   p.queries + static_cast<size_t>(qb + j * 32) * p.d, p.d, dirty, p.status, p.cap, p.soft, lane);
+                                                   p.queries + static_cast<size_t>(qb + j * 32) * p.d, p.d, dirty, p.status, p.cap, p.soft,
+                                                   cand_room - static_cast<long long>(qb + j * 32) * p.cap, lane);
                         } else {
                             // common case: nothing passes. Four independent predicate chains, one per
                             // eight columns, so that the rare case only revisits the eight it concerns.
@@ -797,19 +803,20 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                             if (__any_sync(0xffffffffu, row_ok && (p0 | p1 | p2 | p3))) {
                                 int *cnt_block = cnt + qb + j * 32;
                                 uint64_t *cand_block = my_cand + static_cast<size_t>(qb + j * 32) * p.cap;
+                                const long long room = cand_room - static_cast<long long>(qb + j * 32) * p.cap;
                                 const uint32_t r32 = static_cast<uint32_t>(row);
                                 if (__any_sync(0xffffffffu, row_ok && p0))
                                     tc_append_octet(v[0], v[1], v[2], v[3], v[4], v[5], v[6], v[7], 0, my_thr, cnt_block,
-                                                    cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft);
+                                                    cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft, room);
                                 if (__any_sync(0xffffffffu, row_ok && p1))
                                     tc_append_octet(v[8], v[9], v[10], v[11], v[12], v[13], v[14], v[15], 8, my_thr,
-                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft);
+                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft, room);
                                 if (__any_sync(0xffffffffu, row_ok && p2))
                                     tc_append_octet(v[16], v[17], v[18], v[19], v[20], v[21], v[22], v[23], 16, my_thr,
-                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft);
+                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft, room);
                                 if (__any_sync(0xffffffffu, row_ok && p3))
                                     tc_append_octet(v[24], v[25], v[26], v[27], v[28], v[29], v[30], v[31], 24, my_thr,
-                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft);
+                                                    cnt_block, cand_block, r32, row_ok, dirty, p.status, p.cap, p.soft, room);
                             }
                         }
                     }
@@ -854,7 +861,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < kTcMaxN / 32; ++j) {
                     const int q = h * p.nb + j * 32 + lane;
-                    if (h < p.nhalves && j * 32 < p.nb && q < p.s)
+                    if (h < p.nhalves && j * 32 < p.nb && q < p.s &&
+                        in_bounds((static_cast<long long>(blockIdx.x) * 4 + ew) * p.s_total + p.q_base + q, p.ext.aux, p.status))
                         dst[q] = best[h][j] ? from_ordered_bits(best[h][j]) : -INFINITY;
                 }
         } else {
@@ -866,8 +874,10 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     uint64_t *list = my_cand + static_cast<size_t>(q) * p.cap;
                     if (cnt[q] != sorted[q]) tc_compact_query(list, thr, cnt, sorted, q, p.k, p.cap, lane);
                     const int n = cnt[q];
-                    uint64_t *dst = p.partial + (static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
-                    for (int i = lane; i < p.k; i += 32) dst[i] = (i < n) ? list[i] : 0ull;
+                    const long long first = (static_cast<long long>(blockIdx.x) * p.s_total + p.q_base + q) * p.k;
+                    uint64_t *dst = p.partial + first;
+                    for (int i = lane; i < p.k; i += 32)
+                        if (in_bounds(first + i, p.ext.partial, p.status)) dst[i] = (i < n) ? list[i] : 0ull;
                 }
             }
         }
