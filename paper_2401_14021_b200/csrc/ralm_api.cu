@@ -42,6 +42,7 @@ struct ralm_index {
     bool x8_force;         // use the copy also on corpora too small for a sample phase (testing aid)
     float *tc_thr;         // thresholds from the sample phase of a two-phase scan, [max_s]
     float *tc_gmax;        // tcgen05 scan, sample launch: [num_sms * 4][max_s] maxima per selection warp
+    int *tc_tile_counter;  // tcgen05 scan: the launch's row-tile counter
     bool tc_two_phase;     // sample phase enabled (tuning aid)
     int tc_clusters;       // CTA pairs the device runs at once (-1 = not asked yet)
     uint64_t *tc_cand;     // tcgen05 scan: [num_sms][tc_cand_q][tc_cand_cap] candidate lists, or null
@@ -304,6 +305,10 @@ bool alloc_tc_workspace(ralm_index *idx, int queries) {
         idx->tc_gmax = nullptr;
         return false;
     }
+    if (!idx->tc_tile_counter && device_alloc(&idx->tc_tile_counter, sizeof(int)) != cudaSuccess) {
+        idx->tc_tile_counter = nullptr;
+        return false;
+    }
     if (device_alloc(&idx->tc_cand, bytes) != cudaSuccess) {
         idx->tc_cand = nullptr;
         return false;
@@ -330,6 +335,8 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
     p.thr_init = thr_init;
     p.mode = mode;
     p.gmax = idx->tc_gmax;
+    p.tile_counter = idx->tc_tile_counter;
+    if (cudaMemsetAsync(idx->tc_tile_counter, 0, sizeof(int), st) != cudaSuccess) return RALM_ERR_CUDA;
     p.ext = index_extents(idx, static_cast<long long>(idx->num_sms) * idx->tc_cand_q * idx->tc_cand_cap);
     p.d = idx->d;
     p.slack = static_cast<float>(idx->d) * (1.0f / 2097152.0f);  // as in the small-batch L2 scan
@@ -763,6 +770,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->tc_clusters = -1;
     idx->tc_thr = nullptr;
     idx->tc_gmax = nullptr;
+    idx->tc_tile_counter = nullptr;
     idx->tc_two_phase = true;
     idx->norms = nullptr;
     idx->x8 = nullptr;
@@ -831,6 +839,7 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
     cudaFree(idx->tc_cand);
     cudaFree(idx->tc_thr);
     cudaFree(idx->tc_gmax);
+    cudaFree(idx->tc_tile_counter);
     cudaFree(idx->norms);
     cudaFree(idx->x8);
     cudaFree(idx->x8_bound);
@@ -1061,6 +1070,7 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.tc_clusters = -1;
     view.tc_thr = nullptr;
     view.tc_gmax = nullptr;
+    view.tc_tile_counter = nullptr;
     view.tc_two_phase = false;
     view.spill = nullptr;
     view.spill_cap = 0;

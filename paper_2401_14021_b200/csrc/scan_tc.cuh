@@ -72,6 +72,7 @@ struct TcParams {
     long long tile0;    // first row tile (of 128 rows, 256 for pairs) of this launch
     const float *thr_init;  // [s_total] starting thresholds (scores that k rows are known to reach), or null
     long long ntiles;   // row tiles of this launch
+    int *tile_counter;  // zeroed before the launch: row tiles beyond the first of each CTA (pair) are handed out here
     int nchunks;        // ceil(d / 64)
     int s;              // queries in this pass (<= 512)
     int s_total;
@@ -114,11 +115,15 @@ struct TcHeader {
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t drain;
+    uint64_t tile_full[32];  // tile_ring[i] holds the number of this CTA's (i + 32 n)-th row tile
+    int tile_ring[32];
+    int sel_tile[2];         // the selection warps' copy of their current tile number (even / odd tiles)
     uint32_t tmem_base;
     int abort;
     int dirty[3];  // [u % 3]: some candidate list reached the soft limit during unit u
 };
-constexpr int kTcHeaderBytes = 512;
+constexpr int kTcHeaderBytes = 1024;
+constexpr int kTcTileRing = 32;  // (a power of two; see scan_tc_kernel for why 32 is enough)
 static_assert(sizeof(TcHeader) <= kTcHeaderBytes, "header too large");
 // shared-memory layout after the header
 constexpr int kTcOffThr = kTcHeaderBytes;                      // float [512]
@@ -470,6 +475,36 @@ __device__ __forceinline__ void tc_mma_f16_pair(uint32_t d_tmem, uint64_t a_desc
         : "memory");
 }
 
+// Remote store of one 32-bit value into the other CTA's shared memory that completes 4 bytes of
+// the transaction count of an mbarrier there (so the value is visible to whoever that barrier lets through).
+__device__ __forceinline__ void st_async_u32(uint32_t cluster_addr, uint32_t value, uint32_t cluster_bar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];" ::"r"(cluster_addr),
+                 "r"(value), "r"(cluster_bar)
+                 : "memory");
+}
+
+// Row tiles are handed out dynamically: CTAs (pairs) differ in speed by a few percent, and with a
+// fixed assignment the slowest sets the launch's time. The leader's producer warp takes tile
+// numbers from a global counter one tile ahead of its loads and publishes them in a small ring in
+// shared memory (its own, and by st.async the follower's); every role reads its next tile there.
+// The number of this CTA's seq-th tile, or -1 when there is none left (or the wait gave up). All
+// lanes of the calling warp get the same value. `arm`: this warp is the follower's producer, whose
+// elected lane makes the one arrival of the barrier's phase and announces the 4 bytes to come.
+__device__ __forceinline__ long long tc_read_tile(TcHeader *hdr, long long seq, bool arm, bool elected,
+                                                  volatile int *abort_flag, int *status, int lane) {
+    const int slot = static_cast<int>(seq & (kTcTileRing - 1));
+    const uint32_t bar = smem_u32(&hdr->tile_full[slot]);
+    if (arm && elected) mbar_arrive_expect_tx(bar, 4);
+    if (!tc_wait(bar, static_cast<uint32_t>((seq / kTcTileRing) & 1), abort_flag)) {
+        if (lane == 0 && !*abort_flag) {
+            atomicMax(status, kStatusTimeout);
+            *abort_flag = 1;
+        }
+        return -1;
+    }
+    return *reinterpret_cast<volatile int *>(&hdr->tile_ring[slot]);
+}
+
 // PAIR = false: every CTA is on its own (M = 128 rows per MMA).
 // PAIR = true: clusters of two CTAs. A row tile is 256 rows; CTA r of the pair stages rows
 // 128 r .. 128 r + 127 and half of the query rows of each K chunk, the leader (rank 0) issues
@@ -508,6 +543,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             mbar_init(smem_u32(&hdr->tmem_empty[i]), PAIR ? 8 : 4);
         }
         mbar_init(smem_u32(&hdr->drain), 1);
+        for (int i = 0; i < kTcTileRing; ++i) mbar_init(smem_u32(&hdr->tile_full[i]), 1);
         mbar_fence_init();
         hdr->abort = 0;
         hdr->dirty[0] = hdr->dirty[1] = hdr->dirty[2] = 0;
@@ -554,8 +590,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(&hdr->tmem_base);
 
-    const long long my_tiles = (p.ntiles > group) ? (p.ntiles - group + ngroups - 1) / ngroups : 0;
-    const long long my_units = my_tiles * p.nhalves;
+    // (tile numbers: the ring of kTcTileRing slots is never overrun. A slot is rewritten 32 tiles
+    // later; the publisher runs at most the stage ring (<= 12 tiles) plus one tile ahead of the MMA
+    // warp, which runs at most two units ahead of the selection warps.)
     volatile int *abort_flag = &hdr->abort;
     const uint32_t stage_base = smem_u32(tc_smem + p.off_stage);
 
@@ -572,9 +609,31 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         uint32_t lap = 0;
         long long issued = 0;
         bool ok = true;
-        for (long long u = 0; u < my_units && ok; ++u) {
-            const long long tile = p.tile0 + group + (u / p.nhalves) * ngroups;
+        // The leader publishes this CTA's (pair's) tile numbers: the first is fixed, the others come
+        // from the launch's counter, each taken one tile before its loads are due.
+        bool more = true;   // (leader's elected lane) the last number published was a tile
+        auto publish = [&](long long seq, long long number) {
+            const int slot = static_cast<int>(seq & (kTcTileRing - 1));
+            const int value = number < p.ntiles ? static_cast<int>(number) : -1;
+            more = value >= 0;
+            *reinterpret_cast<volatile int *>(&hdr->tile_ring[slot]) = value;
+            const uint32_t bar = smem_u32(&hdr->tile_full[slot]);
+            mbar_arrive(bar);
+            if (PAIR)
+                st_async_u32(map_to_cta(smem_u32(&hdr->tile_ring[slot]), 1), static_cast<uint32_t>(value),
+                             map_to_cta(bar, 1));
+        };
+        if (leader && elected) publish(0, group);
+        long long tile = -1;
+        for (long long u = 0; ok; ++u) {
             const int half = static_cast<int>(u % p.nhalves);
+            if (half == 0) {
+                const long long seq = u / p.nhalves;
+                if (leader && elected && more) publish(seq + 1, ngroups + atomicAdd(p.tile_counter, 1));
+                tile = tc_read_tile(hdr, seq, PAIR && !leader, elected, abort_flag, p.status, lane);
+                if (tile < 0) break;
+                tile += p.tile0;
+            }
             const int row_y = static_cast<int>(tile * kGroupRows + rank * kTcTileM);
             // a pair splits the N of this unit's MMA, not nb: the follower supplies the upper
             // half of the (rounded) queries this half really has
@@ -635,8 +694,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             int st = 0;
             uint32_t lap = 0;
             bool ok = true;
-            for (long long u = 0; u < my_units && ok; ++u) {
+            for (long long u = 0; ok; ++u) {
                 const int half = static_cast<int>(u % p.nhalves);
+                if (half == 0 && tc_read_tile(hdr, u / p.nhalves, false, elected, abort_flag, p.status, lane) < 0) break;
                 const int acc = static_cast<int>(u & 1);
                 const int nq = (p.s - half * p.nb < p.nb) ? (p.s - half * p.nb) : p.nb;
                 const int n_mma = PAIR ? ((nq + 31) & ~31) : ((nq + 15) & ~15);
@@ -722,9 +782,23 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         for (int h = 0; h < 2; ++h)
 #pragma unroll
             for (int j = 0; j < kTcMaxN / 32; ++j) best[h][j] = 0u;
-        for (long long u = 0; u < my_units; ++u) {
-            const long long tile = p.tile0 + group + (u / p.nhalves) * ngroups;
+        long long tile = -1;
+        for (long long u = 0;; ++u) {
             const int half = static_cast<int>(u % p.nhalves);
+            if (half == 0) {
+                // One warp waits for the tile number and hands it to the others, so that all four
+                // take the same decision (also when that wait gives up) and leave together: they
+                // meet at named barriers that have no time limit.
+                const long long seq = u / p.nhalves;
+                if (ew == 0) {
+                    const long long number = tc_read_tile(hdr, seq, false, false, abort_flag, p.status, lane);
+                    if (lane == 0) *reinterpret_cast<volatile int *>(&hdr->sel_tile[seq & 1]) = static_cast<int>(number);
+                }
+                named_barrier(2, 128);
+                tile = *reinterpret_cast<volatile int *>(&hdr->sel_tile[seq & 1]);
+                if (tile < 0) break;
+                tile += p.tile0;
+            }
             const int acc = static_cast<int>(u & 1);
             const int qb = half * p.nb;
             const int nq = (p.s - qb < p.nb) ? (p.s - qb) : p.nb;

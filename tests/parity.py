@@ -16,6 +16,7 @@ Scores: |gpu_score - oracle_score(gpu_id)| <= 2e-3 * |oracle_score| + 1e-5 * sca
 from dataclasses import dataclass
 
 import numpy as np
+import torch
 
 import oracle
 
@@ -93,3 +94,34 @@ def check_search(gpu_ids, gpu_scores, corpus_np, queries_np, metric, k, exact=Fa
                              lambda j, i=i: oracle.pair_score(corpus_np[j], queries_np[i], metric),
                              metric, scale=scale, n_valid=corpus_np.shape[0])
     return total
+
+
+def sampled_parity(x, q, ids, scores, metric, k, n_chunks, chunk_rows, seed, query_sel=None):
+    """Full-size check on a sub-corpus: seeded random chunks of rows, the first rows, the ragged tail
+    and every row the GPU returned, ranked by the oracle. If the GPU's lists are the top-k of the
+    whole corpus they are the top-k of that sub-corpus too. Returns (Counts, rows in the sub-corpus)
+    and asserts that no swap needed the wide band."""
+    N = x.shape[0]
+    sel = list(range(q.shape[0])) if query_sel is None else list(query_sel)
+    g = torch.Generator().manual_seed(seed)
+    starts = (torch.randint(0, max(1, N // chunk_rows), (n_chunks,), generator=g) * chunk_rows).tolist()
+    starts += [0, max(0, N - chunk_rows + 1)]
+    rows = torch.cat([torch.arange(s0, min(N, s0 + chunk_rows)) for s0 in sorted(set(starts))])
+    gi, gs = ids.cpu(), scores.cpu().numpy()
+    returned = gi[sel].flatten()
+    sub_rows = torch.unique(torch.cat([rows, returned[returned >= 0]]))     # ascending: id order is kept
+    xs = x[sub_rows.to(x.device)].cpu().numpy()
+    qn = q.cpu().numpy()[sel]
+    o_local, o_scores = oracle.search(xs, qn, metric, k)
+    o_ids = np.where(o_local >= 0, sub_rows.numpy()[np.maximum(o_local, 0)], -1)
+    pos = {int(r): i for i, r in enumerate(sub_rows.tolist())}
+    max_norm = float(np.linalg.norm(xs.astype(np.float64), axis=1).max())
+    counts = Counts()
+    for n, i in enumerate(sel):
+        scale = max_norm * float(np.linalg.norm(qn[n].astype(np.float64)))
+        counts += check_lists(gi[i].numpy(), gs[i], o_ids[n], o_scores[n],
+                              lambda j, n=n: oracle.pair_score(xs[pos[j]], qn[n], metric), metric,
+                              scale=scale, n_valid=N)
+    # swaps that fp32 rounding does not explain are accepted by the 2e-3 rule but not expected
+    assert counts.wide == 0, str(counts)
+    return counts, sub_rows.numel()
