@@ -461,12 +461,11 @@ def main():
         # algorithmic bytes of one pass, from what the library says it ran: one read of the fp16
         # rows; the tcgen05 scan reads its sample's rows twice (sample launch, then the scan proper);
         # the 8-bit scan reads the sample in fp16 and the rest as one byte per element + one bound
+        again = sample if dispatch["phases"] == 3 else 0     # sample rows the main launch scans again
         if dispatch["kernel"] == 5:
-            pass_bytes = sample * d * 2 + (local_rows - sample) * (d + 4)
-        elif dispatch["kernel"] in (3, 4):
-            pass_bytes = (local_rows + sample) * d * 2
+            pass_bytes = sample * d * 2 + (local_rows - sample + again) * (d + 4)
         else:
-            pass_bytes = corpus_bytes
+            pass_bytes = (local_rows + again) * d * 2
         achieved = pass_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None
         traffic = None
         if dispatch["kernel"] == 2 and cfg.metric == "ip" and s <= 8 and not args.tune and \
@@ -486,7 +485,7 @@ def main():
         if dispatch["kernel"] in (3, 4) and per_pass_queries > 255:
             # large batch: s flop per corpus byte is beyond the ridge, the tensor pipe bounds it.
             # fp16 runs at the bf16 rate; the kernel is timed inside a long step: sustained peak
-            flops = 2.0 * per_pass_queries * (local_rows + sample) * d
+            flops = 2.0 * per_pass_queries * (local_rows + again) * d
             tf = flops / (scan_avg_ms * 1e-3) / 1e12 if scan_launches else None
             peak_tf = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
             roofline = {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",

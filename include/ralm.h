@@ -256,9 +256,10 @@ ralm_status_t ralm_index_read_timing_list(ralm_index_t *idx, double *ms, int64_t
 /* What the most recent ralm_search / ralm_search_host on this index ran (measurement aid; HOST
  * pointers). kernel: 0 = no search yet, 1 = FMA scan, 2 = warp-MMA scan, 3 = tcgen05 scan with CTA
  * pairs, 4 = tcgen05 scan with single CTAs, 5 = 8-bit scan. passes: passes over the corpus (each
- * serves one slice of the batch). phases: 2 when every pass scans a sample first, else 1.
- * sample_rows: rows of that sample (0 without one). For kernels 1, 2 and 5 the sample's rows are
- * scanned once, by the sample launch; for 3 and 4 the main launch scans them again. */
+ * serves one slice of the batch). phases: 1 = one launch per pass; 2 = a sample of the rows is
+ * scanned first (in fp16) and the main launch covers the other rows; 3 = the sample launch only
+ * yields thresholds and the main launch scans every row, the sample's again (the tcgen05 scan;
+ * the other scans for k >= 128). sample_rows: rows of that sample (0 without one). */
 ralm_status_t ralm_index_last_dispatch(const ralm_index_t *idx, int32_t *kernel, int32_t *passes,
                                        int32_t *phases, int64_t *sample_rows);
 

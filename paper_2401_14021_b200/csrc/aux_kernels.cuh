@@ -25,25 +25,26 @@ __device__ __forceinline__ void write_result(uint64_t key, bool l2, int64_t *id_
 // Threshold from the maxima of a sample launch: one CTA per query. vals holds G values for the
 // query (vals[g * stride + query], -inf = the group saw no row), each the best rank value of a
 // different, disjoint group of rows, so the k-th largest of them is reached by k different rows.
-// Writes it to thr_out[query], or -inf when fewer than k groups saw a row. G <= kMergeSortMax.
+// Writes it to thr_out[query], or -inf when fewer than k groups saw a row. G <= kMaximaSortMax.
 // ------------------------------------------------------------------------------------
+constexpr int kMaximaSortMax = 8192;
 __global__ void __launch_bounds__(kMergeThreads, 1)
 kth_of_maxima_kernel(const float *__restrict__ vals, int G, int stride, int k, float *__restrict__ thr_out) {
-    __shared__ uint64_t buf[kMergeSortMax];
+    __shared__ uint32_t buf[kMaximaSortMax];   // order-preserving bits; 0 = no row
     const int q = blockIdx.x;
     const int tid = threadIdx.x;
     const int P = next_pow2(G > 1 ? G : 2);
     for (int i = tid; i < P; i += kMergeThreads) {
-        uint64_t key = 0;
+        uint32_t bits = 0;
         if (i < G) {
             const float v = vals[static_cast<size_t>(i) * stride + q];
-            if (v != -INFINITY) key = make_key(v, static_cast<uint32_t>(i));
+            if (v != -INFINITY) bits = ordered_bits(v + 0.0f);
         }
-        buf[i] = key;
+        buf[i] = bits;
     }
     __syncthreads();
     bitonic_sort_desc(buf, P, tid, kMergeThreads, -1);
-    if (tid == 0) thr_out[q] = (k <= G && buf[k - 1] != 0ull) ? key_value(buf[k - 1]) : -INFINITY;
+    if (tid == 0) thr_out[q] = (k <= G && buf[k - 1] != 0u) ? from_ordered_bits(buf[k - 1]) : -INFINITY;
 }
 
 // ------------------------------------------------------------------------------------

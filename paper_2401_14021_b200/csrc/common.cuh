@@ -129,14 +129,15 @@ __device__ __forceinline__ void group_sync(int bar_id, int nthr) {
     else if (bar_id == -1) __syncthreads();
     else __syncwarp();
 }
-__device__ inline void bitonic_sort_desc(uint64_t *a, int P, int tid, int nthr, int bar_id) {
+template <typename Key>
+__device__ inline void bitonic_sort_desc(Key *a, int P, int tid, int nthr, int bar_id) {
     for (int size = 2; size <= P; size <<= 1) {
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
             for (int i = tid; i < (P >> 1); i += nthr) {
                 const int lo = 2 * i - (i & (stride - 1));
                 const int hi = lo + stride;
                 const bool desc = (lo & size) == 0;
-                const uint64_t x = a[lo], y = a[hi];
+                const Key x = a[lo], y = a[hi];
                 if ((x < y) == desc) {
                     a[lo] = y;
                     a[hi] = x;

@@ -36,6 +36,7 @@ struct ralm_index {
     uint64_t *spill;       // large k: candidate lists of the small-batch scan, [num_sms][8][spill_cap]
     int spill_cap;
     uint32_t *pub;         // large k: thresholds the scan CTAs publish to each other, [num_sms][max_s]
+    float *scan_gmax;      // large k: per-warp maxima of the small-batch scan's sample launch, [num_sms * 8][max_s]
     float *norms;          // L2: squared norm of every corpus row (fp32 [N]), or null
     uint8_t *x8;           // inner product, optional: one-byte (E5M2) copy of the corpus, [N][d]
     float *x8_bound;       // per row: bound on |q.x - q.x8| per unit of |q| (see scan_q8.cuh)
@@ -71,6 +72,7 @@ struct ScanPlan {
 
 constexpr int kSmemCandBytes = 32 * 1024;  // candidate lists larger than this leave shared memory
 constexpr int kPubMinK = 128;              // from this k on the scan CTAs share thresholds (ScanParams::pub)
+constexpr int kGmaxSlots = 4;              // groups per warp in a sample launch by maxima (ScanParams::gmax_slots)
 
 int align_up(int v, int a) { return (v + a - 1) / a * a; }
 
@@ -99,7 +101,7 @@ cudaError_t device_alloc(T **ptr, size_t bytes) {
 }
 
 // Shared-memory layout of one scan CTA. Returns false if not even two stages fit.
-bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl) {
+bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl, bool maxima = false) {
     // warp-MMA tiles are 16 rows (the M of m16n8k16). The FMA flavour is bound by its
     // arithmetic, so it wants many small tiles: several being scored while more are in flight.
     pl->nwarps = mma ? kMaxConsumerWarps : kMaxConsumerWarps - 1;
@@ -135,6 +137,8 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl)
         // (they are touched rarely) and only the scratch they are sorted in stays here
         pl->spill = s_pass * pl->cap * 8 > kSmemCandBytes && idx->spill && pl->cap <= idx->spill_cap;
         off += (pl->spill ? 1 : s_pass) * pl->cap * 8;
+    } else if (maxima) {
+        off += kMaxConsumerWarps * kGmaxSlots * kScanMaxPassQueries * 8;  // the warps' best keys (ScanParams::gmax)
     }
     pl->off_stage = align_up(off, 128);
     const int room = idx->smem_optin - pl->off_stage;
@@ -453,7 +457,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
         const int per_pass = std::min(kTcMaxQueries, idx->tc_cand_q);
         idx->last_kernel = idx->variant == 4 ? 4 : 3;
         idx->last_passes = (s + per_pass - 1) / per_pass;
-        idx->last_phases = two_phase ? 2 : 1;
+        idx->last_phases = two_phase ? 3 : 1;
         idx->last_sample_rows = two_phase ? sample : 0;
         for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
             const int sp = std::min(per_pass, s - q0);
@@ -514,10 +518,16 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     sample = (sample + 255) / 256 * 256;
     // (two more launches: only worth it when the scan itself takes a millisecond or more)
     const bool two_phase = (k > 1 || use_q8) && idx->tc_thr && idx->tc_two_phase && sample * 32 <= idx->N;
+    // large k: the sample launch only takes per-warp maxima (needs the stored norms for L2, and as
+    // many warps in the sample launch as k asks for)
+    const bool maxima_sample = two_phase && mma && k >= kPubMinK && idx->scan_gmax &&
+                               (idx->metric == RALM_IP || idx->norms) &&
+                               k <= std::min<long long>(idx->num_sms, sample / 16) * 4 * kGmaxSlots &&
+                               idx->num_sms * kMaxConsumerWarps * kGmaxSlots <= kMaximaSortMax;
     int grid = 0;
     idx->last_kernel = use_q8 ? 5 : (mma ? 2 : 1);
     idx->last_passes = (s + per_pass - 1) / per_pass;
-    idx->last_phases = two_phase ? 2 : 1;
+    idx->last_phases = two_phase ? (maxima_sample ? 3 : 2) : 1;
     idx->last_sample_rows = two_phase ? sample : 0;
     for (int q0 = 0; idx->N > 0 && q0 < s; q0 += per_pass) {
         const int sp = std::min(per_pass, s - q0);
@@ -531,6 +541,9 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
         p.sqnorms = nullptr;
         p.pub = nullptr;
         p.pub_rank = 0;
+        p.gmax = nullptr;
+        p.gmax_slots = 1;
+        p.gmax_len = 0;
         p.ext = index_extents(idx, idx->spill ? static_cast<long long>(idx->num_sms) * kScanMaxPassQueries * idx->spill_cap : 0);
         p.spill = pl.spill ? idx->spill : nullptr;
         p.partial = idx->partial;
@@ -588,6 +601,44 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             return idx->metric == RALM_L2 ? launch_fma<true>(p, g, pl.smem_bytes, st)
                                           : launch_fma<false>(p, g, pl.smem_bytes, st);
         };
+        // Sample launch for large k: the k == 1 kernels over rows [0, end), every consumer warp writing
+        // the best rank value of its rows (ScanParams::gmax); then the k-th largest of a query's maxima
+        // becomes its threshold. No lists, no merge: a fraction of what the sample costs otherwise at
+        // k = 1024 (1.1 ms of scan and 0.3 ms of merge on 50 M x 1024).
+        auto sample_by_maxima = [&](long long end) -> cudaError_t {
+            ScanPlan ps;
+            if (!plan_scan(idx, true, sp, 1, &ps, true)) return cudaErrorUnknown;
+            ScanParams q = p;
+            q.spill = nullptr;
+            q.k = 1;
+            q.cap = 0;
+            q.soft_limit = 0;
+            q.tile_rows = ps.tile_rows;
+            q.nwarps = ps.nwarps;
+            q.depth = ps.depth;
+            q.stage_bytes = ps.stage_bytes;
+            q.off_q = ps.off_q;
+            q.off_cand = ps.off_cand;
+            q.off_stage = ps.off_stage;
+            q.row_begin = 0;
+            q.N = end;
+            q.thr_init = nullptr;
+            q.ntiles = (end + ps.tile_rows - 1) / ps.tile_rows;
+            q.gmax = idx->scan_gmax;
+            q.gmax_slots = kGmaxSlots;
+            q.gmax_len = static_cast<long long>(idx->num_sms) * kMaxConsumerWarps * kGmaxSlots * idx->max_s;
+            const int g = static_cast<int>(std::min<long long>(idx->num_sms, (end + 15) / 16));
+            cudaError_t ke;
+            if (idx->metric == RALM_L2 && sp > kScanMaxQueries) ke = launch_scan<true, true, 16, 1, true, true>(q, g, ps.smem_bytes, st);
+            else if (idx->metric == RALM_L2) ke = launch_scan<true, true, 8, 1, true, true>(q, g, ps.smem_bytes, st);
+            else if (sp > 16) ke = launch_scan<true, false, 32, 1, true>(q, g, ps.smem_bytes, st);
+            else if (sp > kScanMaxQueries) ke = launch_scan<true, false, 16, 1, true>(q, g, ps.smem_bytes, st);
+            else ke = launch_scan<true, false, 8, 1, true>(q, g, ps.smem_bytes, st);
+            if (ke != cudaSuccess) return ke;
+            kth_of_maxima_kernel<<<sp, kMergeThreads, 0, st>>>(idx->scan_gmax + q0, g * ps.nwarps * kGmaxSlots, s, k,
+                                                               idx->tc_thr + q0);
+            return cudaGetLastError();
+        };
         auto scan_rows_q8 = [&](long long begin, long long end, const float *thr_init, int *grid_out) -> cudaError_t {
             ScanParams p8 = p;
             p8.x8 = idx->x8;
@@ -628,7 +679,12 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
         cudaError_t e;
         TimedEvents ev{nullptr, nullptr};
         if (!timing_begin(idx, st, &ev)) return RALM_ERR_CUDA;
-        if (use_q8) {
+        if (maxima_sample) {
+            // (the scan proper then covers every row, the sample's too)
+            e = sample_by_maxima(sample);
+            if (e == cudaSuccess) e = use_q8 ? scan_rows_q8(0, idx->N, idx->tc_thr, &grid) : scan_rows(0, idx->N, idx->tc_thr, &grid);
+            idx->launches += 2;
+        } else if (use_q8) {
             if (two_phase) {
                 int grid1 = 0;
                 e = scan_rows(0, sample, nullptr, &grid1);
@@ -662,7 +718,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
         idx->launches++;
     }
     merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, idx->metric == RALM_L2, ids, scores,
-                                              nullptr, nullptr, two_phase ? idx->num_sms : -1);
+                                              nullptr, nullptr, (two_phase && !maxima_sample) ? idx->num_sms : -1);
     if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
     idx->launches++;
     return RALM_OK;
@@ -779,6 +835,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->spill = nullptr;
     idx->spill_cap = 0;
     idx->pub = nullptr;
+    idx->scan_gmax = nullptr;
     cudaError_t first_error = cudaSuccess;
     auto alloc = [&first_error](auto **ptr, size_t bytes) {
         if (first_error == cudaSuccess) first_error = device_alloc(ptr, bytes);
@@ -792,6 +849,8 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
         alloc(&idx->spill, sizeof(uint64_t) * idx->num_sms * kScanMaxPassQueries * static_cast<size_t>(idx->spill_cap));
     }
     if (max_k >= kPubMinK) alloc(&idx->pub, sizeof(uint32_t) * idx->num_sms * static_cast<size_t>(max_s));
+    if (max_k >= kPubMinK)
+        alloc(&idx->scan_gmax, sizeof(float) * idx->num_sms * kMaxConsumerWarps * kGmaxSlots * static_cast<size_t>(max_s));
     if (metric == RALM_L2 && N > 0) alloc(&idx->norms, sizeof(float) * N);
     ScanPlan probe;
     const bool small_scan_fits = plan_scan(idx, true, kScanMaxQueries, 1, &probe);
@@ -845,6 +904,7 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
     cudaFree(idx->x8_bound);
     cudaFree(idx->spill);
     cudaFree(idx->pub);
+    cudaFree(idx->scan_gmax);
     cudaFree(idx->status);
     cudaFree(idx->h_queries);
     cudaFree(idx->h_ids);
@@ -1075,6 +1135,7 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.spill = nullptr;
     view.spill_cap = 0;
     view.pub = nullptr;
+    view.scan_gmax = nullptr;
     view.norms = nullptr;  // no index, no stored norms: the scan derives them on the tensor cores
     view.x8 = nullptr;
     view.x8_bound = nullptr;

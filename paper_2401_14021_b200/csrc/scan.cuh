@@ -83,6 +83,17 @@ struct ScanParams {
     // rows, and every CTA may raise its threshold to it. Null: off.
     uint32_t *pub;
     int pub_rank;
+    // Sample launch for large k (TOP1 instantiations only): instead of one best key per CTA and
+    // query, every consumer warp writes the best rank value among ITS rows to
+    // gmax[group * s_total + q_base + q] (-inf: it saw no row). The warps'
+    // rows are disjoint, so the k-th largest of a query's maxima is reached by k different rows.
+    // A warp keeps gmax_slots groups, taking its tiles in turn, so that a launch has
+    // gridDim.x * nwarps * gmax_slots of them (large k needs many more groups than k for the
+    // threshold to be tight): group (blockIdx.x * nwarps + warp) * gmax_slots + slot.
+    // The bests live in shared memory at off_cand (nwarps x gmax_slots x 32 keys). Null: off.
+    float *gmax;
+    int gmax_slots;
+    long long gmax_len;  // elements of gmax (debug build)
     Extents ext;     // extents of the global arrays, for the debug build's checks
 };
 
@@ -328,6 +339,9 @@ scan_kernel(const ScanParams p) {
         hdr->cnt[threadIdx.x] = 0;
         hdr->best[threadIdx.x] = 0ull;
     }
+    if (TOP1 && p.gmax)
+        for (int i = threadIdx.x; i < p.nwarps * p.gmax_slots * kScanMaxPassQueries; i += blockDim.x)
+            reinterpret_cast<unsigned long long *>(smem + p.off_cand)[i] = 0ull;
     if (MMA) {
         // queries as fp16 [8][d] in shared memory, rows >= s zeroed; rows are padded by
         // kQueryPadBytes so that the eight query rows do not all start on the same bank
@@ -477,6 +491,12 @@ scan_kernel(const ScanParams p) {
         }
 
         const int ph_lo = staged_row(g), ph_hi = staged_row(g + 8);
+        // k == 1: where the best key of every query is kept: the CTA's, or (sample launch for large
+        // k, see ScanParams::gmax) this warp's own
+        unsigned long long *const warp_bests =
+            reinterpret_cast<unsigned long long *>(smem + p.off_cand) + w * p.gmax_slots * kScanMaxPassQueries;
+        unsigned long long *bestq = (TOP1 && p.gmax) ? warp_bests : hdr->best;
+        int gslot = 0;
         int slot = 0;         // position in this warp's private ring
         uint32_t parity = 0;  // phase parity of the ring's current lap
         long long row0 =
@@ -539,6 +559,21 @@ scan_kernel(const ScanParams p) {
             const uint32_t stage_addr =
                 smem_u32(smem + p.off_stage + static_cast<size_t>(st) * p.stage_bytes);
             const uint32_t empty_bar = smem_u32(&hdr->empty[st]);
+            if (TOP1 && p.gmax) {
+                // sample launch by maxima: this tile's rows count for the warp's next group
+                if (MMA && !L2) {
+#pragma unroll
+                    for (int grp = 0; grp < NG; ++grp) {
+                        const int gq = grp * kScanMaxQueries + 2 * t;
+                        if (bestA[grp]) atomicMax(&bestq[gq], static_cast<unsigned long long>(bestA[grp]));
+                        if (bestB[grp]) atomicMax(&bestq[gq + 1], static_cast<unsigned long long>(bestB[grp]));
+                        bestA[grp] = bestB[grp] = 0;
+                    }
+                }
+                __syncwarp();
+                bestq = warp_bests + gslot * kScanMaxPassQueries;
+                if (++gslot == p.gmax_slots) gslot = 0;
+            }
             if (MMA) {
                 // ---- 16 rows x 8 queries on tensor cores; two accumulator sets halve the
                 // dependent chain. For L2 two more products per step, rows x rows, put the
@@ -610,8 +645,8 @@ scan_kernel(const ScanParams p) {
                         const int gq0 = grp * kScanMaxQueries + q0, gq1 = gq0 + 1;
                         float th0, th1;
                         if (TOP1) {
-                            const unsigned long long b0 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[gq0]);
-                            const unsigned long long b1 = *reinterpret_cast<volatile unsigned long long *>(&hdr->best[gq1]);
+                            const unsigned long long b0 = *reinterpret_cast<volatile unsigned long long *>(&bestq[gq0]);
+                            const unsigned long long b1 = *reinterpret_cast<volatile unsigned long long *>(&bestq[gq1]);
                             th0 = b0 ? key_value(b0) : -INFINITY;
                             th1 = b1 ? key_value(b1) : -INFINITY;
                         } else {
@@ -638,7 +673,7 @@ scan_kernel(const ScanParams p) {
                                     const float val = 0.0f - dist;
                                     const uint64_t key = make_key(val, static_cast<uint32_t>(row0 + row_local));
                                     if (TOP1) {
-                                        atomicMax(&hdr->best[q], static_cast<unsigned long long>(key));
+                                        atomicMax(&bestq[q], static_cast<unsigned long long>(key));
                                     } else if (val >= *reinterpret_cast<volatile float *>(&hdr->thr[q])) {
                                         push_candidate(hdr, cand, p.cap, p.soft_limit, q, key, p.status, list_room);
                                     }
@@ -756,17 +791,28 @@ scan_kernel(const ScanParams p) {
 #pragma unroll
                 for (int grp = 0; grp < NG; ++grp) {
                     const int gq = grp * kScanMaxQueries + 2 * t;
-                    if (bestA[grp]) atomicMax(&hdr->best[gq], static_cast<unsigned long long>(bestA[grp]));
-                    if (bestB[grp]) atomicMax(&hdr->best[gq + 1], static_cast<unsigned long long>(bestB[grp]));
+                    if (bestA[grp]) atomicMax(&bestq[gq], static_cast<unsigned long long>(bestA[grp]));
+                    if (bestB[grp]) atomicMax(&bestq[gq + 1], static_cast<unsigned long long>(bestB[grp]));
                 }
             } else {
                 const int jq = (lane >> 1) % SQR;
-                if (bestA[0]) atomicMax(&hdr->best[jq], static_cast<unsigned long long>(bestA[0]));
+                if (bestA[0]) atomicMax(&bestq[jq], static_cast<unsigned long long>(bestA[0]));
             }
-            named_barrier(1, cthreads);
-            if (ctid < p.s && in_bounds(static_cast<long long>(blockIdx.x) * p.s_total + p.q_base + ctid, p.ext.partial, p.status))
-                p.partial[static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + ctid] =
-                    hdr->best[ctid];
+            if (p.gmax) {
+                // this warp's maxima, group by group (lane q writes query q's)
+                __syncwarp();
+                for (int sl = 0; sl < p.gmax_slots; ++sl) {
+                    const unsigned long long best = warp_bests[sl * kScanMaxPassQueries + lane];
+                    const long long at = ((static_cast<long long>(blockIdx.x) * W + w) * p.gmax_slots + sl) * p.s_total +
+                                         p.q_base + lane;
+                    if (lane < p.s && in_bounds(at, p.gmax_len, p.status)) p.gmax[at] = best ? key_value(best) : -INFINITY;
+                }
+            } else {
+                named_barrier(1, cthreads);
+                if (ctid < p.s && in_bounds(static_cast<long long>(blockIdx.x) * p.s_total + p.q_base + ctid, p.ext.partial, p.status))
+                    p.partial[static_cast<size_t>(blockIdx.x) * p.s_total + p.q_base + ctid] =
+                        hdr->best[ctid];
+            }
         } else {
             // this warp is out of tiles; keep answering compaction calls until every warp is
             __syncwarp();
