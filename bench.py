@@ -384,6 +384,18 @@ def main():
     dispatch = idx.last_dispatch()
     idx.set_timing(False)
     gpu_launches = idx.launch_count() - launches0 + args.steps   # + one verify launch per step
+    # the whole search call by itself (scan launches, threshold kernel and merges), a few times
+    n_search = max(3, min(20, args.steps))
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record(stream)
+    for _ in range(n_search):
+        if sharded is None:
+            ralm.search(idx, queries, k, ids, scores, stream)
+        else:
+            sharded.search(queries, k, stream)
+    s1.record(stream)
+    torch.cuda.synchronize()
+    search_ms = s0.elapsed_time(s1) / n_search
     if sharded is not None:
         gpu_launches += 3 * args.steps                           # cache score + rank on the cached vectors, merge_lists
     assert idx.device_status() == 0, "device status word set during the timed region"
@@ -512,6 +524,7 @@ def main():
                              "corpus near L2 size: L2-warm figure, not an HBM number"},
             "scan_gbs": corpus_bytes / (scan_avg_ms * 1e-3) / 1e9 if scan_launches else None,
             "scan_ms": scan_avg_ms, "scan_median_ms": scan_median_ms, "scan_passes_per_step": passes,
+            "search_ms": search_ms,
             "roofline": roofline,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},

@@ -87,7 +87,7 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx);
 
 /* C.retrieve(q_1..q_s): exact top-k of s queries over the whole corpus, one stream of the
  * corpus from HBM per pass (up to 32 queries on the small-batch scan, up to 512 on the
- * large-batch scan, which takes over from 17 inner-product or 9 L2 queries on large corpora).
+ * large-batch scan, which takes over from 9 queries on large corpora, 17 for inner product with k == 1).
  *   queries DEVICE fp16 [s][d], 16-byte aligned.     0 <= s <= max_s
  *   ids     DEVICE int64 [s][k]  (written)           1 <= k <= max_k
  *   scores  DEVICE fp32  [s][k]  (written)
@@ -205,17 +205,17 @@ ralm_status_t ralm_device_status(ralm_index_t *idx, void *stream);
  *   value only filters and the ranked distance is the direct sum of squared differences), 3 = tcgen05 scan (up to 512 queries per pass, k <= 256,
  *   d >= 64; pairs of CTAs share each MMA; for L2 the tensor-core value again only filters,
  *   and the corpus must be large enough to scan a sample first, about 600 K rows), 4 = tcgen05
- *   scan with single CTAs. Automatic: warp-MMA up to 16 queries (inner product; 32 on corpora
- *   too small for a sample launch, about 600 K rows) or 8 (L2), the tcgen05 scan beyond that
- *   where it applies.
+ *   scan with single CTAs. Automatic: warp-MMA up to 16 queries (inner product, k == 1; up to 8
+ *   for k > 1; 32 on corpora too small for a sample launch, about 600 K rows) or 8 (L2), the
+ *   tcgen05 scan beyond that where it applies.
  * UNSUPPORTED if the variant cannot serve the index's metric or dimension. The environment
  * variable RALM_FORCE_VARIANT=<1..4> applies the same pin to every index at creation. */
 ralm_status_t ralm_index_set_variant(ralm_index_t *idx, int32_t variant);
 
 /* Optional: build a one-byte-per-element copy of the corpus (E5M2, N * d bytes, plus one fp32
  * bound per row) that ralm_search then streams instead of the fp16 rows for batches of up to 8
- * queries (any k the index allows) and of 9..16 queries with k <= 64, under the automatic variant
- * (other shapes take the fp16 scans). The copy only
+ * queries (any k the index allows) and of 9..16 queries with k == 1 (k <= 64 when forced), under
+ * the automatic variant (other shapes take the fp16 scans). The copy only
  * FILTERS: by the Cauchy-Schwarz inequality the inner product with the rounded row is within
  * |q| * |x - x8| of the true one, which bounds the score (inner product) or, with the rows' stored
  * squared norms, the squared distance (L2) from the right side; a (row, query) pair whose bound

@@ -421,10 +421,12 @@ ralm_status_t launch_tc_pass(ralm_index *idx, const __half *queries, int sp, int
 
 constexpr int kTcAutoMinQueries = 9;     // batches the 8-query scan cannot serve in one pass
 // From how many queries the automatic variant takes the tcgen05 scan (measured on 21 M x 768 and
-// 50 M x 1024): inner product 24 queries 4.6 against 5.3 ms for the four-group warp-MMA pass, 16
-// queries 4.7 against 4.3-4.7; L2 9 queries 14.9 against 16.4 ms. On corpora too small for a sample
-// launch the small-batch scan keeps batches of up to 32 inner-product queries.
-constexpr int kTcAutoMinQueriesIp = 17;
+// 50 M x 1024): inner product, k = 1: 16 queries 4.42 against 4.34 ms for the two-group warp-MMA
+// pass, 24 queries 4.44 against 5.3 ms; k = 20: 12 queries 4.42 against 4.74 ms; L2 9 queries 14.9
+// against 16.4 ms. On corpora too small for a sample launch the small-batch scan keeps batches of
+// up to 32 inner-product queries.
+constexpr int kTcAutoMinQueriesIp = 17;      // k == 1
+constexpr int kTcAutoMinQueriesIpTopK = 9;   // k > 1
 constexpr int kTcAutoMinQueriesIpSmall = 33;
 constexpr int kTcAutoMinQueriesL2 = 9;
 
@@ -442,11 +444,13 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     tc_sample = (tc_sample + tc_rows - 1) / tc_rows * tc_rows;
     const bool tc_two_phase = tc_sample * 8 <= idx->N && idx->tc_two_phase;
     const bool l2 = idx->metric == RALM_L2;
-    const bool tc = tc_can_serve(idx, k) && (!l2 || tc_two_phase) &&
-                    (idx->variant == 3 || idx->variant == 4 ||
-                     (idx->variant == 0 &&
-                      (s >= (l2 ? kTcAutoMinQueriesL2 : (tc_two_phase ? kTcAutoMinQueriesIp : kTcAutoMinQueriesIpSmall)) ||
-                       (!small_scan_fits && !l2))));
+    // (L2 rows too long for the small-batch scan take this path on any corpus: without a sample
+    // every pair passes the filter and is scored again, which is slow but small corpora are small)
+    const int tc_from = l2 ? kTcAutoMinQueriesL2
+                           : (tc_two_phase ? (k > 1 ? kTcAutoMinQueriesIpTopK : kTcAutoMinQueriesIp) : kTcAutoMinQueriesIpSmall);
+    const bool tc_auto = !small_scan_fits || ((tc_two_phase || !l2) && s >= tc_from);
+    const bool tc = tc_can_serve(idx, k) && (!l2 || tc_two_phase || !small_scan_fits) &&
+                    (idx->variant == 3 || idx->variant == 4 || (idx->variant == 0 && tc_auto));
     if (tc) {
         // Large corpora are scanned in two phases: a small sample first, which gives every query a
         // score that k rows are known to reach; the scan proper then starts from those thresholds,
@@ -482,7 +486,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
                                         l2 ? 2 : 0, &grid, st);
                 idx->launches += 2;
             } else {
-                rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, idx->N, nullptr, 0, &grid, st);
+                rs = launch_tc_pass(idx, qp, sp, s, q0, k, idx->variant != 4, 0, idx->N, nullptr, l2 ? 2 : 0, &grid, st);
             }
             timing_end(idx, st, ev);
             if (rs != RALM_OK) return rs;
@@ -507,7 +511,9 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     ScanPlan pl8;
     // (only where a sample phase is possible: without thresholds nearly every pair passes the filter)
     const long long q8_sample = (std::max<long long>(idx->N / 128, 4LL * idx->num_sms * kTcTileM) + 255) / 256 * 256;
+    // (two query groups only pay at k == 1: 16 queries 3.6 ms against 4.3; at k = 20 4.8 against 4.7 fp16)
     const bool use_q8 = idx->x8 && (idx->metric == RALM_IP || idx->norms) && idx->variant == 0 && s <= kQ8MaxQueries &&
+                        (s <= kScanMaxQueries || k == 1 || idx->x8_force) &&
                         (idx->x8_force || (idx->tc_thr && idx->tc_two_phase && q8_sample * 32 <= idx->N)) &&
                         plan_scan_q8(idx, s, k, &pl8);
     const int per_pass = use_q8 ? kQ8MaxQueries : mma ? (wide ? wide_pass : kScanMaxQueries) : kFmaQueriesPerPass;
@@ -854,7 +860,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     if (metric == RALM_L2 && N > 0) alloc(&idx->norms, sizeof(float) * N);
     ScanPlan probe;
     const bool small_scan_fits = plan_scan(idx, true, kScanMaxQueries, 1, &probe);
-    if ((max_s >= kTcAutoMinQueries || (!small_scan_fits && metric == RALM_IP)) && d >= kTcChunkK &&
+    if ((max_s >= kTcAutoMinQueries || !small_scan_fits) && d >= kTcChunkK &&
         first_error == cudaSuccess &&
         !alloc_tc_workspace(idx, std::min(kTcMaxQueries, align_up(max_s, 16))))
         first_error = cudaErrorMemoryAllocation;

@@ -774,10 +774,19 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         // TMA and the tensor core keep it busy (440 against 100 cycles per block of 32 queries).
         // tl: thresholds (main launches; reloaded after a compaction meeting, the only place where
         // they move). qnl: |q|^2 (L2). best: running maxima of a sample launch.
-        float tl[2][kTcMaxN / 32], qnl[2][kTcMaxN / 32];
+        float tl[2][kTcMaxN / 32], qnl[2][kTcMaxN / 32], al[2][kTcMaxN / 32];
         uint32_t best[2][kTcMaxN / 32];
+        const float wide_slack = p.slack * 1.001f + 1.0f / 1048576.0f;
         tc_load_lane_thresholds(tl, thr, p.nb, p.nhalves, lane);
         if (l2) tc_load_lane_thresholds(qnl, qn, p.nb, p.nhalves, lane);
+        // L2 main launch: the per-query side of the filter, thr / 2 + (1 - slack) |q|^2 / 2
+        auto refresh_rhs = [&]() {
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int j = 0; j < kTcMaxN / 32; ++j) al[h][j] = fmaf(0.5f * (1.0f - wide_slack), qnl[h][j], 0.5f * tl[h][j]);
+        };
+        if (l2 && !sample) refresh_rhs();
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -824,6 +833,8 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                        static_cast<uint32_t>(acc * kTcMaxN);
                 const float nx = (l2 && row_ok && in_bounds(row, p.ext.rows, p.status)) ? __ldg(p.norms + row) : 0.f;
+                // L2: this row's part of the bound (see below)
+                const float row_part = sample ? 0.0f - (1.0f + wide_slack) * nx : 0.0f - 0.5f * (1.0f - wide_slack) * nx;
 #pragma unroll
                 for (int j = 0; j < kTcMaxN / 32; ++j) {
                     if (j * 32 < nq) {
@@ -831,32 +842,32 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         tmem_ld32(t_row + j * 32, v);
                         if (sample) {
                             if (l2) {
-                                // the LOWER bound of -distance^2 (see TcParams::mode)
-                                const float my_qn = half ? qnl[1][j] : qnl[0][j];
+                                // the part of the LOWER bound of -distance^2 that depends on the row:
+                                // 2 x.q - (1 + slack) |x|^2; the query's part is subtracted at the end
 #pragma unroll
-                                for (int c = 0; c < 32; ++c) {
-                                    const float s2 = nx + __shfl_sync(0xffffffffu, my_qn, c);
-                                    const float val = fmaf(2.0f, __uint_as_float(v[c]), 0.0f - s2);
-                                    v[c] = __float_as_uint(fmaf(0.0f - p.slack, s2, val));
-                                }
+                                for (int c = 0; c < 32; ++c)
+                                    v[c] = __float_as_uint(fmaf(2.0f, __uint_as_float(v[c]), row_part));
                             }
                             if (half) tc_fold_block_maxima(v, row_ok, best[1][j], lane);
                             else tc_fold_block_maxima(v, row_ok, best[0][j], lane);
                         } else if (l2) {
-                            // the UPPER bound of -distance^2 against the thresholds
-                            const float my_thr = half ? tl[1][j] : tl[0][j];
-                            const float my_qn = half ? qnl[1][j] : qnl[0][j];
-                            bool p0 = false, p1 = false;
+                            // the UPPER bound of -distance^2 against the thresholds, rearranged so that
+                            // the common path costs what the inner-product one does:
+                            //   2 x.q - (1 - slack)(|x|^2 + |q|^2) >= thr
+                            //   <=>  x.q - (1 - slack)|x|^2 / 2  >=  thr / 2 + (1 - slack)|q|^2 / 2
+                            // (left: per row, right: per query, by shuffle from the lane that holds it;
+                            // the slack used here is a little larger than the append routine's, so
+                            // the rearrangement's own rounding cannot drop a pair that routine keeps)
+                            const float my_rhs = half ? al[1][j] : al[0][j];
+                            bool p0 = false, p1 = false, p2 = false, p3 = false;
 #pragma unroll
-                            for (int c = 0; c < 32; c += 2) {
-                                const float s0 = nx + __shfl_sync(0xffffffffu, my_qn, c);
-                                const float s1 = nx + __shfl_sync(0xffffffffu, my_qn, c + 1);
-                                p0 |= fmaf(p.slack, s0, fmaf(2.0f, __uint_as_float(v[c]), 0.0f - s0)) >=
-                                      __shfl_sync(0xffffffffu, my_thr, c);
-                                p1 |= fmaf(p.slack, s1, fmaf(2.0f, __uint_as_float(v[c + 1]), 0.0f - s1)) >=
-                                      __shfl_sync(0xffffffffu, my_thr, c + 1);
+                            for (int i = 0; i < 8; ++i) {
+                                p0 |= __uint_as_float(v[4 * i + 0]) + row_part >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 0);
+                                p1 |= __uint_as_float(v[4 * i + 1]) + row_part >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 1);
+                                p2 |= __uint_as_float(v[4 * i + 2]) + row_part >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 2);
+                                p3 |= __uint_as_float(v[4 * i + 3]) + row_part >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 3);
                             }
-                            if (__any_sync(0xffffffffu, row_ok && (p0 | p1)))
+                            if (__any_sync(0xffffffffu, row_ok && (p0 | p1 | p2 | p3)))
                                 tc_append_chunk_l2(t_row + j * 32, thr + qb + j * 32, qn + qb + j * 32, cnt + qb + j * 32,
                                                    my_cand + static_cast<size_t>(qb + j * 32) * p.cap,
                                                    static_cast<uint32_t>(row), row_ok, nx, p.slack, p.corpus,
@@ -925,6 +936,7 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 }
                 named_barrier(1, 128);  // thresholds and counts settled before the next unit's pushes
                 tc_load_lane_thresholds(tl, thr, p.nb, p.nhalves, lane);
+                if (l2) refresh_rhs();
             }
         }
         if (sample) {
@@ -937,7 +949,9 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     const int q = h * p.nb + j * 32 + lane;
                     if (h < p.nhalves && j * 32 < p.nb && q < p.s &&
                         in_bounds((static_cast<long long>(blockIdx.x) * 4 + ew) * p.s_total + p.q_base + q, p.ext.aux, p.status))
-                        dst[q] = best[h][j] ? from_ordered_bits(best[h][j]) : -INFINITY;
+                        dst[q] = !best[h][j] ? -INFINITY
+                                 : l2    ? __fmaf_rd(0.0f - (1.0f + wide_slack), qnl[h][j], from_ordered_bits(best[h][j]))
+                                         : from_ordered_bits(best[h][j]);
                 }
         } else {
             // ---- CTA result: every list sorted and cut to k, written as this CTA's partial lists

@@ -286,16 +286,21 @@ def test_tcgen05_scan_adversarial_row_order():
 
 
 def test_long_rows_take_the_tcgen05_scan_even_for_small_batches():
-    """d = 4096: two 16-row stages of the small-batch scan do not fit in shared memory; inner
-    product indexes then use the large-batch scan (64 columns per stage) for any batch size."""
+    """d = 4096: two 16-row stages of the small-batch scan do not fit in shared memory; the index
+    then uses the large-batch scan (64 columns per stage) for any batch size, both metrics."""
     ralm = _ralm()
     x = workloads.integer_valued((900, 4096), seed=91, lo=-3, hi=3, device=DEV)
     q = workloads.integer_valued((3, 4096), seed=92, lo=-3, hi=3, device=DEV)
     ids, scores = _run(x, q, oracle.IP, 4)
     check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, 4, exact=True)
-    idx = ralm.Index(x, oracle.L2, 3, 4)                   # L2 has no such route yet
-    with pytest.raises(ralm.RalmError):
-        ralm.search(idx, q, 4)
+    q[0] = x[17]                                           # L2: a zero-distance copy comes first
+    ids, scores = _run(x, q, oracle.L2, 4)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.L2, 4, exact=True)
+    x2, _ = workloads.mixture_corpus(3000, 3072, 16, seed=97, device=DEV, normalise=False, lognormal_sigma=0.3)
+    q2, src = workloads.noisy_copy_queries(x2, 5, seed=98)
+    ids, scores = _run(x2, q2, oracle.L2, 10)
+    check_search(ids, scores, x2.cpu().numpy(), q2.cpu().numpy(), oracle.L2, 10)
+    assert ids[:, 0].tolist() == src.tolist()
 
 
 def test_largest_batch_and_k_limits_of_the_tcgen05_scan():
