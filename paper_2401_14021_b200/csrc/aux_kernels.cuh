@@ -8,6 +8,16 @@ namespace ralm {
 
 constexpr int kMergeThreads = 1024;
 constexpr int kMergeSortMax = 4096;  // keys sorted in one go when all lists fit
+constexpr int kMergeSelectMaxK = 32;  // up to this k, and from kMergeSelectMin keys on, the merge
+constexpr int kMergeSelectMin = 256;  // selects the k largest keys one by one instead of sorting
+
+// Largest 64-bit key of the warp, in every lane (two 32-bit warp reductions).
+__device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
+    const uint32_t hi = static_cast<uint32_t>(v >> 32);
+    const uint32_t top = __reduce_max_sync(0xffffffffu, hi);
+    const uint32_t lo = __reduce_max_sync(0xffffffffu, hi == top ? static_cast<uint32_t>(v) : 0u);
+    return (static_cast<uint64_t>(top) << 32) | lo;
+}
 
 __device__ __forceinline__ void write_result(uint64_t key, bool l2, int64_t *id_out,
                                              float *score_out) {
@@ -48,62 +58,140 @@ kth_of_maxima_kernel(const float *__restrict__ vals, int G, int stride, int k, f
 }
 
 // ------------------------------------------------------------------------------------
-// Merge: one CTA per query. `partial` holds B lists of k keys, each sorted descending and
-// padded with 0, laid out [B][s][k]. Writes ids [s][k] (int64) and scores [s][k] (fp32).
+// Merge: one CTA per query (and, with gridDim.y > 1, per group of lists). `partial` holds B lists
+// of k keys, each sorted descending and padded with 0, laid out [B][s][k]. Writes ids [s][k]
+// (int64) and scores [s][k] (fp32).
 // ------------------------------------------------------------------------------------
 // extra_slot >= 0: one more list takes part, stored at that block index of `partial`.
-// With keys_out the merged list is written as keys [s][k] instead (and the k-th value, or -inf
-// when there are fewer than k rows, to thr_out[q]): the result of scanning a sample of the
-// corpus, which seeds the thresholds of the main scan and rejoins the final merge as one more
-// partial list.
+// With keys_out the merged list is written as keys instead, at keys_out[(blockIdx.y * s + q) * k]
+// (and, with thr_out, the k-th value, or -inf when there are fewer than k rows, to thr_out[q]):
+// the result of scanning a sample of the corpus, which seeds the thresholds of the main scan and
+// rejoins the final merge as one more partial list; or the first level of a two-level merge,
+// where CTA (q, y) merges the y-th of gridDim.y equal groups of the lists (few queries and long
+// lists leave a single level with a handful of CTAs that each walk through every list).
 __global__ void __launch_bounds__(kMergeThreads, 1)
 merge_kernel(const uint64_t *__restrict__ partial, int B, int s, int k, int l2,
              int64_t *__restrict__ ids, float *__restrict__ scores, uint64_t *__restrict__ keys_out = nullptr,
              float *__restrict__ thr_out = nullptr, int extra_slot = -1) {
     __shared__ uint64_t buf[kMergeSortMax];
+    __shared__ uint64_t warp_best[2][32];
+    __shared__ int kept;
     const int q = blockIdx.x;
     const int tid = threadIdx.x;
-    const int lists = B + (extra_slot >= 0 ? 1 : 0);
+    const int lane = tid & 31, warp = tid >> 5;
+    const int all_lists = B + (extra_slot >= 0 ? 1 : 0);
+    const int per_group = (all_lists + gridDim.y - 1) / gridDim.y;
+    const int first = blockIdx.y * per_group;
+    const int lists = max(min(all_lists - first, per_group), 0);
+    auto list_at = [&](int b) -> const uint64_t * {   // the b-th list of this CTA's group, query q
+        b += first;
+        return partial + (static_cast<size_t>(b < B ? b : extra_slot) * s + q) * k;
+    };
     const long long total = static_cast<long long>(lists) * k;
-    if (total <= kMergeSortMax) {
+    if (total <= kMergeSortMax && total > kMergeSelectMin && k <= kMergeSelectMaxK) {
+        // Many short lists (148 lists of 20 keys): k rounds of "take the largest key left" over
+        // keys held in registers cost a fraction of sorting all of them (a 4096-key bitonic
+        // sort is 78 passes with a barrier each). Keys are distinct: a row is in one list only.
+        uint64_t mine[kMergeSortMax / kMergeThreads];
+#pragma unroll
+        for (int j = 0; j < kMergeSortMax / kMergeThreads; ++j) {
+            const int i = tid + j * kMergeThreads;
+            mine[j] = 0;
+            if (i < total) {
+                const int b = i / k;
+                mine[j] = list_at(b)[i - b * k];
+            }
+        }
+        for (int r = 0; r < k; ++r) {
+            uint64_t m = mine[0];
+#pragma unroll
+            for (int j = 1; j < kMergeSortMax / kMergeThreads; ++j) m = mine[j] > m ? mine[j] : m;
+            m = warp_max_u64(m);
+            if (lane == 0) warp_best[r & 1][warp] = m;
+            __syncthreads();   // (two buffers: a warp is at most one round ahead of another)
+            const uint64_t winner = warp_max_u64(warp_best[r & 1][lane]);
+#pragma unroll
+            for (int j = 0; j < kMergeSortMax / kMergeThreads; ++j)
+                if (mine[j] == winner) mine[j] = 0;
+            if (tid == 0) buf[r] = winner;
+        }
+        __syncthreads();
+    } else if (total <= kMergeSortMax) {
         const int P = next_pow2(total > 1 ? static_cast<int>(total) : 2);
         for (int i = tid; i < P; i += kMergeThreads) {
             uint64_t key = 0;
             if (i < total) {
                 const int b = i / k, j = i - b * k;
-                const int slot = b < B ? b : extra_slot;
-                key = partial[(static_cast<size_t>(slot) * s + q) * k + j];
+                key = list_at(b)[j];
             }
             buf[i] = key;
         }
         __syncthreads();
         bitonic_sort_desc(buf, P, tid, kMergeThreads, -1);
     } else {
-        // running best list merged with one sorted list at a time: the element-wise maximum
-        // of a descending list and a reversed descending list holds the best P keys of both
-        // and is bitonic
-        const int P = next_pow2(k);
-        const int slot0 = B > 0 ? 0 : extra_slot;
-        for (int i = tid; i < P; i += kMergeThreads)
-            buf[i] = (i < k) ? partial[(static_cast<size_t>(slot0) * s + q) * k + i] : 0ull;
+        // Long lists. The largest k-th key of any one list is reached by that list's k keys, so
+        // nothing below it can be among the best k of all: keep the keys from that value up
+        // (with rows dealt to the CTAs in turn that is little more than k keys) and sort them.
+        uint64_t m = 0;
+        for (int b = tid; b < lists; b += kMergeThreads) {
+            const uint64_t last = list_at(b)[k - 1];
+            m = last > m ? last : m;
+        }
+        m = warp_max_u64(m);
+        if (lane == 0) warp_best[0][warp] = m;
+        if (tid == 0) kept = 0;
         __syncthreads();
-        for (int b = 1; b < lists; ++b) {
-            const uint64_t *list = partial + (static_cast<size_t>(b < B ? b : extra_slot) * s + q) * k;
-            for (int i = tid; i < P; i += kMergeThreads) {
-                const int j = P - 1 - i;
-                const uint64_t other = (j < k) ? list[j] : 0ull;
-                const uint64_t mine = buf[i];
-                buf[i] = mine > other ? mine : other;
+        const uint64_t cut = warp_max_u64(warp_best[0][lane]);
+        bool sorted = false;
+        if (cut != 0ull) {   // (0: no list is full, every key would pass)
+            for (int b = warp; b < lists; b += kMergeThreads / 32) {
+                const uint64_t *list = list_at(b);
+                for (int j0 = 0; j0 < k; j0 += 32) {   // descending: the first key below the cut ends the list
+                    const uint64_t key = (j0 + lane < k) ? list[j0 + lane] : 0ull;
+                    if (key >= cut) {
+                        const int at = atomicAdd(&kept, 1);
+                        if (at < kMergeSortMax) buf[at] = key;
+                    }
+                    if (__any_sync(0xffffffffu, key < cut)) break;
+                }
             }
             __syncthreads();
-            bitonic_merge_desc(buf, P, tid, kMergeThreads, -1);
+            const int n = kept;
+            if (n <= kMergeSortMax) {
+                const int P = next_pow2(n > 1 ? n : 2);
+                for (int i = n + tid; i < P; i += kMergeThreads) buf[i] = 0ull;
+                __syncthreads();
+                bitonic_sort_desc(buf, P, tid, kMergeThreads, -1);
+                sorted = true;
+            }
+            __syncthreads();
+        }
+        if (!sorted) {
+            // running best list merged with one sorted list at a time: the element-wise maximum
+            // of a descending list and a reversed descending list holds the best P keys of both
+            // and is bitonic
+            const int P = next_pow2(k);
+            const uint64_t *list0 = list_at(0);
+            for (int i = tid; i < P; i += kMergeThreads) buf[i] = (i < k) ? list0[i] : 0ull;
+            __syncthreads();
+            for (int b = 1; b < lists; ++b) {
+                const uint64_t *list = list_at(b);
+                for (int i = tid; i < P; i += kMergeThreads) {
+                    const int j = P - 1 - i;
+                    const uint64_t other = (j < k) ? list[j] : 0ull;
+                    const uint64_t mine = buf[i];
+                    buf[i] = mine > other ? mine : other;
+                }
+                __syncthreads();
+                bitonic_merge_desc(buf, P, tid, kMergeThreads, -1);
+            }
         }
     }
     for (int i = tid; i < k; i += kMergeThreads) {
         const uint64_t key = (i < total) ? buf[i] : 0ull;
         if (keys_out) {
-            keys_out[static_cast<size_t>(q) * k + i] = key;
-            if (i == k - 1) thr_out[q] = key ? key_value(key) : -INFINITY;
+            keys_out[(static_cast<size_t>(blockIdx.y) * s + q) * k + i] = key;
+            if (thr_out && i == k - 1) thr_out[q] = key ? key_value(key) : -INFINITY;
         } else {
             write_result(key, l2 != 0, ids + static_cast<size_t>(q) * k + i,
                          scores + static_cast<size_t>(q) * k + i);

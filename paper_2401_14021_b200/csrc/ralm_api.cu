@@ -32,6 +32,7 @@ struct ralm_index {
     int tune_warps, tune_depth, tune_rows;  // 0 = library default
     uint64_t *partial;   // [num_sms][max_s][max_k]
     long long partial_keys;  // keys the array holds
+    uint64_t *merge_tmp;   // two-level final merge: [kMergeGroups][kMergeTwoLevelMaxS][max_k] keys, or null
     uint64_t *cache_keys;  // [RALM_MAX_CACHE_KEYS]
     uint64_t *spill;       // large k: candidate lists of the small-batch scan, [num_sms][8][spill_cap]
     int spill_cap;
@@ -73,6 +74,8 @@ struct ScanPlan {
 constexpr int kSmemCandBytes = 32 * 1024;  // candidate lists larger than this leave shared memory
 constexpr int kPubMinK = 128;              // from this k on the scan CTAs share thresholds (ScanParams::pub)
 constexpr int kGmaxSlots = 4;              // groups per warp in a sample launch by maxima (ScanParams::gmax_slots)
+constexpr int kMergeGroups = 16;           // two-level final merge: groups of lists merged side by side first
+constexpr int kMergeTwoLevelMaxS = 16;     // ... for batches up to this size (larger ones have CTAs enough)
 
 int align_up(int v, int a) { return (v + a - 1) / a * a; }
 
@@ -430,6 +433,30 @@ constexpr int kTcAutoMinQueriesIpTopK = 9;   // k > 1
 constexpr int kTcAutoMinQueriesIpSmall = 33;
 constexpr int kTcAutoMinQueriesL2 = 9;
 
+// Final merge of `lists` partial lists per query into ids and scores. One CTA per query walks
+// through its lists one after the other; with few queries and long lists (4 queries, 148 lists of
+// 1024 keys: 0.33 ms) the lists are first merged in kMergeGroups groups side by side, then the
+// groups' results.
+ralm_status_t final_merge(ralm_index *idx, int lists, int s, int k, bool l2, int64_t *ids, float *scores,
+                          int extra_slot, cudaStream_t st) {
+    const int all_lists = lists + (extra_slot >= 0 ? 1 : 0);
+    if (idx->merge_tmp && s <= kMergeTwoLevelMaxS && all_lists >= 4 * kMergeGroups &&
+        static_cast<long long>(all_lists) * k > kMergeSortMax) {
+        merge_kernel<<<dim3(s, kMergeGroups), kMergeThreads, 0, st>>>(idx->partial, lists, s, k, l2 ? 1 : 0, nullptr, nullptr,
+                                                                   idx->merge_tmp, nullptr, extra_slot);
+        if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
+        merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->merge_tmp, kMergeGroups, s, k, l2 ? 1 : 0, ids, scores, nullptr,
+                                                  nullptr, -1);
+        if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
+        idx->launches += 2;
+        return RALM_OK;
+    }
+    merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, lists, s, k, l2 ? 1 : 0, ids, scores, nullptr, nullptr, extra_slot);
+    if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
+    idx->launches++;
+    return RALM_OK;
+}
+
 ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k, int64_t *ids,
                             float *scores, cudaStream_t st) {
     if (s == 0) return RALM_OK;
@@ -492,10 +519,7 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
             if (rs != RALM_OK) return rs;
             idx->launches++;
         }
-        merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, l2 ? 1 : 0, ids, scores, nullptr, nullptr, -1);
-        if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
-        idx->launches++;
-        return RALM_OK;
+        return final_merge(idx, grid, s, k, l2, ids, scores, -1, st);
     }
     const int variant = resolve_variant(idx);
     const bool mma = variant == 2;
@@ -723,11 +747,8 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
         if (e != cudaSuccess) return RALM_ERR_CUDA;
         idx->launches++;
     }
-    merge_kernel<<<s, kMergeThreads, 0, st>>>(idx->partial, grid, s, k, idx->metric == RALM_L2, ids, scores,
-                                              nullptr, nullptr, (two_phase && !maxima_sample) ? idx->num_sms : -1);
-    if (cudaGetLastError() != cudaSuccess) return RALM_ERR_CUDA;
-    idx->launches++;
-    return RALM_OK;
+    return final_merge(idx, grid, s, k, idx->metric == RALM_L2, ids, scores,
+                       (two_phase && !maxima_sample) ? idx->num_sms : -1, st);
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -842,6 +863,7 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     idx->spill_cap = 0;
     idx->pub = nullptr;
     idx->scan_gmax = nullptr;
+    idx->merge_tmp = nullptr;
     cudaError_t first_error = cudaSuccess;
     auto alloc = [&first_error](auto **ptr, size_t bytes) {
         if (first_error == cudaSuccess) first_error = device_alloc(ptr, bytes);
@@ -849,6 +871,8 @@ ralm_status_t ralm_index_create(const void *corpus, int64_t N, int32_t d, ralm_m
     alloc(&idx->partial, partial_bytes);
     idx->partial_keys = static_cast<long long>(partial_bytes / sizeof(uint64_t));
     alloc(&idx->tc_thr, sizeof(float) * max_s);
+    if (static_cast<long long>(idx->num_sms + 1) * max_k > kMergeSortMax)
+        alloc(&idx->merge_tmp, sizeof(uint64_t) * kMergeGroups * kMergeTwoLevelMaxS * static_cast<size_t>(max_k));
     const int pass_queries = std::min(max_s, kScanMaxPassQueries);
     if (max_k > 1 && std::max(512, 2 * next_pow2(max_k)) * 8 * pass_queries > kSmemCandBytes) {
         idx->spill_cap = std::max(512, 2 * next_pow2(max_k));
@@ -901,6 +925,7 @@ ralm_status_t ralm_index_destroy(ralm_index_t *idx) {
     if (!idx) return RALM_OK;
     cudaFree(idx->partial);
     cudaFree(idx->cache_keys);
+    cudaFree(idx->merge_tmp);
     cudaFree(idx->tc_cand);
     cudaFree(idx->tc_thr);
     cudaFree(idx->tc_gmax);
@@ -1130,6 +1155,7 @@ ralm_status_t ralm_search_static(const void *corpus, int64_t N, int32_t d, ralm_
     view.partial = dev->partial;
     view.partial_keys = static_cast<long long>(RALM_STATIC_MAX_BLOCKS) * RALM_STATIC_MAX_S * RALM_STATIC_MAX_K;
     view.cache_keys = nullptr;
+    view.merge_tmp = nullptr;
     view.tc_cand = nullptr;
     view.tc_cand_q = 0;
     view.tc_cand_cap = 0;

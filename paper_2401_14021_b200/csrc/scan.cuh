@@ -561,7 +561,7 @@ scan_kernel(const ScanParams p) {
             const uint32_t empty_bar = smem_u32(&hdr->empty[st]);
             if (TOP1 && p.gmax) {
                 // sample launch by maxima: this tile's rows count for the warp's next group
-                if (MMA && !L2) {
+                if (MMA) {
 #pragma unroll
                     for (int grp = 0; grp < NG; ++grp) {
                         const int gq = grp * kScanMaxQueries + 2 * t;
@@ -640,6 +640,32 @@ scan_kernel(const ScanParams p) {
                         n_hi = __shfl_sync(0xffffffffu, d_hi, diag_lane);
                     }
                     const float sl = p.l2_slack;
+                    if (TOP1 && p.gmax) {
+                        // Sample launch by maxima: the filter value minus its slack is a LOWER bound
+                        // of the rank value the direct form would give, and a threshold only has to
+                        // be a value that k different rows are known to reach. So nothing is scored
+                        // again here: the warp keeps the best lower bound per query and group (the
+                        // slack is widened a little to cover the rounding of these few operations).
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(empty_bar);
+                        const float ws = fmaf(sl, 1.001f, 9.5367431640625e-7f);
+#pragma unroll
+                        for (int grp = 0; grp < NG; ++grp) {
+                            const float a0 = qn0[grp], a1 = qn1[grp];
+                            if (r_lo < p.N) {
+                                const uint64_t k0 = make_key(fmaf(-ws, n_lo + a0, (2.f * acc[grp][0] - n_lo) - a0), static_cast<uint32_t>(r_lo));
+                                const uint64_t k1 = make_key(fmaf(-ws, n_lo + a1, (2.f * acc[grp][1] - n_lo) - a1), static_cast<uint32_t>(r_lo));
+                                bestA[grp] = k0 > bestA[grp] ? k0 : bestA[grp];
+                                bestB[grp] = k1 > bestB[grp] ? k1 : bestB[grp];
+                            }
+                            if (r_hi < p.N) {
+                                const uint64_t k0 = make_key(fmaf(-ws, n_hi + a0, (2.f * acc[grp][2] - n_hi) - a0), static_cast<uint32_t>(r_hi));
+                                const uint64_t k1 = make_key(fmaf(-ws, n_hi + a1, (2.f * acc[grp][3] - n_hi) - a1), static_cast<uint32_t>(r_hi));
+                                bestA[grp] = k0 > bestA[grp] ? k0 : bestA[grp];
+                                bestB[grp] = k1 > bestB[grp] ? k1 : bestB[grp];
+                            }
+                        }
+                    } else {
 #pragma unroll
                     for (int grp = 0; grp < NG; ++grp) {
                         const int gq0 = grp * kScanMaxQueries + q0, gq1 = gq0 + 1;
@@ -683,6 +709,7 @@ scan_kernel(const ScanParams p) {
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(empty_bar);
+                    }
                 } else {
 #pragma unroll
                 for (int grp = 0; grp < NG; ++grp) {
@@ -787,7 +814,7 @@ scan_kernel(const ScanParams p) {
         // ------------------------------------------------------------ CTA result
         if (TOP1) {
             if (MMA) {
-                // (the L2 flavour has put its keys into hdr->best as it went)
+                // (the L2 flavour of a main launch has put its keys into hdr->best as it went)
 #pragma unroll
                 for (int grp = 0; grp < NG; ++grp) {
                     const int gq = grp * kScanMaxQueries + 2 * t;

@@ -272,6 +272,33 @@ def test_small_batch_scan_two_phases_integer_inputs(metric):
             check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), metric, k, exact=True)
 
 
+@pytest.mark.parametrize("N,d,s,k", [(1600, 32, 4, 64), (1040, 32, 3, 100), (5000, 64, 16, 300), (5000, 64, 17, 300),
+                                     (2_500_003, 16, 5, 64), (2_500_003, 16, 2, 1024)])
+def test_final_merge_of_long_lists_integer_inputs(N, d, s, k):
+    """Lists too long to sort in one go: the merge keeps the keys from the largest k-th key of any
+    list up and sorts those; up to 16 queries the partial lists are first merged in 16 groups side
+    by side, then the groups' results. 100 and 65 lists leave the last groups short or empty;
+    2.5 M rows with k = 64 add the sample phase's list as one more."""
+    x = workloads.integer_valued((N, d), seed=1700 + k, lo=-2, hi=2, device=DEV)
+    q = workloads.integer_valued((s, d), seed=1701 + k, lo=-2, hi=2, device=DEV)
+    for metric in (oracle.IP, oracle.L2):
+        ids, scores = _run(x, q, metric, k)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), metric, k, exact=True)
+
+
+@pytest.mark.parametrize("s", [3, 20])
+def test_final_merge_of_long_lists_rows_sorted_by_score(s):
+    """Scores rising along the corpus: every CTA's list reaches far down, more keys pass the
+    merge's cut than it can sort at once, and it merges the lists one after the other instead."""
+    N, d, k = 60_000, 64, 300
+    x = torch.zeros((N, d), dtype=torch.float16, device=DEV)
+    x[:, 0] = (torch.arange(N, device=DEV) // 32).to(torch.float16)
+    q = torch.zeros((s, d), dtype=torch.float16, device=DEV)
+    q[:, 0] = torch.arange(1, s + 1, device=DEV).to(torch.float16) * torch.where(torch.arange(s, device=DEV) % 2 == 0, 1.0, -1.0)
+    ids, scores = _run(x, q, oracle.IP, k)
+    check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+
+
 def test_tcgen05_scan_adversarial_row_order():
     """Scores increase along the corpus: every row passes every threshold, so every unit ends
     in a compaction of every list."""

@@ -82,3 +82,61 @@ def test_speculate_verify_update_schedule():
     assert np.mean(matched_per_round[-4:]) > 0.6               # warm caches: most speculations match
     assert max(strides[4:]) > 1                                # and the scheduler lengthens the stride
     print("strides", strides, "matched fraction", [round(v, 2) for v in matched_per_round])
+
+
+def test_serving_step_replays_from_a_cuda_graph():
+    """The whole retrieval step (cache lookup, batched search, verify, cache update) issues only
+    stream-ordered work, so it can be captured once in a CUDA graph and replayed with new queries
+    in the same buffers, which is how a launch-bound serving loop would run it. Every replay is
+    compared with the oracle, integer-valued data so that ids and scores are exact."""
+    import paper_2401_14021_b200 as ralm
+    from oracle.cache_update import cache_update as oracle_cache_update
+    N, d, R, C, k, stride = 60_000, 64, 4, 64, 5, 4
+    x = workloads.integer_valued((N, d), seed=1801, lo=-3, hi=3, device=DEV)
+    xn = x.cpu().numpy()
+    idx = ralm.Index(x, ralm.IP, max_s=R * stride, max_k=k)
+    q = torch.zeros((R, stride, d), dtype=torch.float16, device=DEV)
+    cache = torch.full((R, C), -1, dtype=torch.int64, device=DEV)
+    cursor = torch.zeros((R,), dtype=torch.int32, device=DEV)
+    spec = torch.empty((R, stride, 1), dtype=torch.int64, device=DEV)
+    spec_scores = torch.empty((R, stride, 1), dtype=torch.float32, device=DEV)
+    ids = torch.empty((R * stride, k), dtype=torch.int64, device=DEV)
+    scores = torch.empty((R * stride, k), dtype=torch.float32, device=DEV)
+    first_mismatch = torch.empty((R,), dtype=torch.int32, device=DEV)
+
+    def step(st):
+        ralm.cache_search(idx, cache, q, 1, spec, spec_scores, st)
+        ralm.search(idx, q.view(R * stride, d), k, ids, scores, st)
+        ralm.verify(spec.view(R, stride), ids.view(R, stride, k), 1, first_mismatch, st)
+        ralm.cache_update(cache, cursor, ids.view(R, stride, k), k, N, stream=st)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step(side)                                   # first use outside the capture (module load)
+    side.synchronize()
+    cache.fill_(-1)
+    cursor.zero_()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+        step(torch.cuda.current_stream())
+    o_cache, o_cursor = cache.cpu().numpy(), cursor.cpu().numpy()
+    for t in range(3):
+        # (the third round repeats the first round's queries: their documents are cached by then)
+        q.copy_(workloads.integer_valued((R, stride, d), seed=1810 + t % 2, lo=-3, hi=3, device=DEV))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert idx.device_status() == 0
+        qn = q.cpu().numpy()
+        o_spec, _ = oracle.cache_search(xn, o_cache, qn, oracle.IP, 1)
+        o_ids, o_scores = oracle.search(xn, qn.reshape(R * stride, d), oracle.IP, k)
+        o_m = oracle.verify(o_spec.reshape(R, stride), o_ids.reshape(R, stride, k))
+        o_cache, o_cursor = oracle_cache_update(o_cache, o_cursor, o_ids.reshape(R, stride, k), k, N=N)
+        assert np.array_equal(spec.cpu().numpy(), o_spec)
+        assert np.array_equal(ids.cpu().numpy(), o_ids)
+        assert np.array_equal(scores.cpu().numpy(), o_scores.astype(np.float32))
+        assert np.array_equal(first_mismatch.cpu().numpy(), o_m)
+        assert np.array_equal(cache.cpu().numpy(), o_cache)
+        assert np.array_equal(cursor.cpu().numpy(), o_cursor)
+    assert o_m.max() > 0                          # the repeated queries found their documents cached
+    idx.close()
