@@ -132,6 +132,8 @@ merge_kernel(const uint64_t *__restrict__ partial, int B, int s, int k, int l2,
         // Long lists. The largest k-th key of any one list is reached by that list's k keys, so
         // nothing below it can be among the best k of all: keep the keys from that value up
         // (with rows dealt to the CTAs in turn that is little more than k keys) and sort them.
+        // Where no list is full (a scan that started from good thresholds leaves each CTA with a
+        // few keys) the cut is 0 and every key held is kept.
         uint64_t m = 0;
         for (int b = tid; b < lists; b += kMergeThreads) {
             const uint64_t last = list_at(b)[k - 1];
@@ -143,22 +145,22 @@ merge_kernel(const uint64_t *__restrict__ partial, int B, int s, int k, int l2,
         __syncthreads();
         const uint64_t cut = warp_max_u64(warp_best[0][lane]);
         bool sorted = false;
-        if (cut != 0ull) {   // (0: no list is full, every key would pass)
+        {
             for (int b = warp; b < lists; b += kMergeThreads / 32) {
                 const uint64_t *list = list_at(b);
                 for (int j0 = 0; j0 < k; j0 += 32) {   // descending: the first key below the cut ends the list
                     const uint64_t key = (j0 + lane < k) ? list[j0 + lane] : 0ull;
-                    if (key >= cut) {
+                    if (key >= cut && key != 0ull) {
                         const int at = atomicAdd(&kept, 1);
                         if (at < kMergeSortMax) buf[at] = key;
                     }
-                    if (__any_sync(0xffffffffu, key < cut)) break;
+                    if (__any_sync(0xffffffffu, key < cut || key == 0ull)) break;
                 }
             }
             __syncthreads();
             const int n = kept;
             if (n <= kMergeSortMax) {
-                const int P = next_pow2(n > 1 ? n : 2);
+                const int P = next_pow2(n > k ? n : (k > 1 ? k : 2));   // (the first k slots are read below)
                 for (int i = n + tid; i < P; i += kMergeThreads) buf[i] = 0ull;
                 __syncthreads();
                 bitonic_sort_desc(buf, P, tid, kMergeThreads, -1);

@@ -638,7 +638,13 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             // a pair splits the N of this unit's MMA, not nb: the follower supplies the upper
             // half of the (rounded) queries this half really has
             const int nq_u = (p.s - half * p.nb < p.nb) ? (p.s - half * p.nb) : p.nb;
-            const int query_y = half * p.nb + (PAIR ? static_cast<int>(rank) * (((nq_u + 31) & ~31) / 2) : 0);
+            int query_y = half * p.nb + (PAIR ? static_cast<int>(rank) * (((nq_u + 31) & ~31) / 2) : 0);
+            // With 16 queries or fewer in this half the follower's rows all lie beyond the last
+            // query. A box that is out of range as a whole costs far more than its zeros are
+            // worth (measured: the whole launch up to 20 % slower, depending on where the query
+            // buffer sits), so the follower then stages the leader's rows once more: those
+            // columns of the product belong to absent queries, which never pass.
+            if (PAIR && query_y >= p.s) query_y = half * p.nb;
             for (int c = 0; c < nchunks; c += SC) {
                 const int kc = (nchunks - c < SC) ? (nchunks - c) : SC;
                 ok = tc_wait(smem_u32(&hdr->empty[st]), (lap & 1) ^ 1, abort_flag);
