@@ -129,21 +129,24 @@ merge_kernel(const uint64_t *__restrict__ partial, int B, int s, int k, int l2,
         __syncthreads();
         bitonic_sort_desc(buf, P, tid, kMergeThreads, -1);
     } else {
-        // Long lists. The largest k-th key of any one list is reached by that list's k keys, so
-        // nothing below it can be among the best k of all: keep the keys from that value up
-        // (with rows dealt to the CTAs in turn that is little more than k keys) and sort them.
-        // Where no list is full (a scan that started from good thresholds leaves each CTA with a
-        // few keys) the cut is 0 and every key held is kept.
-        uint64_t m = 0;
-        for (int b = tid; b < lists; b += kMergeThreads) {
-            const uint64_t last = list_at(b)[k - 1];
-            m = last > m ? last : m;
+        // Long lists. If m lists each hold r keys from some value up, m * r >= k keys reach that
+        // value and nothing below it can be among the best k of all. So: take every list's r-th
+        // key, r = ceil(2k / lists); the m-th largest of them, m = ceil(k / r), is such a value
+        // (the cut). Rows are dealt to the CTAs in turn, so about 2k keys lie above it: those are
+        // kept and sorted at once. Where fewer than m lists hold r keys the cut is 0 and every key
+        // is kept (a scan that started from good thresholds leaves each CTA with a few keys).
+        const int r = min(k, max(1, (2 * k + lists - 1) / lists));
+        const int m = (k + r - 1) / r;
+        uint64_t cut = 0ull;
+        if (lists <= kMergeSortMax) {
+            const int P = next_pow2(lists > 1 ? lists : 2);
+            for (int b = tid; b < P; b += kMergeThreads) buf[b] = (b < lists) ? list_at(b)[r - 1] : 0ull;
+            __syncthreads();
+            bitonic_sort_desc(buf, P, tid, kMergeThreads, -1);
+            cut = (m <= lists) ? buf[m - 1] : 0ull;
         }
-        m = warp_max_u64(m);
-        if (lane == 0) warp_best[0][warp] = m;
         if (tid == 0) kept = 0;
         __syncthreads();
-        const uint64_t cut = warp_max_u64(warp_best[0][lane]);
         bool sorted = false;
         {
             for (int b = warp; b < lists; b += kMergeThreads / 32) {
