@@ -865,13 +865,21 @@ scan_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                             // the slack used here is a little larger than the append routine's, so
                             // the rearrangement's own rounding cannot drop a pair that routine keeps)
                             const float my_rhs = half ? al[1][j] : al[0][j];
+                            // (the row's part is added two columns per instruction)
+                            const float2 row_part2 = make_float2(row_part, row_part);
+#pragma unroll
+                            for (int c = 0; c < 32; c += 2) {
+                                const float2 t = __fadd2_rn(make_float2(__uint_as_float(v[c]), __uint_as_float(v[c + 1])), row_part2);
+                                v[c] = __float_as_uint(t.x);
+                                v[c + 1] = __float_as_uint(t.y);
+                            }
                             bool p0 = false, p1 = false, p2 = false, p3 = false;
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {
-                                p0 |= __uint_as_float(v[4 * i + 0]) + row_part >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 0);
-                                p1 |= __uint_as_float(v[4 * i + 1]) + row_part >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 1);
-                                p2 |= __uint_as_float(v[4 * i + 2]) + row_part >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 2);
-                                p3 |= __uint_as_float(v[4 * i + 3]) + row_part >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 3);
+                                p0 |= __uint_as_float(v[4 * i + 0]) >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 0);
+                                p1 |= __uint_as_float(v[4 * i + 1]) >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 1);
+                                p2 |= __uint_as_float(v[4 * i + 2]) >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 2);
+                                p3 |= __uint_as_float(v[4 * i + 3]) >= __shfl_sync(0xffffffffu, my_rhs, 4 * i + 3);
                             }
                             if (__any_sync(0xffffffffu, row_ok && (p0 | p1 | p2 | p3)))
                                 tc_append_chunk_l2(t_row + j * 32, thr + qb + j * 32, qn + qb + j * 32, cnt + qb + j * 32,
