@@ -57,6 +57,10 @@ def parse_args():
     ap.add_argument("--rows", type=int, default=None, help="override the corpus size (profiling)")
     ap.add_argument("--tune", default=None, help="consumer_warps,ring_depth,tile_rows (0 = default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture one step (cache lookup, search, verify) in a CUDA graph and replay it in the "
+                         "timed region, as a launch-bound serving loop would (small corpora); the scan's own "
+                         "events are then taken from plain steps after the timed region")
     ap.add_argument("--flush-l2", action="store_true",
                     help="write a buffer larger than L2 before every timed step (for corpora near L2 size); "
                          "the step time is then the sum of per-step event intervals, flushes excluded")
@@ -332,10 +336,10 @@ def main():
     retr_view = ids[:nv * vstride].reshape(nv, vstride, k)
 
     if sharded is None:
-        def step():
-            ralm.cache_search(idx, cache, cache_q, 1, spec_ids, spec_scores, stream)
-            ralm.search(idx, queries, k, ids, scores, stream)
-            ralm.verify(spec_view, retr_view, 1, first_mismatch, stream)
+        def step(st=stream):
+            ralm.cache_search(idx, cache, cache_q, 1, spec_ids, spec_scores, st)
+            ralm.search(idx, queries, k, ids, scores, st)
+            ralm.verify(spec_view, retr_view, 1, first_mismatch, st)
     else:
         spec_local = torch.empty((R, stride, 1), dtype=torch.int64, device=device)
 
@@ -354,7 +358,20 @@ def main():
         step()
     barrier()
     idx.read_timing()
-    idx.set_timing(True)
+    use_graph = args.graph and sharded is None and flush is None
+    graph = None
+    if use_graph:
+        # (the library's calls only enqueue work on the stream they are given, so a step can be captured)
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side, capture_error_mode="thread_local"):
+            step(torch.cuda.current_stream())
+        stream.wait_stream(side)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+    idx.set_timing(not use_graph)
     launches0 = idx.launch_count()
     sampler = ClockSampler(local_rank)
     time.sleep(0.25)
@@ -363,7 +380,10 @@ def main():
     if flush is None:
         e0.record(stream)
         for _ in range(args.steps):
-            step()
+            if graph is not None:
+                graph.replay()
+            else:
+                step()
         e1.record(stream)
         barrier()
         total_ms = e0.elapsed_time(e1)
@@ -379,6 +399,13 @@ def main():
         barrier()
         total_ms = sum(a.elapsed_time(b) for a, b in pairs)
     clocks = sampler.stop()
+    if graph is not None:
+        # events cannot be read back from a captured step: the scan's own times come from plain steps
+        idx.set_timing(True)
+        launches0 = idx.launch_count()
+        for _ in range(args.steps):
+            step()
+        torch.cuda.synchronize()
     pass_ms = idx.read_timing_list(max(4096, 8 * args.steps))
     scan_ms, scan_launches = sum(pass_ms), len(pass_ms)
     dispatch = idx.last_dispatch()
@@ -515,7 +542,7 @@ def main():
             "config": {"workload": "%s %dx%d %s s=%d k=%d; cache lookup R=%d C=%d q=%d; verify stride %d"
                                    % (cfg.name, N, d, cfg.metric, s, k, R, cache.shape[1], stride, vstride),
                        "arithmetic": "fp16 corpus and queries, exact fp16 x fp16 products, fp32 accumulation",
-                       "variant": args.variant, "tune": args.tune, "q8": bool(args.q8),
+                       "variant": args.variant, "tune": args.tune, "q8": bool(args.q8), "cuda_graph": bool(use_graph),
                        "replicas": 1 if sharded is not None else world,
                        "row_shards": world if sharded is not None else 1,
                        "dispatch": dispatch, "l2_flushed_every_step": bool(args.flush_l2),
