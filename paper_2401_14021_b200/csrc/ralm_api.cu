@@ -467,7 +467,10 @@ ralm_status_t search_device(ralm_index *idx, const __half *queries, int s, int k
     // L2 on this path always runs sample first (the sample is what keeps its exact rescoring
     // rare), so it needs a corpus large enough for one
     const long long tc_rows = 2 * kTcTileM;
-    long long tc_sample = std::max<long long>(idx->N / 64, 4LL * idx->num_sms * kTcTileM);
+    // (a larger sample for large k: the k-th largest of the launch's 4 maxima per CTA is a tighter
+    // threshold when each maximum is taken over more rows, and at k = 256 the rows that still pass
+    // it in the main launch cost more than the longer sample launch)
+    long long tc_sample = std::max<long long>(idx->N / (k > kTcSmallK ? 16 : 64), 4LL * idx->num_sms * kTcTileM);
     tc_sample = (tc_sample + tc_rows - 1) / tc_rows * tc_rows;
     const bool tc_two_phase = tc_sample * 8 <= idx->N && idx->tc_two_phase;
     const bool l2 = idx->metric == RALM_L2;
