@@ -236,6 +236,17 @@ def test_tcgen05_scan_two_phases_integer_inputs():
         for variant in (3, 4):
             ids, scores = _run(x, q, oracle.IP, k, variant)
             check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+    # k > 64: lists of 512 slots, and a sample of 1/16 of the rows once that exceeds the minimum
+    q = workloads.integer_valued((12, d), seed=80, lo=-2, hi=2, device=DEV)
+    for k in (100, 256):
+        ids, scores = _run(x, q, oracle.IP, k, 3)
+        check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
+    x2 = workloads.integer_valued((1_400_003, 32), seed=81, lo=-2, hi=2, device=DEV)
+    q2 = workloads.integer_valued((20, 32), seed=82, lo=-2, hi=2, device=DEV)
+    for metric in (oracle.IP, oracle.L2):
+        ids, scores = _run(x2, q2, metric, 200)
+        check_search(ids, scores, x2.cpu().numpy(), q2.cpu().numpy(), metric, 200, exact=True)
+    del x2
     # L2 on the same scan: the sample launch ranks lower bounds of the tensor-core value, the main
     # launch filters with it and scores what passes in the direct form
     q = workloads.integer_valued((40, d), seed=79, lo=-2, hi=2, device=DEV)
