@@ -125,7 +125,9 @@ bool plan_scan(const ralm_index *idx, bool mma, int s_pass, int k, ScanPlan *pl,
     pl->spill = false;
     if (k > 1) {
         // after the flag is raised every warp may still finish the tile it is on
-        pl->cap = std::max(512, 2 * next_pow2(k));
+        // (256 slots up to k = 64: with 512 the lists of 8 queries take 32 KB of shared memory, one
+        // stage of the ring, and the scan runs on seven consumer warps instead of eight)
+        pl->cap = k <= 64 ? 256 : std::max(512, 2 * next_pow2(k));
         // (a tuned tile height must leave that room: k kept keys plus one tile from every warp)
         const int unit = mma ? 16 : (s_pass == 1 ? 16 : 4);
         const int max_rows = (pl->cap - k) / (kMaxConsumerWarps + 1) / unit * unit;
