@@ -310,6 +310,29 @@ def test_final_merge_of_long_lists_rows_sorted_by_score(s):
     check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), oracle.IP, k, exact=True)
 
 
+@pytest.mark.parametrize("variant,tuning", [(1, (0, 0, 64)), (1, (3, 2, 32)), (2, (4, 1, 0)), (2, (8, 3, 0))])
+def test_tuned_launch_shapes_give_the_same_results(variant, tuning):
+    """Results do not depend on the tuning (consumer warps, ring depth, tile height). The FMA scan
+    with 64-row tiles and k = 256 on a corpus too small for a sample phase is the case where a list
+    could receive more keys between two compactions than it has room for, had the host not cut
+    the tile height back: ids and scores must still equal the oracle's bit for bit and the status
+    word must stay clear."""
+    import paper_2401_14021_b200 as ralm
+    N, d = 30_000, 64
+    x = workloads.integer_valued((N, d), seed=1900, lo=-3, hi=3, device=DEV)
+    for metric in (oracle.IP, oracle.L2):
+        for s, k in ((4, 256), (3, 20), (1, 1)):
+            q = workloads.integer_valued((s, d), seed=1901 + k, lo=-3, hi=3, device=DEV)
+            idx = ralm.Index(x, metric, max_s=s, max_k=k)
+            idx.set_variant(variant)
+            idx.set_tuning(*tuning)
+            ids, scores = ralm.search(idx, q, k)
+            torch.cuda.synchronize()
+            assert idx.device_status() == 0
+            idx.close()
+            check_search(ids, scores, x.cpu().numpy(), q.cpu().numpy(), metric, k, exact=True)
+
+
 def test_tcgen05_scan_adversarial_row_order():
     """Scores increase along the corpus: every row passes every threshold, so every unit ends
     in a compaction of every list."""
